@@ -1,0 +1,197 @@
+/*
+ * tarflow.h -- C ABI of the B200 selective-Jacobi TarFlow sampling library (libtarflow.so).
+ *
+ * The library implements, as hand-written CUDA kernels for sm_100a, the inference hot path of a
+ * TarFlow-style block-autoregressive normalizing flow:
+ *   - the autoregressive affine block and its inverse            (paper Eq. 4 and Eq. 5),
+ *   - Jacobi decoding of a block's inverse                        (paper Algorithm 1, Eq. 8),
+ *   - the selective policy: per block, sequential decoding with a
+ *     key/value cache or Jacobi iteration                         (paper Sec. 3.5),
+ *   - token-order reversal between blocks                         (remark after Eq. 4).
+ * Notation: mu = g_k, alpha = -s_k, so a block's inverse is  u_l = v_l * exp(alpha_l) + mu_l  and
+ * log|det d z / d x| = -sum(alpha).  Blocks are indexed in GENERATION order: block 0 is the first
+ * inverse applied to the noise (the paper's "first (K-th) layer").
+ *
+ * Conventions for every call
+ *   - Pointers named *_dev are device pointers on the current CUDA device, *_host are host
+ *     pointers.  The caller owns every buffer it passes; the library neither frees nor keeps them
+ *     after the call returns.  Images are fp32 [B, C, H, W], contiguous.
+ *   - `cuda_stream` is a cudaStream_t cast to void* (NULL = the legacy default stream).  Work is
+ *     enqueued on it; calls that fill host outputs synchronise that stream before returning.
+ *   - Return value: 0 = TF_OK; TF_MAXITER (1) = a Jacobi block hit max_iters before every sample
+ *     passed the stopping test (x holds the last iterate; not an error); negative = error, with a
+ *     message available from tf_last_error().  Nothing aborts, throws or traps.
+ *   - A tf_model is not thread-safe: it owns one workspace; use it from one thread/stream at a time.
+ */
+#ifndef TARFLOW_H_
+#define TARFLOW_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TF_OK 0
+#define TF_MAXITER 1
+#define TF_EINVAL (-1)     /* bad argument or configuration                       */
+#define TF_ESIZE (-2)      /* weight blob size / header mismatch                  */
+#define TF_ENOMEM (-3)     /* host or device allocation failed                    */
+#define TF_ECUDA (-4)      /* a CUDA runtime/driver call failed                   */
+#define TF_ETIMEOUT (-5)   /* a bounded device-side wait expired                  */
+#define TF_ENONFINITE (-6) /* NaN/Inf reached the convergence reduction           */
+
+typedef struct tf_model tf_model; /* opaque: device weights, KV cache, workspace */
+
+typedef struct {
+  int32_t C, H, W, patch; /* L = (H/patch)*(W/patch) tokens of D = C*patch*patch values         */
+  int32_t n_blocks;       /* K flow blocks                                                      */
+  int32_t n_layers;       /* transformer layers per block                                       */
+  int32_t width;          /* transformer width d (multiple of n_heads; bf16 engine: of 64)      */
+  int32_t n_heads;        /* head_dim = width / n_heads; bf16 engine needs head_dim == 64       */
+  int32_t mlp_ratio;      /* MLP hidden = mlp_ratio * width                                     */
+  int32_t n_classes;      /* 0 = unconditional, else rows of the per-block class embedding      */
+  int32_t dtype;          /* 0 = fp32 SIMT engine, 1 = bf16 tensor-core engine (fp32 accumulate)*/
+  int32_t max_batch;      /* largest B any later call may use (sizes workspace and KV cache)    */
+} tf_config;
+
+/*
+ * tf_load -- build a model from seeded weights (paper Sec. 3.1: the functions s_k, g_k of Eq. 4).
+ *   weights_host: flat little-endian blob: 16 int32 header {magic 0x31574654, version 1, C, H, W,
+ *     patch, n_blocks, n_layers, width, n_heads, mlp_ratio, n_classes, dtype, seed, 0, 0} followed
+ *     by fp32 tensors, block by block (generation order), each block in this order:
+ *       w_in [d,D], b_in [d], pos [L,d], cls [n_classes,d] (only if n_classes>0),
+ *       per layer: ln1_g[d] ln1_b[d] w_qkv[3d,d] b_qkv[3d] w_o[d,d] b_o[d]
+ *                  ln2_g[d] ln2_b[d] w_1[hid,d] b_1[hid] w_2[d,hid] b_2[d],
+ *       lnf_g[d] lnf_b[d] w_out[2D,d] b_out[2D].
+ *     Linear layers are [out_features, in_features] (y = x W^T + b); w_qkv rows are q | k | v;
+ *     w_out rows are mu~ (first D) | alpha~ (last D).  The blob is copied, not retained.
+ *     For dtype 1 the matrices are converted to bf16 (round to nearest even).
+ *   nbytes: size of the blob; must equal the size implied by cfg (else TF_ESIZE); the header
+ *     fields must equal cfg's (else TF_ESIZE).
+ *   out: receives the model.  Allocates all device memory the other calls use.
+ */
+int tf_load(const tf_config* cfg, const void* weights_host, size_t nbytes, tf_model** out);
+
+/* tf_free -- release a model and everything it owns.  tf_free(NULL) is a no-op. */
+void tf_free(tf_model* m);
+
+/*
+ * tf_forward -- data to latent, x -> z, and logdet = -sum(alpha) (paper Eq. 4 applied through
+ * blocks K-1 .. 0, Eq. 1 for the log-determinant).  One causal pass per block, no iteration.
+ *   x_dev [B,C,H,W] in, labels_dev [B] int32 class ids or NULL, z_dev [B,C,H,W] out,
+ *   logdet_dev [B] fp32 out (may be NULL).  1 <= B <= max_batch.  Asynchronous on the stream.
+ */
+int tf_forward(tf_model* m, const float* x_dev, const int32_t* labels_dev, int32_t B, float* z_dev,
+               float* logdet_dev, void* cuda_stream);
+
+/*
+ * tf_inverse_sequential -- latent to data, z -> x, every block decoded token by token with a
+ * key/value cache (paper Eq. 5; the sequential baseline of Sec. 3.5).  L-1 steps per block.
+ */
+int tf_inverse_sequential(tf_model* m, const float* z_dev, const int32_t* labels_dev, int32_t B,
+                          float* x_dev, void* cuda_stream);
+
+/*
+ * tf_inverse_jacobi -- latent to data under a per-block policy (paper Algorithm 1 and Sec. 3.5).
+ *   policy_host [n_blocks], generation order: 0 = sequential with KV cache, 1 = Jacobi.
+ *     The paper's selective policy is {0,1,1,...}; uniform Jacobi is all ones.
+ *   tau >= 0: a sample leaves a Jacobi block after the first sweep whose
+ *     max over all its L*D entries of |u^t - u^{t-1}| <= tau (per-sample test; converged samples
+ *     are dropped from later sweeps).  tau < 0: fixed-iteration mode, exactly max_iters sweeps.
+ *   max_iters >= 1: sweep cap per Jacobi block (L sweeps reproduce sequential decoding exactly,
+ *     Prop. 3.2; passing the test on an exact iterate can need sweep L+1).
+ *   init_mode: 0 = u^0 = 0 (Algorithm 1);  1 = u^0 = v (the block's input);  other values EINVAL.
+ *   x_dev [B,C,H,W] out.
+ *   iters_block_host [n_blocks] out (may be NULL): sweeps executed by a Jacobi block (max over
+ *     samples, counting the passing sweep); L-1 for a sequential block.
+ *   iters_sample_dev [n_blocks, B] int32 out (may be NULL): the same per sample.
+ *   Synchronises the stream before returning.
+ */
+int tf_inverse_jacobi(tf_model* m, const float* z_dev, const int32_t* labels_dev, int32_t B,
+                      const uint8_t* policy_host, float tau, int32_t max_iters, int32_t init_mode,
+                      float* x_dev, int32_t* iters_block_host, int32_t* iters_sample_dev,
+                      void* cuda_stream);
+
+/*
+ * tf_inverse_jacobi_host -- the same operation for callers that hold host memory: copies z (and
+ * labels) to the device, runs tf_inverse_jacobi, copies x back.  z_host/x_host [B,C,H,W] fp32,
+ * labels_host [B] or NULL; pinned host memory makes the copies asynchronous.  iters_sample_host
+ * [n_blocks,B] may be NULL.  Synchronises before returning.
+ */
+int tf_inverse_jacobi_host(tf_model* m, const float* z_host, const int32_t* labels_host, int32_t B,
+                           const uint8_t* policy_host, float tau, int32_t max_iters,
+                           int32_t init_mode, float* x_host, int32_t* iters_block_host,
+                           int32_t* iters_sample_host, void* cuda_stream);
+
+/*
+ * tf_jacobi_update -- the fused step of Algorithm 1 on its own: given the un-shifted head output
+ * o_dev [B, L, 2D] = (mu~ | alpha~) of one causal pass, the block input v_dev [B,L,D] and the
+ * previous iterate u_dev [B,L,D] (updated in place), set u_1 = v_1, u_l = v_l * exp(alpha~_{l-1})
+ * + mu~_{l-1}, and write maxdiff_dev[b] = max |u^t - u^{t-1}| over sample b.  `reversed` != 0
+ * applies the block permutation (core position l is raster position L-1-l).  Asynchronous.
+ */
+int tf_jacobi_update(const float* o_dev, const float* v_dev, float* u_dev, float* maxdiff_dev,
+                     int32_t B, int32_t L, int32_t D, int32_t reversed, void* cuda_stream);
+
+/*
+ * tf_gemm_bf16 -- the tensor-core GEMM used by every projection of a sweep, exposed for tests and
+ * profiling:  C[M,N] (fp32, row-major) = A[M,K] (bf16 row-major) * W[N,K]^T (bf16 row-major) +
+ * bias[N] (fp32, may be NULL).  K % 64 == 0, N % 8 == 0, pointers 16-byte aligned.  Asynchronous:
+ * a device-side wait that expired is reported by tf_gemm_status.
+ */
+int tf_gemm_bf16(const void* a_dev, const void* w_dev, const float* bias_dev, float* c_dev,
+                 int32_t M, int32_t N, int32_t K, void* cuda_stream);
+
+/* tf_gemm_status -- synchronise `cuda_stream` and report whether any tf_gemm_bf16 launch so far
+ * gave up on a bounded device-side wait (TF_ETIMEOUT) or all completed (TF_OK). */
+int tf_gemm_status(void* cuda_stream);
+
+/*
+ * Profiling aid: when enabled, calls on this model bracket every kernel class with CUDA events on
+ * the caller's stream and accumulate elapsed milliseconds and launch counts.
+ *   tf_profile_enable(m, on): switch on/off and reset the counters.
+ *   tf_profile_read(m, names, ms, launches, cap): fills up to cap entries, returns how many
+ *     classes exist; names[i] points to a static string.
+ *   tf_launch_count(m): kernels launched by the library on this model since load (always counted).
+ */
+int tf_profile_enable(tf_model* m, int32_t on);
+int tf_profile_read(tf_model* m, const char** names, double* ms, int64_t* launches, int32_t cap);
+int64_t tf_launch_count(tf_model* m);
+
+/*
+ * tf_set_precision -- operand precision of Jacobi sweeps on the bf16 engine (no effect on fp32).
+ * With single bf16 operands the rounding of activations puts a floor of a few 1e-3 under
+ * max|u^t - u^{t-1}|, so the stopping test of Algorithm 1 cannot pass for a smaller tau.  In the
+ * two-term mode every activation operand is a bf16 pair (hi + lo, about 16 significant bits) and
+ * every product keeps the leading cross terms; the tensor-core work of such a sweep roughly doubles.
+ *   mode 0 (default): per sample, sweeps use single operands until that sample's max|du| drops to
+ *     switch_threshold, two-term operands afterwards; used only when 0 <= tau < single_ok_tau.
+ *   mode 1: single operands always.   mode 2: two-term operands for every Jacobi sweep.
+ *   switch_threshold / single_ok_tau <= 0 select the defaults 2^-5 and 2^-6.
+ * Fixed-iteration mode (tau < 0) uses single operands unless mode is 2.
+ */
+int tf_set_precision(tf_model* m, int32_t mode, float switch_threshold, float single_ok_tau);
+
+/*
+ * Convergence trace (paper Fig. "Convergence dynamics of Jacobi decoding", and the stopping test of
+ * Algorithm 1): when enabled, every Jacobi sweep of later tf_inverse_jacobi calls records
+ * (block, sweep number, samples active in that sweep, max over those samples of
+ * max|u^t - u^{t-1}|).  Enabling it makes every sweep synchronise, also in fixed-iteration mode.
+ *   tf_trace_read fills up to cap records of the last call and returns how many exist.
+ */
+int tf_trace_enable(tf_model* m, int32_t on);
+int tf_trace_read(tf_model* m, int32_t* block, int32_t* sweep, int32_t* active, float* maxdiff,
+                  int32_t cap);
+
+/* tf_device_bytes -- device memory owned by the model (weights + workspace + KV cache), bytes. */
+int64_t tf_device_bytes(tf_model* m);
+
+/* tf_last_error -- message of the last failing call on this thread ("" if none). */
+const char* tf_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TARFLOW_H_ */

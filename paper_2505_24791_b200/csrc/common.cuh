@@ -1,0 +1,47 @@
+// Shared device/host helpers for the TarFlow selective-Jacobi kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+typedef __nv_bfloat16 bf16;
+
+// Device error word (one per model, in global memory).  A kernel that gives up on a bounded wait
+// stores a non-zero code here and returns; the host reads it at the next synchronising call.
+enum : int {
+  TFERR_NONE = 0,
+  TFERR_WAIT_FULL = 1,        // MMA warp: operand stage never arrived
+  TFERR_WAIT_EMPTY = 2,       // TMA warp: stage never released
+  TFERR_WAIT_TMEM_FULL = 3,   // epilogue: accumulator never committed
+  TFERR_WAIT_TMEM_EMPTY = 4,  // MMA warp: accumulator never drained
+};
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(bf16 x) { return __bfloat162float(x); }
+template <class T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ bf16 from_f32<bf16>(float x) { return __float2bfloat16_rn(x); }
+
+__device__ __forceinline__ float gelu_erf(float x) {
+  return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// max over non-negative floats (and NaN, whose bit pattern compares above +inf) through integer
+// atomics: for x >= 0 the IEEE bit pattern is monotone in x, so the result is order independent.
+__device__ __forceinline__ void atomic_max_nonneg(float* addr, float v) {
+  atomicMax(reinterpret_cast<int*>(addr), __float_as_int(v));
+}
+
+// Core position l of a block <-> raster token index (block permutation: reversal on odd blocks).
+__device__ __forceinline__ int tok_index(int l, int L, int reversed) { return reversed ? (L - 1 - l) : l; }

@@ -1,0 +1,166 @@
+// GEMM epilogue functors.  A GEMM kernel hands each functor NC consecutive accumulator columns of
+// one output row: apply<NC>(row, col0, v, n_valid) with col0 % NC == 0 and n_valid = min(NC, N-col0).
+// NC is 4 for the SIMT GEMM and 32 for the tcgen05 GEMM (one TMEM lane chunk per thread).
+#pragma once
+#include "common.cuh"
+
+// out[row, col] = act(acc + bias[col]).  With `out_lo` set (bf16 only) the value is stored as an
+// error-compensated pair: out = bf16(x), out_lo = bf16(x - out), so that out + out_lo carries about
+// 16 significant bits; the next GEMM/attention consumes both terms.
+template <class OutT, bool GELU>
+struct EpiStore {
+  OutT* out;
+  const float* bias;  // may be null
+  int ldc;
+  OutT* out_lo = nullptr;
+  template <int NC>
+  __device__ __forceinline__ void apply(int row, int col0, const float (&v)[NC], int nv) const {
+    OutT* p = out + (size_t)row * ldc + col0;
+    float r[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+      float x = v[j] + ((bias != nullptr && j < nv) ? bias[col0 + j] : 0.f);
+      r[j] = GELU ? gelu_erf(x) : x;
+    }
+    if constexpr (sizeof(OutT) == 4) {
+      if (nv == NC && (ldc % 4) == 0) {
+#pragma unroll
+        for (int j = 0; j < NC; j += 4)
+          *reinterpret_cast<float4*>(reinterpret_cast<float*>(p) + j) = make_float4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < NC; ++j)
+          if (j < nv) p[j] = from_f32<OutT>(r[j]);
+      }
+    } else {
+      store_bf16<NC>(p, r, nv);
+      if (out_lo != nullptr) {
+#pragma unroll
+        for (int j = 0; j < NC; ++j) r[j] -= __bfloat162float(__float2bfloat16_rn(r[j]));
+        store_bf16<NC>(out_lo + (size_t)row * ldc + col0, r, nv);
+      }
+    }
+  }
+  template <int NC>
+  __device__ __forceinline__ void store_bf16(OutT* p, const float (&r)[NC], int nv) const {
+    if (nv == NC && (ldc % 8) == 0) {
+      if constexpr (NC >= 8) {
+#pragma unroll
+        for (int j = 0; j < NC; j += 8) {
+          __nv_bfloat162 a = __floats2bfloat162_rn(r[j], r[j + 1]), b = __floats2bfloat162_rn(r[j + 2], r[j + 3]);
+          __nv_bfloat162 c = __floats2bfloat162_rn(r[j + 4], r[j + 5]), d = __floats2bfloat162_rn(r[j + 6], r[j + 7]);
+          uint4 u;
+          u.x = *reinterpret_cast<uint32_t*>(&a); u.y = *reinterpret_cast<uint32_t*>(&b);
+          u.z = *reinterpret_cast<uint32_t*>(&c); u.w = *reinterpret_cast<uint32_t*>(&d);
+          *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(p) + j) = u;
+        }
+      } else {
+        __nv_bfloat162 a = __floats2bfloat162_rn(r[0], r[1]), b = __floats2bfloat162_rn(r[2], r[3]);
+        uint2 u;
+        u.x = *reinterpret_cast<uint32_t*>(&a); u.y = *reinterpret_cast<uint32_t*>(&b);
+        *reinterpret_cast<uint2*>(p) = u;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < NC; ++j)
+        if (j < nv) p[j] = from_f32<OutT>(r[j]);
+    }
+  }
+};
+
+struct EpiResid {  // h[row, col] += acc + bias[col]   (fp32 residual stream, in place)
+  float* h;
+  const float* bias;
+  int ldc;
+  template <int NC>
+  __device__ __forceinline__ void apply(int row, int col0, const float (&v)[NC], int nv) const {
+    float* p = h + (size_t)row * ldc + col0;
+    if (nv == NC && (ldc % 4) == 0) {
+#pragma unroll
+      for (int j = 0; j < NC; j += 4) {
+        float4 o = *reinterpret_cast<float4*>(p + j);
+        float4 b = *reinterpret_cast<const float4*>(bias + col0 + j);
+        o.x += v[j] + b.x; o.y += v[j + 1] + b.y; o.z += v[j + 2] + b.z; o.w += v[j + 3] + b.w;
+        *reinterpret_cast<float4*>(p + j) = o;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < NC; ++j)
+        if (j < nv) p[j] += v[j] + bias[col0 + j];
+    }
+  }
+};
+
+// Sequential decoding step: the QKV projection of the one new token per sample.  Column ranges
+// [0,d) -> query buffer q[b, :], [d,2d) -> key cache row t, [2d,3d) -> value cache row t.
+template <class T>
+struct EpiQKVCache {
+  T* q;          // [B, d]
+  T* kc;         // [B, L, d]  this layer's key cache
+  T* vc;         // [B, L, d]
+  const float* bias;
+  int d, L, t;
+  template <int NC>
+  __device__ __forceinline__ void apply(int row, int col0, const float (&v)[NC], int nv) const {
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+      if (j >= nv) break;
+      int col = col0 + j;
+      T val = from_f32<T>(v[j] + bias[col]);
+      if (col < d) q[(size_t)row * d + col] = val;
+      else if (col < 2 * d) kc[((size_t)row * L + t) * d + (col - d)] = val;
+      else vc[((size_t)row * L + t) * d + (col - 2 * d)] = val;
+    }
+  }
+};
+
+// The fused step of Algorithm 1 in the head projection's epilogue.  The head matrix is stored with
+// interleaved rows, so accumulator columns (2c, 2c+1) are (mu~_c, alpha~_c) of output row (slot s,
+// core position l).  That row updates token l+1 of sample b = idx[s]:
+//     u[b, l+1, c] <- v[b, l+1, c] * exp(alpha~) + mu~          (Eq. 5 / Alg. 1 inner line)
+// and the row of the last position, whose head output is unused, performs u[b, 0, :] <- v[b, 0, :]
+// (Alg. 1: the first sub-variable is copied).  u is updated in place (every element is read and
+// written by exactly one thread of this launch); per-sample max |u_new - u_old| is accumulated
+// into maxdiff[b] with an order-independent integer atomic max.
+struct EpiHeadUpdate {
+  const float* v;      // [B, L, D] block input, raster order
+  float* u;            // [B, L, D] iterate, raster order, updated in place
+  float* maxdiff;      // [B]
+  const int* idx;      // [n_slots] slot -> sample (null = identity)
+  const float* bias;   // [2D] interleaved
+  int L, D, reversed;
+  template <int NC>
+  __device__ __forceinline__ void apply(int row, int col0, const float (&acc)[NC], int nv) const {
+    int s = row / L, l = row - s * L;
+    int b = idx ? idx[s] : s;
+    float m = 0.f;
+    if (l < L - 1) {
+      size_t base = ((size_t)b * L + tok_index(l + 1, L, reversed)) * D;
+#pragma unroll
+      for (int j = 0; j < NC; j += 2) {
+        if (j < nv) {
+          int c = (col0 + j) >> 1;
+          float mu = acc[j] + bias[col0 + j], al = acc[j + 1] + bias[col0 + j + 1];
+          float old = u[base + c];
+          float nw = fmaf(v[base + c], expf(al), mu);
+          u[base + c] = nw;
+          float df = fabsf(nw - old);
+          m = (df > m || df != df) ? df : m;
+        }
+      }
+    } else {
+      size_t base = ((size_t)b * L + tok_index(0, L, reversed)) * D;
+#pragma unroll
+      for (int j = 0; j < NC; j += 2) {
+        if (j < nv) {
+          int c = (col0 + j) >> 1;
+          float old = u[base + c], nw = v[base + c];
+          u[base + c] = nw;
+          float df = fabsf(nw - old);
+          m = (df > m || df != df) ? df : m;
+        }
+      }
+    }
+    atomic_max_nonneg(maxdiff + b, m);
+  }
+};

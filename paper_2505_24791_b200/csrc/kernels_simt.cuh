@@ -1,0 +1,398 @@
+// CUDA-core kernels: layout, embedding, LayerNorm, SIMT GEMM (fp32 engine and odd shapes), SIMT
+// attention (fp32 engine), single-query attention over the KV cache, update / forward epilogues
+// as stand-alone kernels, and Jacobi sweep control.
+#pragma once
+#include "common.cuh"
+#include "epilogue.cuh"
+
+// ------------------------------------------------------------------------------------------------
+// image [B,C,H,W] <-> tokens [B,L,D]; raster patch order, (c,py,px) inside a token.
+// ------------------------------------------------------------------------------------------------
+__global__ void patchify_kernel(float* __restrict__ img, float* __restrict__ seq, int B, int C, int H,
+                                int W, int p, int to_seq) {
+  size_t n = (size_t)B * C * H * W;
+  int gw = W / p, D = C * p * p, L = (H / p) * gw;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    int x = i % W, y = (i / W) % H, c = (i / ((size_t)W * H)) % C, b = i / ((size_t)W * H * C);
+    int l = (y / p) * gw + (x / p);
+    int e = (c * p + (y % p)) * p + (x % p);
+    size_t j = ((size_t)b * L + l) * D + e;
+    if (to_seq) seq[j] = img[i]; else img[i] = seq[j];
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// token embedding: h[s,l,:] = u[b,pos(l),:] W_in^T + b_in + pos_emb[l] (+ cls[y_b]), b = idx[s].
+// w_in_t is W_in transposed to [D, d] so consecutive threads read consecutive addresses.
+// One CTA per output row.  `l_fixed` >= 0: rows are samples and every row uses position l_fixed
+// (sequential decoding step).
+// ------------------------------------------------------------------------------------------------
+__global__ void embed_kernel(const float* __restrict__ u, const int* __restrict__ idx, const int* __restrict__ labels,
+                             const float* __restrict__ w_in_t, const float* __restrict__ b_in,
+                             const float* __restrict__ pos, const float* __restrict__ cls, float* __restrict__ h,
+                             int L, int D, int d, int reversed, int l_fixed) {
+  extern __shared__ float s_u[];
+  int row = blockIdx.x;
+  int s = (l_fixed >= 0) ? row : row / L;
+  int l = (l_fixed >= 0) ? l_fixed : row - s * L;
+  int b = idx ? idx[s] : s;
+  const float* up = u + ((size_t)b * L + tok_index(l, L, reversed)) * D;
+  for (int c = threadIdx.x; c < D; c += blockDim.x) s_u[c] = up[c];
+  __syncthreads();
+  const float* cl = (cls != nullptr) ? cls + (size_t)labels[b] * d : nullptr;
+  for (int j = threadIdx.x; j < d; j += blockDim.x) {
+    float acc = 0.f;
+    for (int c = 0; c < D; ++c) acc = fmaf(s_u[c], w_in_t[(size_t)c * d + j], acc);
+    acc += b_in[j] + pos[(size_t)l * d + j];
+    if (cl) acc += cl[j];
+    h[(size_t)row * d + j] = acc;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// LayerNorm over the last dimension (eps 1e-5), fp32 in, T out.  One warp per row, the row is
+// held in registers (d <= 32*4*MAXV).
+// ------------------------------------------------------------------------------------------------
+template <class T, int MAXV>
+__global__ void layernorm_kernel(const float* __restrict__ x, const float* __restrict__ gamma,
+                                 const float* __restrict__ beta, T* __restrict__ y, T* __restrict__ y_lo, int rows,
+                                 int d) {
+  int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= rows) return;
+  const float4* xr = reinterpret_cast<const float4*>(x + (size_t)warp * d);
+  int nv = d >> 2;  // float4 per row
+  float4 v[MAXV];
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    int k = lane + i * 32;
+    if (k < nv) { v[i] = xr[k]; sum += v[i].x + v[i].y + v[i].z + v[i].w; }
+  }
+  float mean = warp_sum(sum) / d;
+  float sq = 0.f;
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    int k = lane + i * 32;
+    if (k < nv) {
+      float a = v[i].x - mean, b = v[i].y - mean, c = v[i].z - mean, e = v[i].w - mean;
+      sq += a * a + b * b + c * c + e * e;
+    }
+  }
+  float rstd = rsqrtf(warp_sum(sq) / d + 1e-5f);
+  T* yr = y + (size_t)warp * d;
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    int k = lane + i * 32;
+    if (k < nv) {
+      float4 g = reinterpret_cast<const float4*>(gamma)[k], bb = reinterpret_cast<const float4*>(beta)[k];
+      float o0 = (v[i].x - mean) * rstd * g.x + bb.x, o1 = (v[i].y - mean) * rstd * g.y + bb.y;
+      float o2 = (v[i].z - mean) * rstd * g.z + bb.z, o3 = (v[i].w - mean) * rstd * g.w + bb.w;
+      if constexpr (sizeof(T) == 4) {
+        reinterpret_cast<float4*>(yr)[k] = make_float4(o0, o1, o2, o3);
+      } else {
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);
+        uint2 w;
+        w.x = *reinterpret_cast<uint32_t*>(&p0); w.y = *reinterpret_cast<uint32_t*>(&p1);
+        reinterpret_cast<uint2*>(yr)[k] = w;
+        if (y_lo != nullptr) {  // second term of the error-compensated pair
+          float2 f0 = __bfloat1622float2(p0), f1 = __bfloat1622float2(p1);
+          __nv_bfloat162 q0 = __floats2bfloat162_rn(o0 - f0.x, o1 - f0.y), q1 = __floats2bfloat162_rn(o2 - f1.x, o3 - f1.y);
+          w.x = *reinterpret_cast<uint32_t*>(&q0); w.y = *reinterpret_cast<uint32_t*>(&q1);
+          reinterpret_cast<uint2*>(y_lo + (size_t)warp * d)[k] = w;
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// SIMT GEMM: C[M,N] = A[M,K] W[N,K]^T, fp32 FMA accumulate, 64x64 tile, 16-wide K slab, 256 threads,
+// 4x4 outputs per thread.  Used by the fp32 engine everywhere and by the bf16 engine for shapes
+// the tensor-core kernels do not take.
+// ------------------------------------------------------------------------------------------------
+template <class TA, class Epi>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const TA* __restrict__ A, const TA* __restrict__ Wt, int M,
+                                                        int N, int K, Epi epi) {
+  __shared__ float sA[16][64 + 4];
+  __shared__ float sB[16][64 + 4];
+  int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  for (int k0 = 0; k0 < K; k0 += 16) {
+    // 64 rows x 16 k per operand = 1024 elements, 4 per thread
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      int e = threadIdx.x + i * 256;
+      int r = e >> 4, k = e & 15;
+      int gm = m0 + r, gn = n0 + r, gk = k0 + k;
+      sA[k][r] = (gm < M && gk < K) ? to_f32(A[(size_t)gm * K + gk]) : 0.f;
+      sB[k][r] = (gn < N && gk < K) ? to_f32(Wt[(size_t)gn * K + gk]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = sA[k][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = sB[k][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    int row = m0 + ty * 4 + i, col0 = n0 + tx * 4;
+    if (row < M && col0 < N) {
+      int nv = N - col0 < 4 ? N - col0 : 4;
+      epi.template apply<4>(row, col0, acc[i], nv);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Causal attention, SIMT: one warp per (slot, head, query position).  qkv rows are [q | k | v],
+// 3d wide.  Scores for keys j <= i in shared memory, fp32 softmax, output a[row, head*hd + c].
+// ------------------------------------------------------------------------------------------------
+template <class T>
+__global__ void attention_simt_kernel(const T* __restrict__ qkv, T* __restrict__ out, int L, int d, int hd,
+                                      float scale) {
+  extern __shared__ float s_p[];  // [warps][L] scores, then [warps][hd] query
+  int warps = blockDim.x >> 5, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int i = blockIdx.x * warps + w;  // query position
+  int head = blockIdx.y, s = blockIdx.z;
+  float* p = s_p + (size_t)w * L;
+  float* sq = s_p + (size_t)warps * L + (size_t)w * hd;
+  if (i >= L) return;
+  size_t ld = 3 * (size_t)d;
+  const T* base = qkv + (size_t)s * L * ld + (size_t)head * hd;
+  for (int c = lane; c < hd; c += 32) sq[c] = to_f32(base[(size_t)i * ld + c]);
+  __syncwarp();
+  float mx = -INFINITY;
+  for (int j = lane; j <= i; j += 32) {
+    const T* kr = base + (size_t)j * ld + d;
+    float acc = 0.f;
+    for (int c = 0; c < hd; ++c) acc = fmaf(sq[c], to_f32(kr[c]), acc);
+    acc *= scale;
+    p[j] = acc;
+    mx = fmaxf(mx, acc);
+  }
+  mx = warp_max(mx);
+  float sum = 0.f;
+  for (int j = lane; j <= i; j += 32) {
+    float e = expf(p[j] - mx);
+    p[j] = e;
+    sum += e;
+  }
+  sum = warp_sum(sum);
+  __syncwarp();
+  float inv = 1.f / sum;
+  for (int c = lane; c < hd; c += 32) {
+    float acc = 0.f;
+    for (int j = 0; j <= i; ++j) acc = fmaf(p[j], to_f32(base[(size_t)j * ld + 2 * d + c]), acc);
+    out[((size_t)s * L + i) * d + (size_t)head * hd + c] = from_f32<T>(acc * inv);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Sequential decoding: one query per (sample, head) over cache rows 0..t.  4 warps split the keys.
+// kc, vc: [B, L, d]; q, out: [B, d].
+// ------------------------------------------------------------------------------------------------
+template <class T>
+__global__ void __launch_bounds__(128) attention_step_kernel(const T* __restrict__ q, const T* __restrict__ kc,
+                                                             const T* __restrict__ vc, T* __restrict__ out, int L,
+                                                             int d, int hd, int t, float scale) {
+  extern __shared__ float sm[];  // p[t+1] | q[hd] | red[8] | acc[4][hd]
+  int head = blockIdx.x, b = blockIdx.y;
+  int nk = t + 1;
+  float* p = sm;
+  float* sq = p + L;
+  float* red = sq + hd;
+  float* sacc = red + 8;
+  int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const T* kb = kc + (size_t)b * L * d + (size_t)head * hd;
+  const T* vb = vc + (size_t)b * L * d + (size_t)head * hd;
+  for (int c = threadIdx.x; c < hd; c += 128) sq[c] = to_f32(q[(size_t)b * d + head * hd + c]);
+  __syncthreads();
+  float mx = -INFINITY;
+  for (int j = threadIdx.x; j < nk; j += 128) {
+    const T* kr = kb + (size_t)j * d;
+    float acc = 0.f;
+    for (int c = 0; c < hd; ++c) acc = fmaf(sq[c], to_f32(kr[c]), acc);
+    acc *= scale;
+    p[j] = acc;
+    mx = fmaxf(mx, acc);
+  }
+  mx = warp_max(mx);
+  if (lane == 0) red[w] = mx;
+  __syncthreads();
+  mx = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+  float sum = 0.f;
+  for (int j = threadIdx.x; j < nk; j += 128) {
+    float e = expf(p[j] - mx);
+    p[j] = e;
+    sum += e;
+  }
+  sum = warp_sum(sum);
+  if (lane == 0) red[4 + w] = sum;
+  __syncthreads();
+  float inv = 1.f / (red[4] + red[5] + red[6] + red[7]);
+  // warp w accumulates keys j = w, w+4, ...; lanes over channels
+  for (int c = lane; c < hd; c += 32) {
+    float acc = 0.f;
+    for (int j = w; j < nk; j += 4) acc = fmaf(p[j], to_f32(vb[(size_t)j * d + c]), acc);
+    sacc[w * hd + c] = acc;
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < hd; c += 128) {
+    float acc = (sacc[c] + sacc[hd + c]) + (sacc[2 * hd + c] + sacc[3 * hd + c]);
+    out[(size_t)b * d + head * hd + c] = from_f32<T>(acc * inv);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Stand-alone Jacobi update (Algorithm 1's inner line + norm) from a stored head output.
+// o: [rows, 2D]; interleaved != 0: columns (2c,2c+1) = (mu~_c, alpha~_c), else [mu~ | alpha~].
+// One thread per (row, c).  u updated in place; maxdiff via order-independent atomic max.
+// ------------------------------------------------------------------------------------------------
+__global__ void jacobi_update_kernel(const float* __restrict__ o, const float* __restrict__ v, float* __restrict__ u,
+                                     float* __restrict__ maxdiff, const int* __restrict__ idx, int n_rows, int L,
+                                     int D, int reversed, int interleaved) {
+  size_t n = (size_t)n_rows * D;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    int c = i % D;
+    int row = i / D;
+    int s = row / L, l = row - s * L;
+    int b = idx ? idx[s] : s;
+    float nw, old;
+    if (l < L - 1) {
+      size_t e = ((size_t)b * L + tok_index(l + 1, L, reversed)) * D + c;
+      const float* orow = o + (size_t)row * 2 * D;
+      float mu = interleaved ? orow[2 * c] : orow[c];
+      float al = interleaved ? orow[2 * c + 1] : orow[D + c];
+      old = u[e];
+      nw = fmaf(v[e], expf(al), mu);
+      u[e] = nw;
+    } else {
+      size_t e = ((size_t)b * L + tok_index(0, L, reversed)) * D + c;
+      old = u[e];
+      nw = v[e];
+      u[e] = nw;
+    }
+    atomic_max_nonneg(maxdiff + b, fabsf(nw - old));
+  }
+}
+
+// Sequential decoding: token t+1 of every sample from the head output of token t (Eq. 5).
+// o: [B, 2D] interleaved.
+__global__ void seq_update_kernel(const float* __restrict__ o, const float* __restrict__ v, float* __restrict__ u,
+                                  int B, int L, int D, int reversed, int t) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B * D) return;
+  int b = i / D, c = i - b * D;
+  size_t e = ((size_t)b * L + tok_index(t + 1, L, reversed)) * D + c;
+  u[e] = fmaf(v[e], expf(o[(size_t)b * 2 * D + 2 * c + 1]), o[(size_t)b * 2 * D + 2 * c]);
+}
+
+// First token of a block passes through unchanged (Eq. 4 / Eq. 5 first row).
+__global__ void copy_first_token_kernel(const float* __restrict__ v, float* __restrict__ u, int B, int L, int D,
+                                        int reversed) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B * D) return;
+  int b = i / D, c = i - b * D;
+  size_t e = ((size_t)b * L + tok_index(0, L, reversed)) * D + c;
+  u[e] = v[e];
+}
+
+// Forward direction (Eq. 4): v_l = (u_l - mu_l) exp(-alpha_l), logdet[b] -= sum alpha.  One CTA per
+// sample so the per-sample sum is a fixed-order tree (deterministic).  o: [B*L, 2D] interleaved.
+__global__ void __launch_bounds__(256) forward_affine_kernel(const float* __restrict__ o, const float* __restrict__ u,
+                                                             float* __restrict__ v, float* __restrict__ logdet, int L,
+                                                             int D, int reversed) {
+  __shared__ float red[8];
+  int b = blockIdx.x;
+  float part = 0.f;
+  for (int i = threadIdx.x; i < L * D; i += 256) {
+    int l = i / D, c = i - l * D;
+    size_t e = ((size_t)b * L + tok_index(l, L, reversed)) * D + c;
+    float mu = 0.f, al = 0.f;
+    if (l > 0) {
+      const float* orow = o + ((size_t)b * L + (l - 1)) * 2 * D;
+      mu = orow[2 * c];
+      al = orow[2 * c + 1];
+    }
+    v[e] = (u[e] - mu) * expf(-al);
+    part += al;
+  }
+  part = warp_sum(part);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = part;
+  __syncthreads();
+  if (threadIdx.x == 0 && logdet != nullptr) {
+    float s = 0.f;
+    for (int i = 0; i < 8; ++i) s += red[i];
+    logdet[b] -= s;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Sweep control (single thread; B is at most a few hundred).  After sweep `t`: record the sweep
+// count of every active sample, drop the samples that passed the test, move a sample to the
+// two-term ("hp") phase once its own max|du| <= switch_thresh, and rebuild the slot list as
+// [single-precision samples..., hp samples...] with a stable partition, so the slot order never
+// depends on timing and a sample's schedule depends on that sample alone.
+// ctrl[0] = n_active, ctrl[1] = non-finite flag, ctrl[2] = bits of max over active samples of
+// maxdiff, ctrl[3] = number of active samples in the hp phase (the tail of idx).
+// ------------------------------------------------------------------------------------------------
+__global__ void jacobi_finalize_kernel(float* __restrict__ maxdiff, int* __restrict__ idx, int* __restrict__ idx_tmp,
+                                       int* __restrict__ phase, int* __restrict__ ctrl, int* __restrict__ iters_sample,
+                                       float tau, float switch_thresh, int t) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  int n = ctrl[0], keep = 0, bad = ctrl[1];
+  float top = 0.f;
+  for (int s = 0; s < n; ++s) {
+    int b = idx[s];
+    float m = maxdiff[b];
+    maxdiff[b] = 0.f;
+    top = (m > top || m != m) ? m : top;
+    if (iters_sample) iters_sample[b] = t;
+    if (!(m <= 3.0e38f)) bad = 1;
+    if (tau < 0.f || !(m <= tau)) {
+      if (m <= switch_thresh) phase[b] = 1;
+      idx_tmp[keep++] = b;
+    }
+  }
+  int k = 0, n_hp = 0;
+  for (int s = 0; s < keep; ++s) if (phase[idx_tmp[s]] == 0) idx[k++] = idx_tmp[s];
+  for (int s = 0; s < keep; ++s) if (phase[idx_tmp[s]] != 0) { idx[k++] = idx_tmp[s]; ++n_hp; }
+  ctrl[0] = keep;
+  ctrl[1] = bad;
+  ctrl[2] = __float_as_int(top);
+  ctrl[3] = n_hp;
+}
+
+__global__ void jacobi_begin_kernel(float* __restrict__ maxdiff, int* __restrict__ idx, int* __restrict__ phase,
+                                    int* __restrict__ ctrl, int B, int start_phase) {
+  for (int b = threadIdx.x; b < B; b += blockDim.x) {
+    maxdiff[b] = 0.f;
+    idx[b] = b;
+    phase[b] = start_phase;
+  }
+  if (threadIdx.x == 0) { ctrl[0] = B; ctrl[1] = 0; ctrl[2] = 0; ctrl[3] = start_phase ? B : 0; }
+}
+
+__global__ void fill_int_kernel(int* p, int n, int v) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = v;
+}
+
+__global__ void f32_to_bf16_kernel(const float* __restrict__ in, bf16* __restrict__ out, size_t n) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    out[i] = __float2bfloat16_rn(in[i]);
+}

@@ -1,0 +1,860 @@
+// libtarflow: host side of the selective-Jacobi TarFlow engine and its C ABI (see include/tarflow.h).
+//
+// One tf_model owns: the weights of K flow blocks (fp32, or bf16 matrices + fp32 vectors), two
+// token-sequence buffers that ping-pong between blocks, the activation workspace of one causal pass
+// over up to max_batch * L rows, the per-layer key/value cache of the sequential path, and the
+// sweep-control words.  All sequences stay in raster token order; the block permutation (reversal
+// on odd blocks) is folded into the index arithmetic of the embedding and update kernels.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/tarflow.h"
+#include "attention_mma.cuh"
+#include "common.cuh"
+#include "epilogue.cuh"
+#include "gemm_tc.cuh"
+#include "kernels_simt.cuh"
+
+// ------------------------------------------------------------------------------------------------
+// errors
+// ------------------------------------------------------------------------------------------------
+static thread_local char g_err[512] = "";
+static int fail(int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+#define CU_OK(expr)                                                                       \
+  do {                                                                                    \
+    cudaError_t e__ = (expr);                                                             \
+    if (e__ != cudaSuccess) return fail(TF_ECUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
+  } while (0)
+#define TF_TRY(expr)            \
+  do {                          \
+    int r__ = (expr);           \
+    if (r__ < 0) return r__;    \
+  } while (0)
+
+// ------------------------------------------------------------------------------------------------
+// TMA tensor maps (driver entry point fetched at run time; libcuda is not linked)
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static encode_tiled_fn get_encode_fn() {
+  static encode_tiled_fn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<encode_tiled_fn>(p);
+  }
+  return fn;
+}
+// bf16 matrix [rows, K] row-major; box = 64 (K) x box_rows, 128-byte swizzle, zero fill outside.
+static int make_map_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K, uint32_t box_rows) {
+  encode_tiled_fn fn = get_encode_fn();
+  if (!fn) return fail(TF_ECUDA, "cuTensorMapEncodeTiled entry point not available");
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || (K * 2) % 16) return fail(TF_EINVAL, "TMA operand not 16-byte aligned");
+  cuuint64_t dims[2] = {K, rows};
+  cuuint64_t strides[1] = {K * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(TF_ECUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+  return TF_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// model
+// ------------------------------------------------------------------------------------------------
+enum KernelClass {
+  KC_LAYOUT, KC_EMBED, KC_LN, KC_GEMM_QKV, KC_ATTN, KC_GEMM_O, KC_GEMM_MLP1, KC_GEMM_MLP2, KC_GEMM_HEAD_UPDATE,
+  KC_GEMM_HEAD, KC_AFFINE, KC_CTRL, KC_SEQ_EMBED, KC_SEQ_LN, KC_SEQ_GEMM, KC_SEQ_ATTN, KC_SEQ_UPDATE, KC_COUNT
+};
+static const char* kKernelClassNames[KC_COUNT] = {
+    "layout", "embed", "layernorm", "gemm_qkv", "attention", "gemm_out", "gemm_mlp_up", "gemm_mlp_down",
+    "gemm_head_update", "gemm_head", "forward_affine", "sweep_control", "seq_embed", "seq_layernorm", "seq_gemm",
+    "seq_attention", "seq_update"};
+
+struct Matrix {       // a linear layer's weight [N, K]
+  void* w = nullptr;  // float* or bf16*
+  int N = 0, K = 0;
+  CUtensorMap map;    // bf16 engine: box 64 x bn
+  int bn = 0;
+};
+struct LayerW {
+  float *ln1_g, *ln1_b, *b_qkv, *b_o, *ln2_g, *ln2_b, *b_1, *b_2;
+  Matrix w_qkv, w_o, w_1, w_2;
+};
+struct BlockW {
+  float *w_in_t, *b_in, *pos, *cls, *lnf_g, *lnf_b, *b_out;  // b_out interleaved (mu_c, alpha_c)
+  Matrix w_out;                                                // rows interleaved the same way
+  std::vector<LayerW> layers;
+};
+
+struct tf_model {
+  tf_config cfg;
+  int L, D, d, hid, hd;
+  int num_sms = 148;
+  std::vector<BlockW> blocks;
+  std::vector<void*> allocs;
+  int64_t device_bytes = 0;
+  // workspace
+  float *seq_a = nullptr, *seq_b = nullptr, *h = nullptr, *o = nullptr, *maxdiff = nullptr;
+  void *xn = nullptr, *qkv = nullptr, *att = nullptr, *mlp = nullptr, *kcache = nullptr, *vcache = nullptr;
+  void *xn_lo = nullptr, *qkv_lo = nullptr, *att_lo = nullptr, *mlp_lo = nullptr;  // second terms (bf16 engine)
+  CUtensorMap map_xn, map_att, map_mlp, map_xn_lo, map_att_lo, map_mlp_lo;
+  int *idx = nullptr, *idx_tmp = nullptr, *phase = nullptr, *ctrl = nullptr, *iters_sample = nullptr, *err = nullptr;
+  // precision policy of Jacobi blocks on the bf16 engine: 0 = escalate per sample, 1 = single bf16
+  // operands only, 2 = two-term operands for every sweep
+  int precision_mode = 0;
+  float switch_threshold = 0.03125f;   // a sample's sweeps use two-term operands once its max|du| <= this
+  float single_ok_tau = 0.015625f;     // tau at or above this never escalates
+  int* ctrl_host = nullptr;  // pinned: n_active, nonfinite, device error
+  float *io_z = nullptr, *io_x = nullptr;  // staging for the host-buffer entry point
+  int* io_labels = nullptr;
+  cudaStream_t stream = nullptr;
+  int64_t launches = 0;
+  // profiling
+  bool prof_on = false;
+  std::vector<cudaEvent_t> ev_pool;
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> ev_pending[KC_COUNT];
+  double prof_ms[KC_COUNT] = {0};
+  int64_t prof_n[KC_COUNT] = {0};
+  cudaEvent_t cur_start = nullptr;
+  // convergence trace (one record per sweep of the last inverse call)
+  struct TraceRec { int block, sweep, active; float maxdiff; };
+  bool trace_on = false;
+  std::vector<TraceRec> trace;
+
+  cudaEvent_t get_event() {
+    if (!ev_pool.empty()) {
+      cudaEvent_t e = ev_pool.back();
+      ev_pool.pop_back();
+      return e;
+    }
+    cudaEvent_t e;
+    cudaEventCreate(&e);
+    return e;
+  }
+  void pre(int) {
+    if (prof_on) {
+      cur_start = get_event();
+      cudaEventRecord(cur_start, stream);
+    }
+  }
+  void post(int cls) {
+    ++launches;
+    if (prof_on) {
+      cudaEvent_t e = get_event();
+      cudaEventRecord(e, stream);
+      ev_pending[cls].push_back({cur_start, e});
+    }
+  }
+  void prof_collect() {
+    for (int c = 0; c < KC_COUNT; ++c) {
+      for (auto& pr : ev_pending[c]) {
+        float ms = 0.f;
+        cudaEventSynchronize(pr.second);
+        cudaEventElapsedTime(&ms, pr.first, pr.second);
+        prof_ms[c] += ms;
+        prof_n[c] += 1;
+        ev_pool.push_back(pr.first);
+        ev_pool.push_back(pr.second);
+      }
+      ev_pending[c].clear();
+    }
+  }
+};
+
+#define LAUNCH(m, cls, kern, grid, block, smem, ...)           \
+  do {                                                         \
+    (m)->pre(cls);                                             \
+    kern<<<(grid), (block), (smem), (m)->stream>>>(__VA_ARGS__); \
+    (m)->post(cls);                                            \
+  } while (0)
+
+static int check_launch(const char* what) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(TF_ECUDA, "%s: %s", what, cudaGetErrorString(e));
+  return TF_OK;
+}
+
+template <class T>
+static int dev_alloc(tf_model* m, T** p, size_t count) {
+  size_t bytes = ((count * sizeof(T)) + 255) & ~(size_t)255;
+  if (bytes == 0) bytes = 256;
+  void* q = nullptr;
+  cudaError_t e = cudaMalloc(&q, bytes);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(TF_ENOMEM, "cudaMalloc(%zu bytes) failed: %s", bytes, cudaGetErrorString(e));
+  }
+  m->allocs.push_back(q);
+  m->device_bytes += (int64_t)bytes;
+  *p = reinterpret_cast<T*>(q);
+  return TF_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// GEMM dispatch
+// ------------------------------------------------------------------------------------------------
+template <int BN, int STAGES, class Epi>
+static int launch_gemm_tc(tf_model* m, int cls, cudaStream_t stream, const CUtensorMap& ma, const CUtensorMap* ma_lo,
+                          const CUtensorMap& mw, int M, int N, int K, const Epi& epi, int* err, int num_sms,
+                          int64_t* launches) {
+  using SL = tc::SmemLayout<BN, STAGES>;
+  auto kern = tc::gemm_tc_kernel<BN, STAGES, Epi>;
+  static bool configured = false;  // per instantiation
+  if (!configured) {
+    CU_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::TOTAL));
+    configured = true;
+  }
+  int tiles = ((M + tc::BM - 1) / tc::BM) * ((N + BN - 1) / BN);
+  int grid = tiles < num_sms ? tiles : num_sms;
+  if (m) m->pre(cls);
+  kern<<<grid, tc::NUM_THREADS, SL::TOTAL, stream>>>(ma, ma_lo ? *ma_lo : ma, mw, M, N, K, ma_lo ? 1 : 0, epi, err);
+  if (m) m->post(cls); else if (launches) ++*launches;
+  return check_launch("gemm_tc_kernel");
+}
+
+template <class T, class Epi>
+static int launch_gemm_simt(tf_model* m, int cls, const T* A, const Matrix& W, int M, const Epi& epi) {
+  dim3 grid((W.N + 63) / 64, (M + 63) / 64);
+  LAUNCH(m, cls, (gemm_simt_kernel<T, Epi>), grid, 256, 0, A, reinterpret_cast<const T*>(W.w), M, W.N, W.K, epi);
+  return check_launch("gemm_simt_kernel");
+}
+
+// A [M, K] activations (type T) times W^T.  bf16 engine: tensor-core kernel (map_a_lo != null: A is a
+// two-term pair); fp32 engine: SIMT kernel.
+template <class T, class Epi>
+static int gemm(tf_model* m, int cls, const T* A, const CUtensorMap* map_a, const CUtensorMap* map_a_lo,
+                const Matrix& W, int M, const Epi& epi) {
+  if constexpr (sizeof(T) == 2) {
+    if (W.bn == 256)
+      return launch_gemm_tc<256, 4, Epi>(m, cls, m->stream, *map_a, map_a_lo, W.map, M, W.N, W.K, epi, m->err,
+                                         m->num_sms, nullptr);
+    return launch_gemm_tc<128, 6, Epi>(m, cls, m->stream, *map_a, map_a_lo, W.map, M, W.N, W.K, epi, m->err,
+                                       m->num_sms, nullptr);
+  } else {
+    return launch_gemm_simt<T, Epi>(m, cls, A, W, M, epi);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// one causal pass over n_slots * L rows (a Jacobi sweep, or the forward direction)
+// ------------------------------------------------------------------------------------------------
+template <class T>
+static int layernorm(tf_model* m, int cls, const float* x, const float* g, const float* b, T* y, T* y_lo, int rows) {
+  int d = m->d;
+  int blocks = (rows * 32 + 255) / 256;
+  if (d <= 128 * 1) LAUNCH(m, cls, (layernorm_kernel<T, 1>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
+  else if (d <= 128 * 4) LAUNCH(m, cls, (layernorm_kernel<T, 4>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
+  else if (d <= 128 * 8) LAUNCH(m, cls, (layernorm_kernel<T, 8>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
+  else LAUNCH(m, cls, (layernorm_kernel<T, 16>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
+  return check_launch("layernorm_kernel");
+}
+
+enum PassMode { PASS_JACOBI, PASS_FORWARD };
+
+// hp: every bf16 operand travels as a two-term pair (bf16 engine only).
+template <class T>
+static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const int* idx, const int* labels,
+                    PassMode mode, const float* v, float* u_upd, bool hp) {
+  const BlockW& bw = m->blocks[g];
+  const int L = m->L, D = m->D, d = m->d, M = n_slots * L, rev = g & 1;
+  T* xn = reinterpret_cast<T*>(m->xn);
+  T* qkv = reinterpret_cast<T*>(m->qkv);
+  T* att = reinterpret_cast<T*>(m->att);
+  T* mlp = reinterpret_cast<T*>(m->mlp);
+  T* xn_lo = hp ? reinterpret_cast<T*>(m->xn_lo) : nullptr;
+  T* qkv_lo = hp ? reinterpret_cast<T*>(m->qkv_lo) : nullptr;
+  T* att_lo = hp ? reinterpret_cast<T*>(m->att_lo) : nullptr;
+  T* mlp_lo = hp ? reinterpret_cast<T*>(m->mlp_lo) : nullptr;
+  const CUtensorMap* mxl = hp ? &m->map_xn_lo : nullptr;
+  const CUtensorMap* mal = hp ? &m->map_att_lo : nullptr;
+  const CUtensorMap* mml = hp ? &m->map_mlp_lo : nullptr;
+  int ethreads = d < 256 ? d : 256;
+  LAUNCH(m, KC_EMBED, embed_kernel, M, ethreads, D * sizeof(float), u_src, idx, labels, bw.w_in_t, bw.b_in, bw.pos,
+         bw.cls, m->h, L, D, d, rev, -1);
+  TF_TRY(check_launch("embed_kernel"));
+  for (const LayerW& lw : bw.layers) {
+    TF_TRY(layernorm<T>(m, KC_LN, m->h, lw.ln1_g, lw.ln1_b, xn, xn_lo, M));
+    TF_TRY(gemm<T>(m, KC_GEMM_QKV, xn, &m->map_xn, mxl, lw.w_qkv, M, EpiStore<T, false>{qkv, lw.b_qkv, 3 * d, qkv_lo}));
+    if constexpr (sizeof(T) == 2) {
+      dim3 grid((L + attn::BQ - 1) / attn::BQ, m->cfg.n_heads, n_slots);
+      const float sl2 = 1.4426950408889634f / sqrtf((float)m->hd);
+      if (hp)
+        LAUNCH(m, KC_ATTN, attn::attention_mma_kernel<true>, grid, 128, attn::smem_bytes<true>(), qkv, qkv_lo, att,
+               att_lo, L, d, sl2);
+      else
+        LAUNCH(m, KC_ATTN, attn::attention_mma_kernel<false>, grid, 128, attn::smem_bytes<false>(), qkv, qkv_lo, att,
+               att_lo, L, d, sl2);
+    } else {
+      const int warps = 4;
+      dim3 grid((L + warps - 1) / warps, m->cfg.n_heads, n_slots);
+      size_t smem = (size_t)warps * (L + m->hd) * sizeof(float);
+      LAUNCH(m, KC_ATTN, (attention_simt_kernel<T>), grid, warps * 32, smem, qkv, att, L, d, m->hd,
+             1.0f / sqrtf((float)m->hd));
+    }
+    TF_TRY(check_launch("attention kernel"));
+    TF_TRY(gemm<T>(m, KC_GEMM_O, att, &m->map_att, mal, lw.w_o, M, EpiResid{m->h, lw.b_o, d}));
+    TF_TRY(layernorm<T>(m, KC_LN, m->h, lw.ln2_g, lw.ln2_b, xn, xn_lo, M));
+    TF_TRY(gemm<T>(m, KC_GEMM_MLP1, xn, &m->map_xn, mxl, lw.w_1, M, EpiStore<T, true>{mlp, lw.b_1, m->hid, mlp_lo}));
+    TF_TRY(gemm<T>(m, KC_GEMM_MLP2, mlp, &m->map_mlp, mml, lw.w_2, M, EpiResid{m->h, lw.b_2, d}));
+  }
+  TF_TRY(layernorm<T>(m, KC_LN, m->h, bw.lnf_g, bw.lnf_b, xn, xn_lo, M));
+  if (mode == PASS_JACOBI) {
+    EpiHeadUpdate epi{v, u_upd, m->maxdiff, idx, bw.b_out, L, D, rev};
+    TF_TRY(gemm<T>(m, KC_GEMM_HEAD_UPDATE, xn, &m->map_xn, mxl, bw.w_out, M, epi));
+  } else {
+    TF_TRY(gemm<T>(m, KC_GEMM_HEAD, xn, &m->map_xn, mxl, bw.w_out, M, EpiStore<float, false>{m->o, bw.b_out, 2 * D}));
+  }
+  return TF_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// sequential block with KV cache (Eq. 5): L-1 single-token passes
+// ------------------------------------------------------------------------------------------------
+template <class T>
+static int run_sequential_block(tf_model* m, int g, int B, const int* labels, const float* v, float* u) {
+  const BlockW& bw = m->blocks[g];
+  const int L = m->L, D = m->D, d = m->d, rev = g & 1, nl = m->cfg.n_layers;
+  T* xn = reinterpret_cast<T*>(m->xn);
+  T* q = reinterpret_cast<T*>(m->qkv);
+  T* att = reinterpret_cast<T*>(m->att);
+  T* mlp = reinterpret_cast<T*>(m->mlp);
+  const size_t layer_stride = (size_t)m->cfg.max_batch * L * d;
+  const float scale = 1.0f / sqrtf((float)m->hd);
+  int ethreads = d < 256 ? d : 256;
+  LAUNCH(m, KC_SEQ_UPDATE, copy_first_token_kernel, (B * D + 127) / 128, 128, 0, v, u, B, L, D, rev);
+  for (int t = 0; t + 1 < L; ++t) {
+    LAUNCH(m, KC_SEQ_EMBED, embed_kernel, B, ethreads, D * sizeof(float), u, (const int*)nullptr, labels, bw.w_in_t,
+           bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, t);
+    for (int i = 0; i < nl; ++i) {
+      const LayerW& lw = bw.layers[i];
+      T* kc = reinterpret_cast<T*>(m->kcache) + i * layer_stride;
+      T* vc = reinterpret_cast<T*>(m->vcache) + i * layer_stride;
+      TF_TRY(layernorm<T>(m, KC_SEQ_LN, m->h, lw.ln1_g, lw.ln1_b, xn, (T*)nullptr, B));
+      TF_TRY(launch_gemm_simt<T>(m, KC_SEQ_GEMM, xn, lw.w_qkv, B, EpiQKVCache<T>{q, kc, vc, lw.b_qkv, d, L, t}));
+      size_t smem = (size_t)(L + m->hd + 8 + 4 * m->hd) * sizeof(float);
+      LAUNCH(m, KC_SEQ_ATTN, (attention_step_kernel<T>), dim3(m->cfg.n_heads, B), 128, smem, q, kc, vc, att, L, d,
+             m->hd, t, scale);
+      TF_TRY(launch_gemm_simt<T>(m, KC_SEQ_GEMM, att, lw.w_o, B, EpiResid{m->h, lw.b_o, d}));
+      TF_TRY(layernorm<T>(m, KC_SEQ_LN, m->h, lw.ln2_g, lw.ln2_b, xn, (T*)nullptr, B));
+      TF_TRY(launch_gemm_simt<T>(m, KC_SEQ_GEMM, xn, lw.w_1, B, EpiStore<T, true>{mlp, lw.b_1, m->hid}));
+      TF_TRY(launch_gemm_simt<T>(m, KC_SEQ_GEMM, mlp, lw.w_2, B, EpiResid{m->h, lw.b_2, d}));
+    }
+    TF_TRY(layernorm<T>(m, KC_SEQ_LN, m->h, bw.lnf_g, bw.lnf_b, xn, (T*)nullptr, B));
+    TF_TRY(launch_gemm_simt<T>(m, KC_SEQ_GEMM, xn, bw.w_out, B, EpiStore<float, false>{m->o, bw.b_out, 2 * D}));
+    LAUNCH(m, KC_SEQ_UPDATE, seq_update_kernel, (B * D + 127) / 128, 128, 0, m->o, v, u, B, L, D, rev, t);
+  }
+  return check_launch("sequential block");
+}
+
+// ------------------------------------------------------------------------------------------------
+// Jacobi block (Algorithm 1) with per-sample stopping and active-set compaction
+// ------------------------------------------------------------------------------------------------
+static int read_ctrl(tf_model* m) {
+  CU_OK(cudaMemcpyAsync(m->ctrl_host, m->ctrl, 2 * sizeof(int), cudaMemcpyDeviceToHost, m->stream));
+  CU_OK(cudaMemcpyAsync(m->ctrl_host + 3, m->ctrl + 2, 2 * sizeof(int), cudaMemcpyDeviceToHost, m->stream));
+  CU_OK(cudaMemcpyAsync(m->ctrl_host + 2, m->err, sizeof(int), cudaMemcpyDeviceToHost, m->stream));
+  CU_OK(cudaStreamSynchronize(m->stream));
+  if (m->ctrl_host[2] != 0) return fail(TF_ETIMEOUT, "device-side wait expired (code %d)", m->ctrl_host[2]);
+  if (m->ctrl_host[1] != 0) return fail(TF_ENONFINITE, "non-finite value in the convergence reduction");
+  return TF_OK;
+}
+
+// synchronise the stream and turn a recorded device-side timeout into an error
+static int sync_check(tf_model* m) {
+  CU_OK(cudaMemcpyAsync(m->ctrl_host + 2, m->err, sizeof(int), cudaMemcpyDeviceToHost, m->stream));
+  CU_OK(cudaStreamSynchronize(m->stream));
+  if (m->ctrl_host[2] != 0) return fail(TF_ETIMEOUT, "device-side wait expired (code %d)", m->ctrl_host[2]);
+  return TF_OK;
+}
+
+template <class T>
+static int run_jacobi_block(tf_model* m, int g, int B, const int* labels, const float* v, float* u, float tau,
+                            int max_iters, int init_mode, int* sweeps_out, int* iters_row) {
+  const size_t n = (size_t)B * m->L * m->D;
+  if (init_mode == 0) CU_OK(cudaMemsetAsync(u, 0, n * sizeof(float), m->stream));
+  else CU_OK(cudaMemcpyAsync(u, v, n * sizeof(float), cudaMemcpyDeviceToDevice, m->stream));
+  // precision policy (bf16 engine): which sweeps of a sample use two-term operands
+  int start_phase = 0;
+  float sw = -1.f;  // never escalate
+  if (sizeof(T) == 2) {
+    if (m->precision_mode == 2) start_phase = 1;
+    else if (m->precision_mode == 0 && tau >= 0.f && tau < m->single_ok_tau) sw = m->switch_threshold;
+  }
+  LAUNCH(m, KC_CTRL, jacobi_begin_kernel, 1, 256, 0, m->maxdiff, m->idx, m->phase, m->ctrl, B, start_phase);
+  int n_active = B, n_hp = start_phase ? B : 0, t = 0;
+  while (t < max_iters && n_active > 0) {
+    ++t;
+    const int n_lp = n_active - n_hp;
+    if (n_lp > 0) TF_TRY(run_pass<T>(m, g, n_lp, u, m->idx, labels, PASS_JACOBI, v, u, false));
+    if (n_hp > 0) TF_TRY(run_pass<T>(m, g, n_hp, u, m->idx + n_lp, labels, PASS_JACOBI, v, u, true));
+    LAUNCH(m, KC_CTRL, jacobi_finalize_kernel, 1, 32, 0, m->maxdiff, m->idx, m->idx_tmp, m->phase, m->ctrl, iters_row,
+           tau, sw, t);
+    if (tau >= 0.f || t == max_iters || m->trace_on) {
+      const int before = n_active;
+      TF_TRY(read_ctrl(m));
+      n_active = m->ctrl_host[0];
+      n_hp = m->ctrl_host[4];
+      if (m->trace_on) {
+        float top;
+        memcpy(&top, &m->ctrl_host[3], sizeof(float));
+        m->trace.push_back({g, t, before, top});
+      }
+    }
+  }
+  *sweeps_out = t;
+  return (tau >= 0.f && n_active > 0) ? TF_MAXITER : TF_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// whole-model drivers
+// ------------------------------------------------------------------------------------------------
+static int layout(tf_model* m, float* img, float* seq, int B, int to_seq) {
+  size_t n = (size_t)B * m->cfg.C * m->cfg.H * m->cfg.W;
+  int blocks = (int)((n + 255) / 256);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  LAUNCH(m, KC_LAYOUT, patchify_kernel, blocks, 256, 0, img, seq, B, m->cfg.C, m->cfg.H, m->cfg.W, m->cfg.patch, to_seq);
+  return check_launch("patchify_kernel");
+}
+
+template <class T>
+static int inverse_impl(tf_model* m, const float* z, const int* labels, int B, const uint8_t* policy, float tau,
+                        int max_iters, int init_mode, float* x, int* iters_block_host, int* iters_sample_dev) {
+  const int K = m->cfg.n_blocks;
+  float *v = m->seq_a, *u = m->seq_b;
+  m->trace.clear();
+  TF_TRY(layout(m, const_cast<float*>(z), v, B, 1));
+  int status = TF_OK;
+  for (int g = 0; g < K; ++g) {
+    int* iters_row = m->iters_sample + (size_t)g * m->cfg.max_batch;
+    int sweeps = m->L - 1;
+    if (policy[g] == 0) {
+      TF_TRY(run_sequential_block<T>(m, g, B, labels, v, u));
+      LAUNCH(m, KC_CTRL, fill_int_kernel, (B + 127) / 128, 128, 0, iters_row, B, m->L - 1);
+    } else {
+      int r = run_jacobi_block<T>(m, g, B, labels, v, u, tau, max_iters, init_mode, &sweeps, iters_row);
+      if (r < 0) return r;
+      if (r == TF_MAXITER) status = TF_MAXITER;
+    }
+    if (iters_block_host) iters_block_host[g] = sweeps;
+    float* tmp = v; v = u; u = tmp;
+  }
+  TF_TRY(layout(m, x, v, B, 0));
+  if (iters_sample_dev) {
+    for (int g = 0; g < K; ++g)
+      CU_OK(cudaMemcpyAsync(iters_sample_dev + (size_t)g * B, m->iters_sample + (size_t)g * m->cfg.max_batch,
+                            B * sizeof(int), cudaMemcpyDeviceToDevice, m->stream));
+  }
+  TF_TRY(sync_check(m));
+  return status;
+}
+
+template <class T>
+static int forward_impl(tf_model* m, const float* x, const int* labels, int B, float* z, float* logdet) {
+  float *u = m->seq_a, *v = m->seq_b;
+  TF_TRY(layout(m, const_cast<float*>(x), u, B, 1));
+  if (logdet) CU_OK(cudaMemsetAsync(logdet, 0, B * sizeof(float), m->stream));
+  for (int g = m->cfg.n_blocks - 1; g >= 0; --g) {
+    TF_TRY(run_pass<T>(m, g, B, u, nullptr, labels, PASS_FORWARD, nullptr, nullptr, false));
+    LAUNCH(m, KC_AFFINE, forward_affine_kernel, B, 256, 0, m->o, u, v, logdet, m->L, m->D, g & 1);
+    TF_TRY(check_launch("forward_affine_kernel"));
+    float* tmp = v; v = u; u = tmp;
+  }
+  return layout(m, z, u, B, 0);
+}
+
+// ------------------------------------------------------------------------------------------------
+// loading
+// ------------------------------------------------------------------------------------------------
+struct BlobReader {
+  const float* p;
+  const float* end;
+  const float* take(size_t n) {
+    const float* r = p;
+    p += n;
+    return r;
+  }
+};
+
+static int upload_f32(tf_model* m, float** dst, const float* src, size_t n) {
+  TF_TRY(dev_alloc(m, dst, n));
+  CU_OK(cudaMemcpy(*dst, src, n * sizeof(float), cudaMemcpyHostToDevice));
+  return TF_OK;
+}
+
+// matrix [N, K]: fp32 engine keeps fp32; bf16 engine converts on the device (round to nearest even)
+static int upload_matrix(tf_model* m, Matrix* W, const float* src, int N, int K, float* staging) {
+  W->N = N;
+  W->K = K;
+  size_t n = (size_t)N * K;
+  if (m->cfg.dtype == 0) {
+    float* w;
+    TF_TRY(upload_f32(m, &w, src, n));
+    W->w = w;
+    return TF_OK;
+  }
+  bf16* w;
+  TF_TRY(dev_alloc(m, &w, n));
+  CU_OK(cudaMemcpy(staging, src, n * sizeof(float), cudaMemcpyHostToDevice));
+  f32_to_bf16_kernel<<<148 * 4, 256>>>(staging, w, n);
+  CU_OK(cudaDeviceSynchronize());
+  W->w = w;
+  W->bn = (N % 256 == 0) ? 256 : 128;
+  return make_map_bf16(&W->map, w, (uint64_t)N, (uint64_t)K, (uint32_t)W->bn);
+}
+
+static size_t block_floats(const tf_config& c, int L, int D) {
+  size_t d = c.width, hid = (size_t)c.mlp_ratio * d;
+  size_t n = d * D + d + (size_t)L * d + (size_t)c.n_classes * d;
+  n += (size_t)c.n_layers * (2 * d + 3 * d * d + 3 * d + d * d + d + 2 * d + hid * d + hid + d * hid + d);
+  n += 2 * d + 2 * (size_t)D * d + 2 * D;
+  return n;
+}
+
+static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
+  const tf_config& c = m->cfg;
+  const int L = m->L, D = m->D, d = m->d, hid = m->hid;
+  const size_t want = 64 + 4 * block_floats(c, L, D) * c.n_blocks;
+  if (nbytes != want) return fail(TF_ESIZE, "weight blob is %zu bytes, configuration needs %zu", nbytes, want);
+  const int32_t* hdr = reinterpret_cast<const int32_t*>(blob);
+  const int32_t expect[13] = {0x31574654, 1, c.C, c.H, c.W, c.patch, c.n_blocks, c.n_layers, c.width, c.n_heads,
+                              c.mlp_ratio, c.n_classes, c.dtype};
+  for (int i = 0; i < 13; ++i)
+    if (hdr[i] != expect[i]) return fail(TF_ESIZE, "weight blob header field %d is %d, expected %d", i, hdr[i], expect[i]);
+
+  int dev = 0;
+  CU_OK(cudaGetDevice(&dev));
+  CU_OK(cudaDeviceGetAttribute(&m->num_sms, cudaDevAttrMultiProcessorCount, dev));
+
+  float* staging = nullptr;
+  size_t max_mat = (size_t)hid * d;
+  if ((size_t)3 * d * d > max_mat) max_mat = (size_t)3 * d * d;
+  if (c.dtype == 1) CU_OK(cudaMalloc(&staging, max_mat * sizeof(float)));
+  struct Guard { float* p; ~Guard() { if (p) cudaFree(p); } } guard{staging};
+
+  BlobReader rd{reinterpret_cast<const float*>(reinterpret_cast<const char*>(blob) + 64), nullptr};
+  m->blocks.resize(c.n_blocks);
+  std::vector<float> tmp;
+  for (int g = 0; g < c.n_blocks; ++g) {
+    BlockW& bw = m->blocks[g];
+    const float* w_in = rd.take((size_t)d * D);
+    tmp.resize((size_t)d * D);
+    for (int j = 0; j < d; ++j)
+      for (int cc = 0; cc < D; ++cc) tmp[(size_t)cc * d + j] = w_in[(size_t)j * D + cc];
+    TF_TRY(upload_f32(m, &bw.w_in_t, tmp.data(), tmp.size()));
+    TF_TRY(upload_f32(m, &bw.b_in, rd.take(d), d));
+    TF_TRY(upload_f32(m, &bw.pos, rd.take((size_t)L * d), (size_t)L * d));
+    bw.cls = nullptr;
+    if (c.n_classes > 0) TF_TRY(upload_f32(m, &bw.cls, rd.take((size_t)c.n_classes * d), (size_t)c.n_classes * d));
+    bw.layers.resize(c.n_layers);
+    for (LayerW& lw : bw.layers) {
+      TF_TRY(upload_f32(m, &lw.ln1_g, rd.take(d), d));
+      TF_TRY(upload_f32(m, &lw.ln1_b, rd.take(d), d));
+      TF_TRY(upload_matrix(m, &lw.w_qkv, rd.take((size_t)3 * d * d), 3 * d, d, staging));
+      TF_TRY(upload_f32(m, &lw.b_qkv, rd.take(3 * d), 3 * d));
+      TF_TRY(upload_matrix(m, &lw.w_o, rd.take((size_t)d * d), d, d, staging));
+      TF_TRY(upload_f32(m, &lw.b_o, rd.take(d), d));
+      TF_TRY(upload_f32(m, &lw.ln2_g, rd.take(d), d));
+      TF_TRY(upload_f32(m, &lw.ln2_b, rd.take(d), d));
+      TF_TRY(upload_matrix(m, &lw.w_1, rd.take((size_t)hid * d), hid, d, staging));
+      TF_TRY(upload_f32(m, &lw.b_1, rd.take(hid), hid));
+      TF_TRY(upload_matrix(m, &lw.w_2, rd.take((size_t)d * hid), d, hid, staging));
+      TF_TRY(upload_f32(m, &lw.b_2, rd.take(d), d));
+    }
+    TF_TRY(upload_f32(m, &bw.lnf_g, rd.take(d), d));
+    TF_TRY(upload_f32(m, &bw.lnf_b, rd.take(d), d));
+    // head: interleave rows so that outputs (2c, 2c+1) = (mu~_c, alpha~_c)
+    const float* w_out = rd.take((size_t)2 * D * d);
+    const float* b_out = rd.take((size_t)2 * D);
+    tmp.resize((size_t)2 * D * d);
+    std::vector<float> btmp(2 * D);
+    for (int cc = 0; cc < D; ++cc) {
+      memcpy(&tmp[(size_t)(2 * cc) * d], &w_out[(size_t)cc * d], d * sizeof(float));
+      memcpy(&tmp[(size_t)(2 * cc + 1) * d], &w_out[(size_t)(D + cc) * d], d * sizeof(float));
+      btmp[2 * cc] = b_out[cc];
+      btmp[2 * cc + 1] = b_out[D + cc];
+    }
+    TF_TRY(upload_matrix(m, &bw.w_out, tmp.data(), 2 * D, d, staging));
+    TF_TRY(upload_f32(m, &bw.b_out, btmp.data(), btmp.size()));
+  }
+
+  // workspace
+  const size_t B = c.max_batch, M = B * L, esz = c.dtype == 1 ? 2 : 4;
+  TF_TRY(dev_alloc(m, &m->seq_a, M * D));
+  TF_TRY(dev_alloc(m, &m->seq_b, M * D));
+  TF_TRY(dev_alloc(m, &m->h, M * d));
+  TF_TRY(dev_alloc(m, &m->o, M * 2 * D));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->xn), M * d * esz));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->qkv), M * 3 * d * esz));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->att), M * d * esz));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->mlp), M * hid * esz));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->kcache), (size_t)c.n_layers * M * d * esz));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->vcache), (size_t)c.n_layers * M * d * esz));
+  if (c.dtype == 1) {
+    TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->xn_lo), M * d * esz));
+    TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->qkv_lo), M * 3 * d * esz));
+    TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->att_lo), M * d * esz));
+    TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->mlp_lo), M * hid * esz));
+  }
+  TF_TRY(dev_alloc(m, &m->maxdiff, B));
+  TF_TRY(dev_alloc(m, &m->idx, B));
+  TF_TRY(dev_alloc(m, &m->idx_tmp, B));
+  TF_TRY(dev_alloc(m, &m->phase, B));
+  TF_TRY(dev_alloc(m, &m->ctrl, 8));
+  TF_TRY(dev_alloc(m, &m->err, 1));
+  TF_TRY(dev_alloc(m, &m->iters_sample, (size_t)c.n_blocks * B));
+  TF_TRY(dev_alloc(m, &m->io_z, B * c.C * c.H * c.W));
+  TF_TRY(dev_alloc(m, &m->io_x, B * c.C * c.H * c.W));
+  TF_TRY(dev_alloc(m, &m->io_labels, B));
+  CU_OK(cudaMemset(m->ctrl, 0, 8 * sizeof(int)));
+  CU_OK(cudaMemset(m->err, 0, sizeof(int)));
+  CU_OK(cudaMemset(m->iters_sample, 0, (size_t)c.n_blocks * B * sizeof(int)));
+  CU_OK(cudaMallocHost(&m->ctrl_host, 8 * sizeof(int)));
+  if (c.dtype == 1) {
+    TF_TRY(make_map_bf16(&m->map_xn, m->xn, M, d, tc::BM));
+    TF_TRY(make_map_bf16(&m->map_att, m->att, M, d, tc::BM));
+    TF_TRY(make_map_bf16(&m->map_mlp, m->mlp, M, hid, tc::BM));
+    TF_TRY(make_map_bf16(&m->map_xn_lo, m->xn_lo, M, d, tc::BM));
+    TF_TRY(make_map_bf16(&m->map_att_lo, m->att_lo, M, d, tc::BM));
+    TF_TRY(make_map_bf16(&m->map_mlp_lo, m->mlp_lo, M, hid, tc::BM));
+    CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               attn::smem_bytes<true>()));
+    CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               attn::smem_bytes<false>()));
+  }
+  CU_OK(cudaDeviceSynchronize());
+  return TF_OK;
+}
+
+static int check_call(tf_model* m, int B) {
+  if (!m) return fail(TF_EINVAL, "model is NULL");
+  if (B < 1 || B > m->cfg.max_batch) return fail(TF_EINVAL, "B=%d outside [1, max_batch=%d]", B, m->cfg.max_batch);
+  return TF_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// C ABI
+// ------------------------------------------------------------------------------------------------
+extern "C" {
+
+const char* tf_last_error(void) { return g_err; }
+
+int tf_load(const tf_config* cfg, const void* weights_host, size_t nbytes, tf_model** out) {
+  g_err[0] = 0;
+  if (!cfg || !weights_host || !out) return fail(TF_EINVAL, "NULL argument");
+  *out = nullptr;
+  const tf_config& c = *cfg;
+  if (c.C < 1 || c.H < 1 || c.W < 1 || c.patch < 1 || c.H % c.patch || c.W % c.patch)
+    return fail(TF_EINVAL, "image %dx%dx%d not divisible by patch %d", c.C, c.H, c.W, c.patch);
+  if (c.n_blocks < 1 || c.n_layers < 1 || c.width < 4 || c.n_heads < 1 || c.width % c.n_heads || c.width % 4 ||
+      c.mlp_ratio < 1 || c.n_classes < 0 || c.max_batch < 1)
+    return fail(TF_EINVAL, "bad model dimensions");
+  if (c.dtype != 0 && c.dtype != 1) return fail(TF_EINVAL, "dtype must be 0 (fp32) or 1 (bf16)");
+  if (c.dtype == 1 && (c.width % 64 || c.width / c.n_heads != 64))
+    return fail(TF_EINVAL, "bf16 engine needs width %% 64 == 0 and head_dim == 64");
+  if (c.width > 2048) return fail(TF_EINVAL, "width > 2048 not supported");
+  tf_model* m = new (std::nothrow) tf_model();
+  if (!m) return fail(TF_ENOMEM, "host allocation failed");
+  m->cfg = c;
+  m->L = (c.H / c.patch) * (c.W / c.patch);
+  m->D = c.C * c.patch * c.patch;
+  m->d = c.width;
+  m->hid = c.mlp_ratio * c.width;
+  m->hd = c.width / c.n_heads;
+  if (m->L < 2) { delete m; return fail(TF_EINVAL, "need at least 2 tokens"); }
+  int r = load_impl(m, weights_host, nbytes);
+  if (r != TF_OK) {
+    tf_free(m);
+    return r;
+  }
+  *out = m;
+  return TF_OK;
+}
+
+void tf_free(tf_model* m) {
+  if (!m) return;
+  cudaDeviceSynchronize();
+  m->prof_collect();
+  for (cudaEvent_t e : m->ev_pool) cudaEventDestroy(e);
+  for (void* p : m->allocs) cudaFree(p);
+  if (m->ctrl_host) cudaFreeHost(m->ctrl_host);
+  delete m;
+}
+
+int tf_forward(tf_model* m, const float* x_dev, const int32_t* labels_dev, int32_t B, float* z_dev, float* logdet_dev,
+               void* cuda_stream) {
+  g_err[0] = 0;
+  TF_TRY(check_call(m, B));
+  if (!x_dev || !z_dev) return fail(TF_EINVAL, "NULL buffer");
+  if (m->cfg.n_classes > 0 && !labels_dev) return fail(TF_EINVAL, "class-conditional model needs labels");
+  m->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  return m->cfg.dtype == 1 ? forward_impl<bf16>(m, x_dev, labels_dev, B, z_dev, logdet_dev)
+                           : forward_impl<float>(m, x_dev, labels_dev, B, z_dev, logdet_dev);
+}
+
+int tf_inverse_jacobi(tf_model* m, const float* z_dev, const int32_t* labels_dev, int32_t B, const uint8_t* policy_host,
+                      float tau, int32_t max_iters, int32_t init_mode, float* x_dev, int32_t* iters_block_host,
+                      int32_t* iters_sample_dev, void* cuda_stream) {
+  g_err[0] = 0;
+  TF_TRY(check_call(m, B));
+  if (!z_dev || !x_dev || !policy_host) return fail(TF_EINVAL, "NULL buffer");
+  if (m->cfg.n_classes > 0 && !labels_dev) return fail(TF_EINVAL, "class-conditional model needs labels");
+  if (max_iters < 1) return fail(TF_EINVAL, "max_iters must be >= 1");
+  if (init_mode != 0 && init_mode != 1) return fail(TF_EINVAL, "init_mode must be 0 or 1");
+  if (tau != tau) return fail(TF_EINVAL, "tau is NaN");
+  for (int g = 0; g < m->cfg.n_blocks; ++g)
+    if (policy_host[g] > 1) return fail(TF_EINVAL, "policy[%d]=%d is neither 0 nor 1", g, (int)policy_host[g]);
+  m->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  return m->cfg.dtype == 1 ? inverse_impl<bf16>(m, z_dev, labels_dev, B, policy_host, tau, max_iters, init_mode, x_dev,
+                                                iters_block_host, iters_sample_dev)
+                           : inverse_impl<float>(m, z_dev, labels_dev, B, policy_host, tau, max_iters, init_mode, x_dev,
+                                                 iters_block_host, iters_sample_dev);
+}
+
+int tf_inverse_sequential(tf_model* m, const float* z_dev, const int32_t* labels_dev, int32_t B, float* x_dev,
+                          void* cuda_stream) {
+  if (!m) return fail(TF_EINVAL, "model is NULL");
+  std::vector<uint8_t> policy(m->cfg.n_blocks, 0);
+  return tf_inverse_jacobi(m, z_dev, labels_dev, B, policy.data(), 0.f, 1, 0, x_dev, nullptr, nullptr, cuda_stream);
+}
+
+int tf_inverse_jacobi_host(tf_model* m, const float* z_host, const int32_t* labels_host, int32_t B,
+                           const uint8_t* policy_host, float tau, int32_t max_iters, int32_t init_mode, float* x_host,
+                           int32_t* iters_block_host, int32_t* iters_sample_host, void* cuda_stream) {
+  g_err[0] = 0;
+  TF_TRY(check_call(m, B));
+  if (!z_host || !x_host) return fail(TF_EINVAL, "NULL buffer");
+  if (m->cfg.n_classes > 0 && !labels_host) return fail(TF_EINVAL, "class-conditional model needs labels");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  size_t n = (size_t)B * m->cfg.C * m->cfg.H * m->cfg.W;
+  CU_OK(cudaMemcpyAsync(m->io_z, z_host, n * sizeof(float), cudaMemcpyHostToDevice, st));
+  if (labels_host) CU_OK(cudaMemcpyAsync(m->io_labels, labels_host, B * sizeof(int), cudaMemcpyHostToDevice, st));
+  int r = tf_inverse_jacobi(m, m->io_z, labels_host ? m->io_labels : nullptr, B, policy_host, tau, max_iters, init_mode,
+                            m->io_x, iters_block_host, nullptr, cuda_stream);
+  if (r < 0) return r;
+  CU_OK(cudaMemcpyAsync(x_host, m->io_x, n * sizeof(float), cudaMemcpyDeviceToHost, st));
+  if (iters_sample_host)
+    for (int g = 0; g < m->cfg.n_blocks; ++g)
+      CU_OK(cudaMemcpyAsync(iters_sample_host + (size_t)g * B, m->iters_sample + (size_t)g * m->cfg.max_batch,
+                            B * sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU_OK(cudaStreamSynchronize(st));
+  return r;
+}
+
+int tf_jacobi_update(const float* o_dev, const float* v_dev, float* u_dev, float* maxdiff_dev, int32_t B, int32_t L,
+                     int32_t D, int32_t reversed, void* cuda_stream) {
+  g_err[0] = 0;
+  if (!o_dev || !v_dev || !u_dev || !maxdiff_dev) return fail(TF_EINVAL, "NULL buffer");
+  if (B < 1 || L < 2 || D < 1) return fail(TF_EINVAL, "bad sizes");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  CU_OK(cudaMemsetAsync(maxdiff_dev, 0, B * sizeof(float), st));
+  size_t n = (size_t)B * L * D;
+  int blocks = (int)((n + 255) / 256);
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  jacobi_update_kernel<<<blocks, 256, 0, st>>>(o_dev, v_dev, u_dev, maxdiff_dev, nullptr, B * L, L, D, reversed, 0);
+  return check_launch("jacobi_update_kernel");
+}
+
+static int* g_gemm_err = nullptr;  // error word of the model-less GEMM entry point (allocated once)
+
+int tf_gemm_bf16(const void* a_dev, const void* w_dev, const float* bias_dev, float* c_dev, int32_t M, int32_t N,
+                 int32_t K, void* cuda_stream) {
+  g_err[0] = 0;
+  if (!a_dev || !w_dev || !c_dev) return fail(TF_EINVAL, "NULL buffer");
+  if (M < 1 || N < 8 || K < 64 || K % 64 || N % 8) return fail(TF_EINVAL, "need M>=1, N%%8==0, K%%64==0");
+  if (!g_gemm_err) {
+    CU_OK(cudaMalloc(&g_gemm_err, sizeof(int)));
+    CU_OK(cudaMemset(g_gemm_err, 0, sizeof(int)));
+  }
+  int dev = 0, sms = 148;
+  CU_OK(cudaGetDevice(&dev));
+  CU_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const int bn = (N % 256 == 0) ? 256 : 128;
+  CUtensorMap ma, mw;
+  TF_TRY(make_map_bf16(&ma, a_dev, M, K, tc::BM));
+  TF_TRY(make_map_bf16(&mw, w_dev, N, K, bn));
+  EpiStore<float, false> epi{c_dev, bias_dev, N};
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (bn == 256) return launch_gemm_tc<256, 4>(nullptr, 0, st, ma, nullptr, mw, M, N, K, epi, g_gemm_err, sms, nullptr);
+  return launch_gemm_tc<128, 6>(nullptr, 0, st, ma, nullptr, mw, M, N, K, epi, g_gemm_err, sms, nullptr);
+}
+
+int tf_gemm_status(void* cuda_stream) {
+  g_err[0] = 0;
+  CU_OK(cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(cuda_stream)));
+  if (!g_gemm_err) return TF_OK;
+  int e = 0;
+  CU_OK(cudaMemcpy(&e, g_gemm_err, sizeof(int), cudaMemcpyDeviceToHost));
+  if (e != 0) return fail(TF_ETIMEOUT, "device-side wait expired in tf_gemm_bf16 (code %d)", e);
+  return TF_OK;
+}
+
+int tf_profile_enable(tf_model* m, int32_t on) {
+  if (!m) return fail(TF_EINVAL, "model is NULL");
+  cudaDeviceSynchronize();
+  m->prof_collect();
+  for (int c = 0; c < KC_COUNT; ++c) { m->prof_ms[c] = 0; m->prof_n[c] = 0; }
+  m->prof_on = on != 0;
+  return TF_OK;
+}
+
+int tf_profile_read(tf_model* m, const char** names, double* ms, int64_t* launches, int32_t cap) {
+  if (!m) return fail(TF_EINVAL, "model is NULL");
+  m->prof_collect();
+  for (int c = 0; c < KC_COUNT && c < cap; ++c) {
+    if (names) names[c] = kKernelClassNames[c];
+    if (ms) ms[c] = m->prof_ms[c];
+    if (launches) launches[c] = m->prof_n[c];
+  }
+  return KC_COUNT;
+}
+
+int tf_set_precision(tf_model* m, int32_t mode, float switch_threshold, float single_ok_tau) {
+  if (!m) return fail(TF_EINVAL, "model is NULL");
+  if (mode < 0 || mode > 2) return fail(TF_EINVAL, "precision mode must be 0, 1 or 2");
+  m->precision_mode = mode;
+  m->switch_threshold = switch_threshold > 0.f ? switch_threshold : 0.03125f;
+  m->single_ok_tau = single_ok_tau > 0.f ? single_ok_tau : 0.015625f;
+  return TF_OK;
+}
+
+int tf_trace_enable(tf_model* m, int32_t on) {
+  if (!m) return fail(TF_EINVAL, "model is NULL");
+  m->trace_on = on != 0;
+  m->trace.clear();
+  return TF_OK;
+}
+
+int tf_trace_read(tf_model* m, int32_t* block, int32_t* sweep, int32_t* active, float* maxdiff, int32_t cap) {
+  if (!m) return fail(TF_EINVAL, "model is NULL");
+  int n = (int)m->trace.size();
+  for (int i = 0; i < n && i < cap; ++i) {
+    if (block) block[i] = m->trace[i].block;
+    if (sweep) sweep[i] = m->trace[i].sweep;
+    if (active) active[i] = m->trace[i].active;
+    if (maxdiff) maxdiff[i] = m->trace[i].maxdiff;
+  }
+  return n;
+}
+
+int64_t tf_launch_count(tf_model* m) { return m ? m->launches : 0; }
+int64_t tf_device_bytes(tf_model* m) { return m ? m->device_bytes : 0; }
+
+}  // extern "C"
