@@ -152,12 +152,14 @@ int tf_gemm_status(void* cuda_stream);
  * Profiling aid: when enabled, calls on this model bracket every kernel class with CUDA events on
  * the caller's stream and accumulate elapsed milliseconds and launch counts.
  *   tf_profile_enable(m, on): switch on/off and reset the counters.
- *   tf_profile_read(m, names, ms, launches, cap): fills up to cap entries, returns how many
- *     classes exist; names[i] points to a static string.
+ *   tf_profile_read(m, names, ms, launches, rows, cap): fills up to cap entries, returns how many
+ *     classes exist; names[i] points to a static string; rows[i] is the number of activation
+ *     rows (tokens of a sweep, samples of a sequential step) the class's launches processed.
  *   tf_launch_count(m): kernels launched by the library on this model since load (always counted).
  */
 int tf_profile_enable(tf_model* m, int32_t on);
-int tf_profile_read(tf_model* m, const char** names, double* ms, int64_t* launches, int32_t cap);
+int tf_profile_read(tf_model* m, const char** names, double* ms, int64_t* launches, double* rows,
+                    int32_t cap);
 int64_t tf_launch_count(tf_model* m);
 
 /*

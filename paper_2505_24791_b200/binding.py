@@ -51,7 +51,7 @@ def lib():
         L.tf_gemm_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
         L.tf_gemm_status.argtypes = [vp]
         L.tf_profile_enable.argtypes = [vp, i32]
-        L.tf_profile_read.argtypes = [vp, vp, vp, vp, i32]
+        L.tf_profile_read.argtypes = [vp, vp, vp, vp, vp, i32]
         L.tf_set_precision.argtypes = [vp, i32, f32, f32]
         L.tf_trace_enable.argtypes = [vp, i32]
         L.tf_trace_read.argtypes = [vp, vp, vp, vp, vp, i32]
@@ -149,13 +149,14 @@ def tf_profile_enable(m, on):
 
 
 def tf_profile_read(m):
-    """-> {kernel class: (milliseconds, launches)} accumulated since tf_profile_enable."""
+    """-> {kernel class: (milliseconds, launches, rows)} accumulated since tf_profile_enable."""
     cap = 64
     names = (C.c_char_p * cap)()
     ms = (C.c_double * cap)()
     n = (C.c_int64 * cap)()
-    k = _check(lib().tf_profile_read(m, names, ms, n, cap))
-    return {names[i].decode(): (ms[i], n[i]) for i in range(min(k, cap))}
+    rows = (C.c_double * cap)()
+    k = _check(lib().tf_profile_read(m, names, ms, n, rows, cap))
+    return {names[i].decode(): (ms[i], n[i], rows[i]) for i in range(min(k, cap))}
 
 
 def tf_set_precision(m, mode, switch_threshold=0.0, single_ok_tau=0.0):

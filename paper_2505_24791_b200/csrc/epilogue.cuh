@@ -1,6 +1,11 @@
-// GEMM epilogue functors.  A GEMM kernel hands each functor NC consecutive accumulator columns of
-// one output row: apply<NC>(row, col0, v, n_valid) with col0 % NC == 0 and n_valid = min(NC, N-col0).
-// NC is 4 for the SIMT GEMM and 32 for the tcgen05 GEMM (one TMEM lane chunk per thread).
+// GEMM epilogue functors, with two calling conventions.
+//   * apply<NC>(row, col0, v, n_valid): the thread owns NC consecutive accumulator columns of one
+//     output row (col0 % NC == 0, n_valid = min(NC, N - col0)).  Used by the SIMT GEMM (NC = 4).
+//   * col_const(col) / store(row, col, acc, cc, lane): the tcgen05 GEMM transposes each 32x32
+//     accumulator chunk through shared memory, so that the 32 lanes of a warp hold 32 consecutive
+//     columns of ONE row and every global access of a warp is a contiguous row segment.
+//     col_const is evaluated once per chunk (the bias of the lane's column), store once per row.
+//     All 32 lanes call store together (it may shuffle); lanes with col >= N pass col_ok = false.
 #pragma once
 #include "common.cuh"
 
@@ -41,6 +46,27 @@ struct EpiStore {
       }
     }
   }
+  __device__ __forceinline__ float col_const(int col, bool col_ok) const {
+    return (bias != nullptr && col_ok) ? bias[col] : 0.f;
+  }
+  __device__ __forceinline__ void store(int row, int col, float acc, float cc, bool col_ok, int) const {
+    float x = acc + cc;
+    if (GELU) x = (sizeof(OutT) == 2) ? gelu_erf_fast(x) : gelu_erf(x);
+    if (!col_ok) return;
+    const size_t e = (size_t)row * ldc + col;
+    if constexpr (sizeof(OutT) == 4) {
+      out[e] = from_f32<OutT>(x);
+    } else {
+      const bf16 hi = __float2bfloat16_rn(x);
+      out[e] = hi;
+      if (out_lo != nullptr) out_lo[e] = __float2bfloat16_rn(x - __bfloat162float(hi));
+    }
+  }
+  template <int R>
+  __device__ __forceinline__ void store_rows(int row0, int col, const float (&acc)[R], float cc, bool col_ok, int lane) const {
+#pragma unroll
+    for (int r = 0; r < R; ++r) store(row0 + r, col, acc[r], cc, col_ok, lane);
+  }
   template <int NC>
   __device__ __forceinline__ void store_bf16(OutT* p, const float (&r)[NC], int nv) const {
     if (nv == NC && (ldc % 8) == 0) {
@@ -72,6 +98,24 @@ struct EpiResid {  // h[row, col] += acc + bias[col]   (fp32 residual stream, in
   float* h;
   const float* bias;
   int ldc;
+  __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
+  __device__ __forceinline__ void store(int row, int col, float acc, float cc, bool col_ok, int) const {
+    if (col_ok) {
+      float* p = h + (size_t)row * ldc + col;
+      *p = *p + (acc + cc);
+    }
+  }
+  // all loads of the residual stream are issued before the first store, so their latencies overlap
+  template <int R>
+  __device__ __forceinline__ void store_rows(int row0, int col, const float (&acc)[R], float cc, bool col_ok, int) const {
+    if (!col_ok) return;
+    float* p = h + (size_t)row0 * ldc + col;
+    float old[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) old[r] = __ldcg(p + (size_t)r * ldc);
+#pragma unroll
+    for (int r = 0; r < R; ++r) p[(size_t)r * ldc] = old[r] + (acc[r] + cc);
+  }
   template <int NC>
   __device__ __forceinline__ void apply(int row, int col0, const float (&v)[NC], int nv) const {
     float* p = h + (size_t)row * ldc + col0;
@@ -129,6 +173,36 @@ struct EpiHeadUpdate {
   const int* idx;      // [n_slots] slot -> sample (null = identity)
   const float* bias;   // [2D] interleaved
   int L, D, reversed;
+  __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
+  // lane-per-column form: even lanes hold mu~_c, the next lane alpha~_c
+  __device__ __forceinline__ void store(int row, int col, float acc, float cc, bool col_ok, int lane) const {
+    const float mine = acc + cc;
+    const float al = __shfl_down_sync(0xffffffffu, mine, 1);
+    const int s = row / L, l = row - s * L;
+    const int b = idx ? idx[s] : s;
+    float df = 0.f;
+    if (col_ok && (lane & 1) == 0) {
+      const int c = col >> 1;
+      const bool upd = l < L - 1;  // the last position's head output is unused: that row copies token 0
+      const size_t e = ((size_t)b * L + tok_index(upd ? l + 1 : 0, L, reversed)) * D + c;
+      const float old = u[e], vv = v[e];
+      const float nw = upd ? fmaf(vv, expf(al), mine) : vv;
+      u[e] = nw;
+      df = fabsf(nw - old);
+    }
+    // NaN-propagating max over the warp, then one atomic per row
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float other = __shfl_xor_sync(0xffffffffu, df, o);
+      df = (other > df || other != other) ? other : df;
+    }
+    if (lane == 0) atomic_max_nonneg(maxdiff + b, df);
+  }
+  template <int R>
+  __device__ __forceinline__ void store_rows(int row0, int col, const float (&acc)[R], float cc, bool col_ok, int lane) const {
+#pragma unroll
+    for (int r = 0; r < R; ++r) store(row0 + r, col, acc[r], cc, col_ok, lane);
+  }
   template <int NC>
   __device__ __forceinline__ void apply(int row, int col0, const float (&acc)[NC], int nv) const {
     int s = row / L, l = row - s * L;

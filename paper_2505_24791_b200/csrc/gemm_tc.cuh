@@ -7,8 +7,9 @@
 //   * optionally A is a two-term bf16 pair (hi + lo, about 16 significant bits): the same tile then
 //     accumulates A_hi W^T + A_lo W^T;
 //   * the kernel is persistent: gridDim.x CTAs walk the tile list with a fixed stride;
-//   * warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 =
-//     epilogue (tcgen05.ld -> registers -> functor).
+//   * warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..9 =
+//     epilogue (tcgen05.ld -> registers -> 32x32 transpose in shared memory -> functor, so that a
+//     warp's global accesses are contiguous row segments).
 // Every wait is bounded by wall time; a wait that expires records a code in *err and every role
 // leaves its loops, so the kernel always returns and frees its tensor memory.
 // No cluster launch and no multicast is used: each CTA loads its own operands.
@@ -23,7 +24,8 @@ namespace tc {
 constexpr int BM = 128;
 constexpr int BK = 64;  // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_EPI_WARPS = 8;  // two warps per TMEM lane quadrant, alternating 32-column chunks
+constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -139,7 +141,9 @@ struct SmemLayout {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
   static constexpr int NUM_BARS = 2 * STAGES + 4;
-  static constexpr int TOTAL = BAR_OFFSET + NUM_BARS * 8 + 16 + 1024;  // + tmem slot + alignment slack
+  static constexpr int STAGE_OUT_OFFSET = BAR_OFFSET + NUM_BARS * 8 + 16;  // after barriers + tmem slot
+  static constexpr int STAGE_OUT_BYTES = NUM_EPI_WARPS * 32 * 33 * 4;  // one padded 32x32 fp32 chunk per epilogue warp
+  static constexpr int TOTAL = STAGE_OUT_OFFSET + STAGE_OUT_BYTES + 1024;  // + alignment slack
 };
 
 template <int BN, int STAGES, class Epi>
@@ -178,7 +182,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 4);
+      mbar_init(tempty_bar(a), NUM_EPI_WARPS);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -245,6 +249,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int quad = warp & 3;  // TMEM lane quadrant this warp may read
+    const int cgroup = (warp - 2) >> 2;  // which of the NUM_EPI_WARPS/4 column groups of a quadrant
+    float* stage_out = reinterpret_cast<float*>(smem + SL::STAGE_OUT_OFFSET) + (warp - 2) * (32 * 33);
     bool ok = true;
     int it = 0;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
@@ -253,17 +259,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint32_t acc_phase = (it >> 1) & 1;
       if (!mbar_wait(tfull_bar(acc), acc_phase, err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
       tcgen05_fence_after();
-      const int row = m0 + quad * 32 + lane;
+      const int row0 = m0 + quad * 32;
+      const int nrows = (M - row0) < 32 ? (M - row0) : 32;  // rows of this warp inside the matrix (may be <= 0)
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int c = cgroup; c < BN / 32; c += NUM_EPI_WARPS / 4) {
         const int col0 = n0 + c * 32;
         if (col0 >= N) break;  // uniform across the warp
         float v[32];
         tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c * 32), v);
-        if (row < M) {
-          const int nv = (N - col0) < 32 ? (N - col0) : 32;
-          epi.template apply<32>(row, col0, v, nv);
+        // transpose through shared memory: lane = row on the way in, lane = column on the way out
+#pragma unroll
+        for (int j = 0; j < 32; ++j) stage_out[lane * 33 + j] = v[j];
+        __syncwarp();
+        const int col = col0 + lane;
+        const bool col_ok = col < N;
+        const float cc = epi.col_const(col, col_ok);
+        if (nrows == 32) {
+#pragma unroll
+          for (int r0 = 0; r0 < 32; r0 += 8) {
+            float a[8];
+#pragma unroll
+            for (int r = 0; r < 8; ++r) a[r] = stage_out[(r0 + r) * 33 + lane];
+            epi.template store_rows<8>(row0 + r0, col, a, cc, col_ok, lane);
+          }
+        } else {
+          for (int r = 0; r < nrows; ++r) epi.store(row0 + r, col, stage_out[r * 33 + lane], cc, col_ok, lane);
         }
+        __syncwarp();
       }
       tcgen05_fence_before();
       __syncwarp();

@@ -11,6 +11,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <string>
 #include <vector>
 
@@ -20,6 +21,7 @@
 #include "epilogue.cuh"
 #include "gemm_tc.cuh"
 #include "kernels_simt.cuh"
+#include "seq_decode.cuh"
 
 // ------------------------------------------------------------------------------------------------
 // errors
@@ -123,6 +125,14 @@ struct tf_model {
   float switch_threshold = 0.03125f;   // a sample's sweeps use two-term operands once its max|du| <= this
   float single_ok_tau = 0.015625f;     // tau at or above this never escalates
   int* ctrl_host = nullptr;  // pinned: n_active, nonfinite, device error
+  // sequential decoding on the bf16 engine: step counter on the device, model-owned copy of the labels
+  // (fixed address for captured graphs), one instantiated graph of `unroll` steps per (block, batch)
+  int* step_ctr = nullptr;
+  int* labels_own = nullptr;
+  cudaStream_t cap_stream = nullptr;
+  struct SeqGraph { cudaGraphExec_t exec = nullptr; int unroll = 0; int nodes = 0; };
+  std::map<std::pair<int, int>, SeqGraph> seq_graphs;  // (block g, B)
+  bool use_graphs = true;
   float *io_z = nullptr, *io_x = nullptr;  // staging for the host-buffer entry point
   int* io_labels = nullptr;
   cudaStream_t stream = nullptr;
@@ -133,6 +143,8 @@ struct tf_model {
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> ev_pending[KC_COUNT];
   double prof_ms[KC_COUNT] = {0};
   int64_t prof_n[KC_COUNT] = {0};
+  double prof_rows[KC_COUNT] = {0};  // activation rows the timed launches of a class processed
+  int64_t cur_rows = 0;              // rows of the launches being issued (set by the pass drivers)
   cudaEvent_t cur_start = nullptr;
   // convergence trace (one record per sweep of the last inverse call)
   struct TraceRec { int block, sweep, active; float maxdiff; };
@@ -161,6 +173,7 @@ struct tf_model {
       cudaEvent_t e = get_event();
       cudaEventRecord(e, stream);
       ev_pending[cls].push_back({cur_start, e});
+      prof_rows[cls] += (double)cur_rows;
     }
   }
   void prof_collect() {
@@ -287,6 +300,7 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
   const CUtensorMap* mal = hp ? &m->map_att_lo : nullptr;
   const CUtensorMap* mml = hp ? &m->map_mlp_lo : nullptr;
   int ethreads = d < 256 ? d : 256;
+  m->cur_rows = M;
   LAUNCH(m, KC_EMBED, embed_kernel, M, ethreads, D * sizeof(float), u_src, idx, labels, bw.w_in_t, bw.b_in, bw.pos,
          bw.cls, m->h, L, D, d, rev, -1);
   TF_TRY(check_launch("embed_kernel"));
@@ -339,6 +353,7 @@ static int run_sequential_block(tf_model* m, int g, int B, const int* labels, co
   const size_t layer_stride = (size_t)m->cfg.max_batch * L * d;
   const float scale = 1.0f / sqrtf((float)m->hd);
   int ethreads = d < 256 ? d : 256;
+  m->cur_rows = B;
   LAUNCH(m, KC_SEQ_UPDATE, copy_first_token_kernel, (B * D + 127) / 128, 128, 0, v, u, B, L, D, rev);
   for (int t = 0; t + 1 < L; ++t) {
     LAUNCH(m, KC_SEQ_EMBED, embed_kernel, B, ethreads, D * sizeof(float), u, (const int*)nullptr, labels, bw.w_in_t,
@@ -362,6 +377,129 @@ static int run_sequential_block(tf_model* m, int g, int B, const int* labels, co
     LAUNCH(m, KC_SEQ_UPDATE, seq_update_kernel, (B * D + 127) / 128, 128, 0, m->o, v, u, B, L, D, rev, t);
   }
   return check_launch("sequential block");
+}
+
+// ---- bf16 engine: fused-LayerNorm skinny GEMMs on tensor cores, replayed from a CUDA graph -------
+template <bool LN, class Epi>
+static int seq_gemm(tf_model* m, int cls, const void* A, const float* gamma, const float* beta, const Matrix& W, int B,
+                    const Epi& epi, int step_off) {
+  const int N = W.N, K = W.K, n_steps = m->L - 1;
+  // k-splits per CTA need K % (32 * splits) == 0; prefer narrow column slices (more CTAs) while they fit
+  int nc = 32;
+  if (K % 256 == 0 && N / 8 <= 2 * m->num_sms) nc = 8;
+  else if (K % 128 == 0 && N / 16 <= 2 * m->num_sms) nc = 16;
+  dim3 grid((N + nc - 1) / nc, (B + seq::ROWS - 1) / seq::ROWS);
+  const bf16* w = reinterpret_cast<const bf16*>(W.w);
+  const int smem = seq::gemm_smem_bytes();
+  if (nc == 8)
+    LAUNCH(m, cls, (seq::seq_gemm_kernel<8, LN, Epi>), grid, seq::THREADS, smem, A, gamma, beta, w, B, N, K, epi,
+           m->step_ctr, step_off, n_steps);
+  else if (nc == 16)
+    LAUNCH(m, cls, (seq::seq_gemm_kernel<16, LN, Epi>), grid, seq::THREADS, smem, A, gamma, beta, w, B, N, K, epi,
+           m->step_ctr, step_off, n_steps);
+  else
+    LAUNCH(m, cls, (seq::seq_gemm_kernel<32, LN, Epi>), grid, seq::THREADS, smem, A, gamma, beta, w, B, N, K, epi,
+           m->step_ctr, step_off, n_steps);
+  return TF_OK;
+}
+
+template <bool LN, class Epi>
+static int seq_gemm_configure() {
+  const int smem = seq::gemm_smem_bytes();
+  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<8, LN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<16, LN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<32, LN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  return TF_OK;
+}
+
+// kernels of decoding steps step_off .. step_off+count-1 relative to the device step counter
+static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const float* v, float* u, int count) {
+  const BlockW& bw = m->blocks[g];
+  const int L = m->L, D = m->D, d = m->d, rev = g & 1, nl = m->cfg.n_layers, heads = m->cfg.n_heads;
+  bf16* q = reinterpret_cast<bf16*>(m->qkv);
+  bf16* att = reinterpret_cast<bf16*>(m->att);
+  bf16* mlp = reinterpret_cast<bf16*>(m->mlp);
+  const size_t layer_stride = (size_t)m->cfg.max_batch * L * d;
+  const float scale = 1.0f / sqrtf((float)m->hd);
+  const int ethreads = d < 256 ? d : 256;
+  m->cur_rows = B;
+  for (int s = 0; s < count; ++s) {
+    for (int i = 0; i < nl; ++i) {
+      const LayerW& lw = bw.layers[i];
+      bf16* kc = reinterpret_cast<bf16*>(m->kcache) + i * layer_stride;
+      bf16* vc = reinterpret_cast<bf16*>(m->vcache) + i * layer_stride;
+      TF_TRY((seq_gemm<true>(m, KC_SEQ_GEMM, m->h, lw.ln1_g, lw.ln1_b, lw.w_qkv, B,
+                             seq::EpiQKV{q, kc, vc, lw.b_qkv, d, L, heads}, s)));
+      LAUNCH(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, q, kc, vc, att, L, d, heads,
+             scale * 1.4426950408889634f, m->step_ctr, s, L - 1);
+      TF_TRY((seq_gemm<false>(m, KC_SEQ_GEMM, att, nullptr, nullptr, lw.w_o, B, seq::EpiResidual{m->h, lw.b_o, d}, s)));
+      TF_TRY((seq_gemm<true>(m, KC_SEQ_GEMM, m->h, lw.ln2_g, lw.ln2_b, lw.w_1, B, seq::EpiGelu{mlp, lw.b_1, m->hid}, s)));
+      TF_TRY((seq_gemm<false>(m, KC_SEQ_GEMM, mlp, nullptr, nullptr, lw.w_2, B, seq::EpiResidual{m->h, lw.b_2, d}, s)));
+    }
+    TF_TRY((seq_gemm<true>(m, KC_SEQ_GEMM, m->h, bw.lnf_g, bw.lnf_b, bw.w_out, B, seq::EpiHead{m->o, bw.b_out, 2 * D}, s)));
+    LAUNCH(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, B, ethreads, D * sizeof(float), m->o, v, u, labels, bw.w_in_t,
+           bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 0, m->step_ctr, s, L - 1);
+  }
+  return check_launch("sequential step kernels");
+}
+
+static int seq_unroll(int n_steps) {  // steps per graph: a divisor of n_steps close to 16, so no step is a no-op
+  int best = 1;
+  for (int c = 1; c <= 32 && c <= n_steps; ++c)
+    if (n_steps % c == 0) best = c;
+  return best >= 4 ? best : (n_steps < 16 ? n_steps : 16);
+}
+
+static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* labels, const float* v, float* u) {
+  const BlockW& bw = m->blocks[g];
+  const int L = m->L, D = m->D, d = m->d, rev = g & 1, n_steps = L - 1;
+  const int ethreads = d < 256 ? d : 256;
+  cudaStream_t user = m->stream;
+  CU_OK(cudaMemsetAsync(m->step_ctr, 0, sizeof(int), user));
+  m->cur_rows = B;
+  LAUNCH(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, B, ethreads, D * sizeof(float), m->o, v, u, labels, bw.w_in_t,
+         bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 1, m->step_ctr, 0, n_steps);
+  TF_TRY(check_launch("seq_update_embed_kernel"));
+  if (m->prof_on || !m->use_graphs) {  // direct launches (per-kernel events need them)
+    for (int t = 0; t < n_steps; ++t) {
+      TF_TRY(seq_enqueue_steps(m, g, B, labels, v, u, 1));
+      LAUNCH(m, KC_CTRL, seq::seq_advance_kernel, 1, 32, 0, m->step_ctr, 1);
+    }
+    return check_launch("sequential block");
+  }
+  auto key = std::make_pair(g, B);
+  auto it = m->seq_graphs.find(key);
+  if (it == m->seq_graphs.end()) {
+    tf_model::SeqGraph sg;
+    sg.unroll = seq_unroll(n_steps);
+    const int64_t before = m->launches;
+    cudaGraph_t graph = nullptr;
+    m->stream = m->cap_stream;
+    cudaError_t e = cudaStreamBeginCapture(m->cap_stream, cudaStreamCaptureModeThreadLocal);
+    int r = TF_OK;
+    if (e == cudaSuccess) {
+      r = seq_enqueue_steps(m, g, B, labels, v, u, sg.unroll);
+      LAUNCH(m, KC_CTRL, seq::seq_advance_kernel, 1, 32, 0, m->step_ctr, sg.unroll);
+      e = cudaStreamEndCapture(m->cap_stream, &graph);
+    }
+    m->stream = user;
+    sg.nodes = (int)(m->launches - before);
+    m->launches = before;
+    if (e != cudaSuccess || r != TF_OK || !graph) {
+      if (graph) cudaGraphDestroy(graph);
+      cudaGetLastError();
+      return r != TF_OK ? r : fail(TF_ECUDA, "capturing the sequential-step graph failed: %s", cudaGetErrorString(e));
+    }
+    e = cudaGraphInstantiate(&sg.exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) return fail(TF_ECUDA, "cudaGraphInstantiate: %s", cudaGetErrorString(e));
+    it = m->seq_graphs.emplace(key, sg).first;
+  }
+  const tf_model::SeqGraph& sg = it->second;
+  const int replays = (n_steps + sg.unroll - 1) / sg.unroll;  // steps past n_steps return at once
+  for (int i = 0; i < replays; ++i) CU_OK(cudaGraphLaunch(sg.exec, user));
+  m->launches += (int64_t)replays * sg.nodes;
+  return TF_OK;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -440,13 +578,18 @@ static int inverse_impl(tf_model* m, const float* z, const int* labels, int B, c
   const int K = m->cfg.n_blocks;
   float *v = m->seq_a, *u = m->seq_b;
   m->trace.clear();
+  if (labels) {  // model-owned copy: captured graphs keep a fixed address
+    CU_OK(cudaMemcpyAsync(m->labels_own, labels, B * sizeof(int), cudaMemcpyDeviceToDevice, m->stream));
+    labels = m->labels_own;
+  }
   TF_TRY(layout(m, const_cast<float*>(z), v, B, 1));
   int status = TF_OK;
   for (int g = 0; g < K; ++g) {
     int* iters_row = m->iters_sample + (size_t)g * m->cfg.max_batch;
     int sweeps = m->L - 1;
     if (policy[g] == 0) {
-      TF_TRY(run_sequential_block<T>(m, g, B, labels, v, u));
+      if constexpr (sizeof(T) == 2) TF_TRY(run_sequential_block_bf16(m, g, B, labels, v, u));
+      else TF_TRY(run_sequential_block<T>(m, g, B, labels, v, u));
       LAUNCH(m, KC_CTRL, fill_int_kernel, (B + 127) / 128, 128, 0, iters_row, B, m->L - 1);
     } else {
       int r = run_jacobi_block<T>(m, g, B, labels, v, u, tau, max_iters, init_mode, &sweeps, iters_row);
@@ -623,6 +766,9 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
   TF_TRY(dev_alloc(m, &m->io_z, B * c.C * c.H * c.W));
   TF_TRY(dev_alloc(m, &m->io_x, B * c.C * c.H * c.W));
   TF_TRY(dev_alloc(m, &m->io_labels, B));
+  TF_TRY(dev_alloc(m, &m->labels_own, B));
+  TF_TRY(dev_alloc(m, &m->step_ctr, 1));
+  CU_OK(cudaMemset(m->step_ctr, 0, sizeof(int)));
   CU_OK(cudaMemset(m->ctrl, 0, 8 * sizeof(int)));
   CU_OK(cudaMemset(m->err, 0, sizeof(int)));
   CU_OK(cudaMemset(m->iters_sample, 0, (size_t)c.n_blocks * B * sizeof(int)));
@@ -638,6 +784,11 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
                                attn::smem_bytes<true>()));
     CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                attn::smem_bytes<false>()));
+    TF_TRY((seq_gemm_configure<true, seq::EpiQKV>()));
+    TF_TRY((seq_gemm_configure<true, seq::EpiGelu>()));
+    TF_TRY((seq_gemm_configure<true, seq::EpiHead>()));
+    TF_TRY((seq_gemm_configure<false, seq::EpiResidual>()));
+    CU_OK(cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking));
   }
   CU_OK(cudaDeviceSynchronize());
   return TF_OK;
@@ -693,6 +844,8 @@ void tf_free(tf_model* m) {
   cudaDeviceSynchronize();
   m->prof_collect();
   for (cudaEvent_t e : m->ev_pool) cudaEventDestroy(e);
+  for (auto& kv : m->seq_graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+  if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
   for (void* p : m->allocs) cudaFree(p);
   if (m->ctrl_host) cudaFreeHost(m->ctrl_host);
   delete m;
@@ -810,18 +963,19 @@ int tf_profile_enable(tf_model* m, int32_t on) {
   if (!m) return fail(TF_EINVAL, "model is NULL");
   cudaDeviceSynchronize();
   m->prof_collect();
-  for (int c = 0; c < KC_COUNT; ++c) { m->prof_ms[c] = 0; m->prof_n[c] = 0; }
+  for (int c = 0; c < KC_COUNT; ++c) { m->prof_ms[c] = 0; m->prof_n[c] = 0; m->prof_rows[c] = 0; }
   m->prof_on = on != 0;
   return TF_OK;
 }
 
-int tf_profile_read(tf_model* m, const char** names, double* ms, int64_t* launches, int32_t cap) {
+int tf_profile_read(tf_model* m, const char** names, double* ms, int64_t* launches, double* rows, int32_t cap) {
   if (!m) return fail(TF_EINVAL, "model is NULL");
   m->prof_collect();
   for (int c = 0; c < KC_COUNT && c < cap; ++c) {
     if (names) names[c] = kKernelClassNames[c];
     if (ms) ms[c] = m->prof_ms[c];
     if (launches) launches[c] = m->prof_n[c];
+    if (rows) rows[c] = m->prof_rows[c];
   }
   return KC_COUNT;
 }
