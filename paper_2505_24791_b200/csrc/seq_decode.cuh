@@ -1,44 +1,49 @@
 // Sequential decoding with a key/value cache on the bf16 engine (Eq. 5; the sequential baseline and
 // block 0 of the selective policy, Sec. 3.5).  One decoding step pushes ONE token per sample through
 // the block's transformer, so every projection is a skinny GEMM  out[B, N] = A[B, K] W[N, K]^T  with
-// B <= a few hundred rows: the cost is streaming W (from L2 or HBM) and launch latency, not FLOPs.
-//
-//   seq_gemm_kernel     one CTA per slice of NC output columns.  The activation rows (after an optional
-//                       fused LayerNorm) are staged once in shared memory as bf16; each warp streams
-//                       its 8 rows of W straight from global memory into registers with 16-byte loads
-//                       (nothing of W is shared between warps, so it never touches shared memory) and
-//                       multiplies with mma.sync m16n8k16; the K range is split over the warps of the
-//                       CTA and reduced in shared memory in a fixed order (deterministic).
-//   seq_attention_kernel one CTA per (sample, head): single query against cache rows 0..t.
+// B <= a few hundred rows: the cost is streaming W (from L2 or HBM) and the latency of a chain of
+// small dependent kernels, not FLOPs.  The chain per layer is
+//   resid_ln -> gemm(QKV, cache append) -> attention -> gemm(out, partials)
+//   resid_ln -> gemm(MLP up, GELU)      -> gemm(MLP down, partials)
+// where
+//   seq_gemm_kernel      one CTA per (slice of NC output columns, slice of K).  The activation slice is
+//                        staged once in shared memory with asynchronous copies; each warp streams its
+//                        8 rows of W straight from global memory into registers with 16-byte loads
+//                        (nothing of W is shared between warps, so it never touches shared memory) and
+//                        multiplies with mma.sync m16n8k16; the warps of a CTA split its K slice and
+//                        reduce in shared memory in a fixed order.  Projections that feed the residual
+//                        stream are split along K over several CTAs and write fp32 partial tiles;
+//   seq_resid_ln_kernel  h += sum of those partial tiles + bias (fixed order: deterministic), then the
+//                        LayerNorm of the next projection's input, written as bf16;
+//   seq_attention_kernel one CTA per (sample, head): single query against cache rows 0..t;
 //   seq_update_embed_kernel  affine update of token t+1 (Eq. 5) and its embedding for the next step.
-// The step index is read from device memory (*step_base + step_off), so one captured CUDA graph of
-// a few steps can be replayed for the whole block.
+// Consecutive kernels are chained with programmatic dependent launch, and the step index is read from
+// device memory (*step_base + step_off), so one captured CUDA graph of a few steps can be replayed
+// for the whole block.
 #pragma once
 #include "common.cuh"
 
 namespace seq {
 
 constexpr int ROWS = 64;           // activation rows per CTA pass (4 m16 tiles)
-constexpr int KC = 1024;           // K chunk staged in shared memory at a time
-constexpr int A_PITCH = KC + 8;    // bf16 elements; +16 bytes per row keeps ldmatrix conflict-free
+constexpr int KC = 1024;           // largest K slice staged in shared memory
 constexpr int THREADS = 256;
 constexpr int WARPS = THREADS / 32;
 constexpr int HD = 64;             // head_dim of the bf16 engine
 
-__host__ __device__ constexpr int a_smem_bytes() { return ROWS * A_PITCH * 2; }
-__host__ __device__ constexpr int red_smem_bytes() { return WARPS * ROWS * 8 * 4; }
-__host__ __device__ constexpr int stat_smem_bytes() { return ROWS * 2 * 4; }
-__host__ __device__ constexpr int gemm_smem_bytes() { return a_smem_bytes() + red_smem_bytes() + stat_smem_bytes(); }
+// staged activation slice (row pitch klen + 8 bf16: the 16 extra bytes keep ldmatrix conflict-free)
+// + one [64, 8] fp32 tile per warp for the in-CTA reduction
+__host__ __device__ constexpr int gemm_smem_bytes(int klen) { return ROWS * (klen + 8) * 2 + WARPS * ROWS * 8 * 4; }
 
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const bf16* p) {
   uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+  asm("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
 }
 __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ uint4 ld_stream16(const void* p) {  // weights: read once per step, keep out of L1
   uint4 v;
@@ -46,84 +51,50 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p) {  // weights: read 
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
 }
-
-// Position inside a staged row of the element with (chunk-local) reduction index k.  A lane's 16-byte
-// weight load covers 8 consecutive k; the two m16n8k16 steps of a 32-wide k group then take the
-// lane's elements {0,1 | 2,3} and {4,5 | 6,7} as their B fragments.  The activation row is stored
-// so that a plain ldmatrix of step (32c + 16j) delivers the matching elements:
-//   k = 32c + 8t + 4j + 2h + e   ->   32c + 16j + 8h + 2t + e.
-__device__ __forceinline__ int perm_k(int k) {
-  const int c = k & ~31, r = k & 31;
-  const int t = r >> 3, j = (r >> 2) & 1, h = (r >> 1) & 1, e = r & 1;
-  return c + 16 * j + 8 * h + 2 * t + e;
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+  const uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
 }
 
-// LayerNorm of RF rows at a time by one warp, rows held in registers (NV float4 per lane, K <= 128*NV):
-// one round of global loads per RF rows, two-pass statistics from registers (eps 1e-5), result written
-// as bf16 in the permuted order.  Rows >= nrows are written as zeros.
-template <int RF, int NV>
-__device__ __forceinline__ void ln_stage_rows(const float* __restrict__ h, const float* __restrict__ gamma,
-                                              const float* __restrict__ beta, bf16* __restrict__ sA, int K, int row0,
-                                              int nrows, int srows, int pitch) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nv4 = K >> 2;
-  for (int rb = warp * RF; rb < srows; rb += WARPS * RF) {
-    float4 v[RF][NV];
+// Programmatic dependent launch: a kernel lets its successor in the stream start early (its CTAs are
+// scheduled, fetch weights, and then block in pdl_wait) and itself waits for its predecessor's
+// results only where it first needs them.  Every kernel of the chain calls pdl_wait before it ends,
+// so "kernel k finished" always implies "kernels < k finished".
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// B fragments from 16-byte weight loads.  Lane (g, t) of a warp loads W[n0 + g][k0 + 8t .. k0 + 8t + 7],
+// i.e. the four lanes of a quad hold the four 16-byte chunks of one 32-wide k group of row g, as pairs
+// in[0..3].  The m16n8k16 B fragment of k step s (s = 0, 1) wants, in lane t, the pairs
+// (k = 16s + 2t, +1) and (k = 16s + 8 + 2t, +1): pair t of chunk 2s and pair t of chunk 2s + 1.
+// A 4x4 transpose across the quad delivers out[c] = pair t of chunk c with three shuffles.
+__device__ __forceinline__ uint32_t pick4(const uint32_t (&v)[4], int i) {
+  return i == 0 ? v[0] : i == 1 ? v[1] : i == 2 ? v[2] : v[3];
+}
+__device__ __forceinline__ void quad_transpose(const uint4& w, int lane, uint32_t (&out)[4]) {
+  const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+  const int t = lane & 3;
+  uint32_t got[4];
+  got[0] = pick4(in, t);  // round 0: own chunk
 #pragma unroll
-    for (int rr = 0; rr < RF; ++rr) {
-      const bool rok = (rb + rr) < nrows;
-      const float4* xr = reinterpret_cast<const float4*>(h + (size_t)(row0 + rb + rr) * K);
+  for (int r = 1; r < 4; ++r)  // round r: lane t reads lane (t + r) & 3, which offers its pair (own index - r) & 3
+    got[r] = __shfl_sync(0xffffffffu, pick4(in, (t - r) & 3), (lane & ~3) | ((t + r) & 3));
+  // got[r] is pair t of chunk (t + r) & 3
 #pragma unroll
-      for (int i = 0; i < NV; ++i) {
-        const int idx = i * 32 + lane;
-        v[rr][i] = (rok && idx < nv4) ? __ldcg(xr + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-    }
-#pragma unroll
-    for (int rr = 0; rr < RF; ++rr) {
-      if (rb + rr >= srows) break;
-      float s = 0.f;
-#pragma unroll
-      for (int i = 0; i < NV; ++i) s += (v[rr][i].x + v[rr][i].y) + (v[rr][i].z + v[rr][i].w);
-      const float mean = warp_sum(s) / K;
-      float sq = 0.f;
-#pragma unroll
-      for (int i = 0; i < NV; ++i) {
-        if (i * 32 + lane < nv4) {
-          const float a = v[rr][i].x - mean, b = v[rr][i].y - mean, c = v[rr][i].z - mean, e = v[rr][i].w - mean;
-          sq += (a * a + b * b) + (c * c + e * e);
-        }
-      }
-      const float rstd = rsqrtf(warp_sum(sq) / K + 1e-5f);
-      const bool rok = (rb + rr) < nrows;
-      bf16* dst = sA + (rb + rr) * pitch;
-#pragma unroll
-      for (int i = 0; i < NV; ++i) {
-        const int idx = i * 32 + lane;
-        if (idx < nv4) {
-          float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (rok) {
-            const float4 gg = *reinterpret_cast<const float4*>(gamma + 4 * idx);
-            const float4 bb = *reinterpret_cast<const float4*>(beta + 4 * idx);
-            o.x = (v[rr][i].x - mean) * rstd * gg.x + bb.x; o.y = (v[rr][i].y - mean) * rstd * gg.y + bb.y;
-            o.z = (v[rr][i].z - mean) * rstd * gg.z + bb.z; o.w = (v[rr][i].w - mean) * rstd * gg.w + bb.w;
-          }
-          *reinterpret_cast<__nv_bfloat162*>(dst + perm_k(4 * idx)) = __floats2bfloat162_rn(o.x, o.y);
-          *reinterpret_cast<__nv_bfloat162*>(dst + perm_k(4 * idx + 2)) = __floats2bfloat162_rn(o.z, o.w);
-        }
-      }
-    }
-  }
+  for (int c = 0; c < 4; ++c) out[c] = pick4(got, (c - t) & 3);
 }
 
 // ---------------------------------------------------------------------------------------------
-// epilogues: apply(row b, column n, value) for one finished output element (bias not yet added)
+// epilogues: apply(row b, column n, value, step t, k-slice index) for one finished output element
 // ---------------------------------------------------------------------------------------------
 struct EpiQKV {  // q -> q[b, :]; k, v -> cache row t of (b, head): cache layout [B][heads][L][64]
   bf16 *q, *kc, *vc;
   const float* bias;
   int d, L, heads;
-  __device__ __forceinline__ void apply(int b, int n, float x, int t) const {
+  __device__ __forceinline__ void apply(int b, int n, float x, int t, int) const {
     const bf16 val = __float2bfloat16_rn(x + bias[n]);
     if (n < d) { q[(size_t)b * d + n] = val; return; }
     const int nn = n < 2 * d ? n - d : n - 2 * d;
@@ -131,20 +102,18 @@ struct EpiQKV {  // q -> q[b, :]; k, v -> cache row t of (b, head): cache layout
     cache[(((size_t)b * heads + (nn >> 6)) * L + t) * HD + (nn & 63)] = val;
   }
 };
-struct EpiResidual {  // h[b, n] += x + bias[n]
-  float* h;
-  const float* bias;
-  int ldh;
-  __device__ __forceinline__ void apply(int b, int n, float x, int) const {
-    float* p = h + (size_t)b * ldh + n;
-    *p = *p + (x + bias[n]);
+struct EpiPartial {  // part[ks][b][n] = x : summed (with the bias) by seq_resid_ln_kernel
+  float* part;
+  int B, N;
+  __device__ __forceinline__ void apply(int b, int n, float x, int, int ks) const {
+    part[((size_t)ks * B + b) * N + n] = x;
   }
 };
 struct EpiGelu {  // out[b, n] = bf16(gelu(x + bias[n]))
   bf16* out;
   const float* bias;
   int ld;
-  __device__ __forceinline__ void apply(int b, int n, float x, int) const {
+  __device__ __forceinline__ void apply(int b, int n, float x, int, int) const {
     out[(size_t)b * ld + n] = __float2bfloat16_rn(gelu_erf(x + bias[n]));
   }
 };
@@ -152,146 +121,84 @@ struct EpiHead {  // o[b, n] = x + bias[n]  (fp32, interleaved mu~ / alpha~ colu
   float* o;
   const float* bias;
   int ld;
-  __device__ __forceinline__ void apply(int b, int n, float x, int) const { o[(size_t)b * ld + n] = x + bias[n]; }
+  __device__ __forceinline__ void apply(int b, int n, float x, int, int) const { o[(size_t)b * ld + n] = x + bias[n]; }
 };
 
 // ---------------------------------------------------------------------------------------------
-// out[B, N] = LN?(A)[B, K] * W[N, K]^T.   grid = (ceil(N / NC), ceil(B / 64)),  NC in {8, 16, 32}.
-//   LN = true : A is the fp32 residual stream h [B, K] (K = width), normalised with gamma/beta.
-//   LN = false: A is a bf16 matrix [B, K].
-// Warp w owns the 8-column tile (w % (NC/8)) and the k-split (w / (NC/8)) of every staged K chunk.
+// out[B, N] (or a partial of it) = A[B, k-slice] * W[N, k-slice]^T,  A bf16 [B, K] row-major.
+//   grid = (ceil(N / NC), K / klen, ceil(B / 64)),  NC in {8, 16, 32, 64},  klen % (32 * 64 / NC) == 0.
+// Warp w owns the 8-column tile (w % (NC/8)) and the part (w / (NC/8)) of the CTA's K slice.
 // ---------------------------------------------------------------------------------------------
-template <int NC, bool LN, class Epi>
-__global__ void __launch_bounds__(THREADS, 1)
-seq_gemm_kernel(const void* __restrict__ A_, const float* __restrict__ gamma, const float* __restrict__ beta,
-                const bf16* __restrict__ W, int B, int N, int K, Epi epi, const int* __restrict__ step_base,
-                int step_off, int n_steps) {
-  const int t = *step_base + step_off;
-  if (t >= n_steps) return;
+template <int NC, class Epi>
+__global__ void __launch_bounds__(THREADS)
+seq_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W, int B, int N, int K, int klen, Epi epi,
+                const int* __restrict__ step_base, int step_off, int n_steps, int check_steps) {
+  pdl_launch_dependents();
   extern __shared__ __align__(128) uint8_t smem_seq[];
+  const int pitch = klen + 8;
   bf16* sA = reinterpret_cast<bf16*>(smem_seq);
-  float* sRed = reinterpret_cast<float*>(smem_seq + a_smem_bytes());
-  float* sStat = reinterpret_cast<float*>(smem_seq + a_smem_bytes() + red_smem_bytes());
+  float* sRed = reinterpret_cast<float*>(smem_seq + ROWS * pitch * 2);
   constexpr int NT = NC / 8;       // 8-column tiles per CTA
-  constexpr int KS = WARPS / NT;   // k-splits
+  constexpr int KS = WARPS / NT;   // warps splitting the CTA's K slice
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, tq = lane & 3;
   const int nt = warp % NT, ks = warp / NT;
   const int n0 = blockIdx.x * NC + nt * 8;
-  const int row0 = blockIdx.y * ROWS;
+  const int kbase = blockIdx.y * klen;
+  const int row0 = blockIdx.z * ROWS;
   const int nrows = (B - row0) < ROWS ? (B - row0) : ROWS;
   const int mtiles = (nrows + 15) >> 4;  // m16 tiles that hold real rows
   const int srows = mtiles * 16;         // rows staged in shared memory (rows past B are zero)
+  const int kper = klen / KS, ngroups = kper >> 5;  // 32-wide k groups of this warp
 
-  const bool ln_fast = LN && K <= KC;  // whole rows fit the register-resident LayerNorm staging
-  if (LN && !ln_fast) {  // general path: row statistics first (two-pass, eps 1e-5), one warp per row
-    const float* h = reinterpret_cast<const float*>(A_);
-    for (int r = warp; r < srows; r += WARPS) {
-      float mean = 0.f, rstd = 0.f;
-      if (r < nrows) {
-        const float4* xr = reinterpret_cast<const float4*>(h + (size_t)(row0 + r) * K);
-        float s = 0.f;
-        for (int i = lane; i < (K >> 2); i += 32) { float4 v = xr[i]; s += (v.x + v.y) + (v.z + v.w); }
-        mean = warp_sum(s) / K;
-        float sq = 0.f;
-        for (int i = lane; i < (K >> 2); i += 32) {
-          float4 v = xr[i];
-          float a = v.x - mean, b2 = v.y - mean, c = v.z - mean, e = v.w - mean;
-          sq += (a * a + b2 * b2) + (c * c + e * e);
-        }
-        rstd = rsqrtf(warp_sum(sq) / K + 1e-5f);
-      }
-      if (lane == 0) { sStat[2 * r] = mean; sStat[2 * r + 1] = rstd; }
-    }
-    __syncthreads();
+  // weights are constants: the first batch is requested before waiting for the previous kernel
+  const int wrow = (n0 + g) < N ? (n0 + g) : (N - 1);  // columns past N are computed but never stored
+  const bf16* wp = W + (size_t)wrow * K + kbase + ks * kper + 8 * tq;
+  uint4 wreg[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+    if (i < ngroups) wreg[i] = ld_stream16(wp + i * 32);
+
+  pdl_wait();  // activations and the step counter are complete from here on
+  const int t = *step_base + step_off;  // only the epilogue needs it, unless steps past the end can occur
+  if (check_steps && t >= n_steps) return;
+
+  // stage A[row0 .. row0+63][kbase .. kbase+klen) row-major with asynchronous 16-byte copies (one L2 round
+  // trip for the whole slice, no registers held); rows past B inside the last m16 tile are zero
+  const int per_row = klen >> 3, total = srows * per_row;
+  for (int i = threadIdx.x; i < total; i += THREADS) {
+    const int r = i / per_row, k8 = (i - r * per_row) << 3;
+    if (r < nrows) cp_async16(sA + r * pitch + k8, A + (size_t)(row0 + r) * K + kbase + k8);
+    else *reinterpret_cast<uint4*>(sA + r * pitch + k8) = make_uint4(0u, 0u, 0u, 0u);
   }
+  cp_async_wait_all();
+  __syncthreads();
 
   float acc[4][4];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-
-  const int wrow = (n0 + g) < N ? (n0 + g) : (N - 1);  // clamp: columns past N are computed but never stored
-  const bf16* wbase = W + (size_t)wrow * K;
-
-  for (int k0 = 0; k0 < K; k0 += KC) {
-    const int kc = (K - k0) < KC ? (K - k0) : KC;  // multiple of 32
-    const int kper = kc / KS;                       // k range of one warp in this chunk (multiple of 32 by host check)
-    uint4 wreg[8];
-    const int ngroups = kper >> 5;
-    const bf16* wp = wbase + k0 + ks * kper + 8 * tq;
-    // stage A[row0 .. row0+63][k0 .. k0+kc) as bf16 with the k permutation, zero rows past B
-    if (k0 > 0) __syncthreads();  // previous chunk fully consumed
-    if (ln_fast) {
-      const float* h = reinterpret_cast<const float*>(A_);
-      if (K <= 512) ln_stage_rows<4, 4>(h, gamma, beta, sA, K, row0, nrows, srows, A_PITCH);
-      else ln_stage_rows<2, 8>(h, gamma, beta, sA, K, row0, nrows, srows, A_PITCH);
-    } else if constexpr (LN) {
-      const float* h = reinterpret_cast<const float*>(A_);
-      for (int i = threadIdx.x; i < srows * (kc >> 2); i += THREADS) {
-        const int r = i / (kc >> 2), k4 = (i - r * (kc >> 2)) << 2;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (r < nrows) {
-          v = *reinterpret_cast<const float4*>(h + (size_t)(row0 + r) * K + k0 + k4);
-          const float mean = sStat[2 * r], rstd = sStat[2 * r + 1];
-          const float4 gg = *reinterpret_cast<const float4*>(gamma + k0 + k4);
-          const float4 bb = *reinterpret_cast<const float4*>(beta + k0 + k4);
-          v.x = (v.x - mean) * rstd * gg.x + bb.x; v.y = (v.y - mean) * rstd * gg.y + bb.y;
-          v.z = (v.z - mean) * rstd * gg.z + bb.z; v.w = (v.w - mean) * rstd * gg.w + bb.w;
-        }
-        // k4 % 4 == 0: elements (k4, k4+1) and (k4+2, k4+3) are the two adjacent pairs h = 0, 1
-        bf16* dst = sA + r * A_PITCH;
-        *reinterpret_cast<__nv_bfloat162*>(dst + perm_k(k4)) = __floats2bfloat162_rn(v.x, v.y);
-        *reinterpret_cast<__nv_bfloat162*>(dst + perm_k(k4 + 2)) = __floats2bfloat162_rn(v.z, v.w);
-      }
-    } else {
-      const bf16* a = reinterpret_cast<const bf16*>(A_);
-      const int per_row = kc >> 3, total = srows * per_row;
-      for (int i0 = threadIdx.x; i0 < total; i0 += 8 * THREADS) {  // 8 loads in flight per thread
-        uint4 v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int i = i0 + u * THREADS;
-          const int r = i / per_row, k8 = (i - r * per_row) << 3;
-          v[u] = (i < total && r < nrows) ? __ldcg(reinterpret_cast<const uint4*>(a + (size_t)(row0 + r) * K + k0 + k8))
-                                          : make_uint4(0u, 0u, 0u, 0u);
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int i = i0 + u * THREADS;
-          if (i < total) {
-            const int r = i / per_row, k8 = (i - r * per_row) << 3;
-            // 8 consecutive k = one lane's load (t = (k8 >> 3) & 3): pairs go to j*16 + h*8 + 2t
-            bf16* dst = sA + r * A_PITCH + (k8 & ~31) + 2 * ((k8 >> 3) & 3);
-            *reinterpret_cast<uint32_t*>(dst) = v[u].x;
-            *reinterpret_cast<uint32_t*>(dst + 8) = v[u].y;
-            *reinterpret_cast<uint32_t*>(dst + 16) = v[u].z;
-            *reinterpret_cast<uint32_t*>(dst + 24) = v[u].w;
-          }
-        }
-      }
-    }
-    __syncthreads();
-    // stream the warp's weights in batches of up to 8 outstanding 16-byte loads per lane
-    for (int g0 = 0; g0 < ngroups; g0 += 8) {
-      const int nb = (ngroups - g0) < 8 ? (ngroups - g0) : 8;
+  const bf16* a_lane = sA + ((lane & 7) + ((lane >> 3) & 1) * 8) * pitch + ks * kper + (lane >> 4) * 8;
+  for (int g0 = 0; g0 < ngroups; g0 += 8) {
+    if (g0 > 0) {
 #pragma unroll
       for (int i = 0; i < 8; ++i)
-        if (i < nb) wreg[i] = ld_stream16(wp + (size_t)(g0 + i) * 32);
+        if (g0 + i < ngroups) wreg[i] = ld_stream16(wp + (g0 + i) * 32);
+    }
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        if (i < nb) {
-          const int kk = ks * kper + (g0 + i) * 32;  // chunk-local k of this 32-wide group
+    for (int i = 0; i < 8; ++i) {
+      if (g0 + i < ngroups) {
+        uint32_t bq[4];
+        quad_transpose(wreg[i], lane, bq);
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const uint32_t b0 = j == 0 ? wreg[i].x : wreg[i].z, b1 = j == 0 ? wreg[i].y : wreg[i].w;
+        for (int j = 0; j < 2; ++j) {
 #pragma unroll
-            for (int mt = 0; mt < 4; ++mt) {
-              if (mt >= mtiles) break;  // uniform across the CTA
+          for (int mt = 0; mt < 4; ++mt) {
+            if (mt < mtiles) {  // uniform across the CTA
               uint32_t af[4];
-              ldsm_x4(af, sA + (mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * A_PITCH + kk + 16 * j + (lane >> 4) * 8);
-              mma_bf16(acc[mt], af, b0, b1);
+              ldsm_x4(af, a_lane + mt * 16 * pitch + (g0 + i) * 32 + 16 * j);
+              mma_bf16(acc[mt], af, bq[2 * j], bq[2 * j + 1]);
             }
           }
         }
@@ -299,7 +206,7 @@ seq_gemm_kernel(const void* __restrict__ A_, const float* __restrict__ gamma, co
     }
   }
 
-  // k-split reduction in shared memory (fixed order), then the epilogue: thread -> (row, column)
+  // reduction over the CTA's warps in shared memory (fixed order), then the epilogue: thread -> (row, column)
   float* my = sRed + warp * (ROWS * 8);
 #pragma unroll
   for (int mt = 0; mt < 4; ++mt) {
@@ -307,15 +214,69 @@ seq_gemm_kernel(const void* __restrict__ A_, const float* __restrict__ gamma, co
     *reinterpret_cast<float2*>(my + (mt * 16 + g + 8) * 8 + 2 * tq) = make_float2(acc[mt][2], acc[mt][3]);
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < ROWS * NC; i += THREADS) {
+  for (int i = threadIdx.x; i < nrows * NC; i += THREADS) {
     const int r = i / NC, c = i - r * NC;
     const int tile = c >> 3, cc = c & 7;
     float s = 0.f;
 #pragma unroll
     for (int k = 0; k < KS; ++k) s += sRed[(k * NT + tile) * (ROWS * 8) + r * 8 + cc];
     const int n = blockIdx.x * NC + c;
-    if (r < nrows && n < N) epi.apply(row0 + r, n, s, t);
+    if (n < N) epi.apply(row0 + r, n, s, t, (int)blockIdx.y);
   }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Residual update and LayerNorm of one row per CTA (blockDim.x = d / 4, one float4 per thread):
+//   h[b, :] += bias + sum_{s < nsplit} part[s][b][:]      (skipped when nsplit == 0)
+//   xn[b, :] = bf16( LayerNorm(h[b, :]) * gamma + beta )   (two-pass statistics, eps 1e-5)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512)
+seq_resid_ln_kernel(float* __restrict__ h, const float* __restrict__ part, const float* __restrict__ bias, int nsplit,
+                    const float* __restrict__ gamma, const float* __restrict__ beta, bf16* __restrict__ xn, int B, int d,
+                    const int* __restrict__ step_base, int step_off, int n_steps, int check_steps) {
+  pdl_launch_dependents();
+  __shared__ float red[2][16];
+  const int b = blockIdx.x, i = threadIdx.x;  // i < d / 4
+  const float4 gg = reinterpret_cast<const float4*>(gamma)[i];
+  const float4 bb = reinterpret_cast<const float4*>(beta)[i];
+  float4 add = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (nsplit > 0) add = reinterpret_cast<const float4*>(bias)[i];
+  pdl_wait();
+  if (check_steps && *step_base + step_off >= n_steps) return;
+  float4 x = __ldcg(reinterpret_cast<const float4*>(h + (size_t)b * d) + i);
+  if (nsplit > 0) {
+    float4 p[8];
+    for (int s0 = 0; s0 < nsplit; s0 += 8) {
+#pragma unroll
+      for (int s = 0; s < 8; ++s)
+        if (s0 + s < nsplit) p[s] = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)(s0 + s) * B + b) * d) + i);
+#pragma unroll
+      for (int s = 0; s < 8; ++s)
+        if (s0 + s < nsplit) { add.x += p[s].x; add.y += p[s].y; add.z += p[s].z; add.w += p[s].w; }
+    }
+    x.x += add.x; x.y += add.y; x.z += add.z; x.w += add.w;
+    reinterpret_cast<float4*>(h + (size_t)b * d)[i] = x;
+  }
+  const int warp = i >> 5, lane = i & 31, nwarps = (blockDim.x + 31) >> 5;
+  float s = warp_sum((x.x + x.y) + (x.z + x.w));
+  if (lane == 0) red[0][warp] = s;
+  __syncthreads();
+  float tot = 0.f;
+  for (int w = 0; w < nwarps; ++w) tot += red[0][w];
+  const float mean = tot / d;
+  const float a0 = x.x - mean, a1 = x.y - mean, a2 = x.z - mean, a3 = x.w - mean;
+  float sq = warp_sum((a0 * a0 + a1 * a1) + (a2 * a2 + a3 * a3));
+  if (lane == 0) red[1][warp] = sq;
+  __syncthreads();
+  tot = 0.f;
+  for (int w = 0; w < nwarps; ++w) tot += red[1][w];
+  const float rstd = rsqrtf(tot / d + 1e-5f);
+  const __nv_bfloat162 o0 = __floats2bfloat162_rn(a0 * rstd * gg.x + bb.x, a1 * rstd * gg.y + bb.y);
+  const __nv_bfloat162 o1 = __floats2bfloat162_rn(a2 * rstd * gg.z + bb.z, a3 * rstd * gg.w + bb.w);
+  uint2 w2;
+  w2.x = *reinterpret_cast<const uint32_t*>(&o0);
+  w2.y = *reinterpret_cast<const uint32_t*>(&o1);
+  reinterpret_cast<uint2*>(xn + (size_t)b * d)[i] = w2;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -329,6 +290,8 @@ __global__ void __launch_bounds__(256)
 seq_attention_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc, const bf16* __restrict__ vc,
                      bf16* __restrict__ out, int L, int d, int heads, float scale_log2e,
                      const int* __restrict__ step_base, int step_off, int n_steps) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int t = *step_base + step_off;
   if (t >= n_steps) return;
   __shared__ float s_m[32], s_l[32], s_o[32][HD];
@@ -428,6 +391,8 @@ __global__ void seq_update_embed_kernel(const float* __restrict__ o, const float
                                         const float* __restrict__ cls, float* __restrict__ h, int L, int D, int d,
                                         int reversed, int first, const int* __restrict__ step_base, int step_off,
                                         int n_steps) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int t = *step_base + step_off;
   if (!first && t >= n_steps) return;
   extern __shared__ float s_tok[];
@@ -453,6 +418,7 @@ __global__ void seq_update_embed_kernel(const float* __restrict__ o, const float
 }
 
 __global__ void seq_advance_kernel(int* step_base, int by) {
+  pdl_wait();  // every kernel of the replayed steps has finished reading the counter
   if (threadIdx.x == 0 && blockIdx.x == 0) *step_base += by;
 }
 

@@ -133,6 +133,8 @@ struct tf_model {
   struct SeqGraph { cudaGraphExec_t exec = nullptr; int unroll = 0; int nodes = 0; };
   std::map<std::pair<int, int>, SeqGraph> seq_graphs;  // (block g, B)
   bool use_graphs = true;
+  int seq_check_steps = 0;    // 1 when a replayed graph can run past the last step (kernels then test the counter)
+  float* seq_part = nullptr;  // [<=16 K slices][max_batch][d] fp32 partial tiles of the residual projections
   float *io_z = nullptr, *io_x = nullptr;  // staging for the host-buffer entry point
   int* io_labels = nullptr;
   cudaStream_t stream = nullptr;
@@ -380,65 +382,114 @@ static int run_sequential_block(tf_model* m, int g, int B, const int* labels, co
 }
 
 // ---- bf16 engine: fused-LayerNorm skinny GEMMs on tensor cores, replayed from a CUDA graph -------
-template <bool LN, class Epi>
-static int seq_gemm(tf_model* m, int cls, const void* A, const float* gamma, const float* beta, const Matrix& W, int B,
-                    const Epi& epi, int step_off) {
-  const int N = W.N, K = W.K, n_steps = m->L - 1;
-  // k-splits per CTA need K % (32 * splits) == 0; prefer narrow column slices (more CTAs) while they fit
-  int nc = 32;
-  if (K % 256 == 0 && N / 8 <= 2 * m->num_sms) nc = 8;
-  else if (K % 128 == 0 && N / 16 <= 2 * m->num_sms) nc = 16;
-  dim3 grid((N + nc - 1) / nc, (B + seq::ROWS - 1) / seq::ROWS);
-  const bf16* w = reinterpret_cast<const bf16*>(W.w);
-  const int smem = seq::gemm_smem_bytes();
-  if (nc == 8)
-    LAUNCH(m, cls, (seq::seq_gemm_kernel<8, LN, Epi>), grid, seq::THREADS, smem, A, gamma, beta, w, B, N, K, epi,
-           m->step_ctr, step_off, n_steps);
-  else if (nc == 16)
-    LAUNCH(m, cls, (seq::seq_gemm_kernel<16, LN, Epi>), grid, seq::THREADS, smem, A, gamma, beta, w, B, N, K, epi,
-           m->step_ctr, step_off, n_steps);
-  else
-    LAUNCH(m, cls, (seq::seq_gemm_kernel<32, LN, Epi>), grid, seq::THREADS, smem, A, gamma, beta, w, B, N, K, epi,
-           m->step_ctr, step_off, n_steps);
+// Launch of a sequential-step kernel with programmatic dependent launch, so that consecutive kernels of
+// the chain overlap their launch latency and weight prefetch (see seq_decode.cuh).
+template <class... KArgs, class... Args>
+static int launch_seq(tf_model* m, int cls, void (*kern)(KArgs...), dim3 grid, int threads, int smem, Args... args) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = grid;
+  lc.blockDim = dim3(threads);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = m->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  m->pre(cls);
+  cudaError_t e = cudaLaunchKernelEx(&lc, kern, static_cast<KArgs>(args)...);
+  m->post(cls);
+  if (e != cudaSuccess) return fail(TF_ECUDA, "sequential-step kernel launch failed: %s", cudaGetErrorString(e));
   return TF_OK;
 }
 
-template <bool LN, class Epi>
+// One skinny GEMM of a decoding step.  `partial`: the projection feeds the residual stream, so it is split
+// along K over several CTAs that write fp32 partial tiles (the number of K slices is returned in *nsplit).
+template <class Epi>
+static int seq_gemm(tf_model* m, int cls, const bf16* A, const Matrix& W, int B, const Epi& epi, int step_off,
+                    bool partial, int* nsplit) {
+  const int N = W.N, K = W.K, n_steps = m->L - 1;
+  const bf16* w = reinterpret_cast<const bf16*>(W.w);
+  const int row_tiles = (B + seq::ROWS - 1) / seq::ROWS;
+  int klen = K;
+  if (partial && K % 256 == 0) {
+    klen = 256;
+    while (((N + 31) / 32) * (K / klen) > 2 * m->num_sms && klen * 2 <= seq::KC && K % (klen * 2) == 0) klen *= 2;
+  }
+  if (klen > seq::KC || (partial && K / klen > 16))
+    return fail(TF_EINVAL, "sequential decoding: reduction length %d not supported", K);
+  const int ksplit = K / klen;
+  if (nsplit) *nsplit = ksplit;
+  // column slices: as narrow as the K slice allows (klen % (32 * 64 / NC) == 0) while the grid stays <= 2 waves;
+  // measured on B200, more and smaller CTAs win although every CTA re-reads its activation slice from L2
+  int nc = 64;
+  if (klen % 256 == 0 && ((N + 7) / 8) * ksplit <= 2 * m->num_sms) nc = 8;
+  else if (klen % 128 == 0 && ((N + 15) / 16) * ksplit <= 2 * m->num_sms) nc = 16;
+  else if (klen % 64 == 0 && ((N + 31) / 32) * ksplit <= 2 * m->num_sms) nc = 32;
+  dim3 grid((N + nc - 1) / nc, ksplit, row_tiles);
+  const int smem = seq::gemm_smem_bytes(klen);
+#define TF_SEQ_GEMM_CASE(NCV)                                                                                     \
+  if (nc == NCV)                                                                                                  \
+    return launch_seq(m, cls, seq::seq_gemm_kernel<NCV, Epi>, grid, seq::THREADS, smem, A, w, B, N, K, klen, epi, \
+                      m->step_ctr, step_off, n_steps, m->seq_check_steps);
+  TF_SEQ_GEMM_CASE(8)
+  TF_SEQ_GEMM_CASE(16)
+  TF_SEQ_GEMM_CASE(32)
+  TF_SEQ_GEMM_CASE(64)
+#undef TF_SEQ_GEMM_CASE
+  return fail(TF_EINVAL, "no sequential GEMM variant for this shape");
+}
+
+template <class Epi>
 static int seq_gemm_configure() {
-  const int smem = seq::gemm_smem_bytes();
-  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<8, LN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<16, LN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<32, LN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  const int smem = seq::gemm_smem_bytes(seq::KC);
+  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<8, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<16, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<32, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<64, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
   return TF_OK;
+}
+
+static int seq_resid_ln(tf_model* m, const float* bias, int nsplit, const float* gamma, const float* beta, int B,
+                        int step_off) {
+  return launch_seq(m, KC_SEQ_LN, seq::seq_resid_ln_kernel, dim3(B), m->d / 4, 0, m->h, m->seq_part, bias, nsplit, gamma,
+                    beta, reinterpret_cast<bf16*>(m->xn), B, m->d, m->step_ctr, step_off, m->L - 1, m->seq_check_steps);
 }
 
 // kernels of decoding steps step_off .. step_off+count-1 relative to the device step counter
 static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const float* v, float* u, int count) {
   const BlockW& bw = m->blocks[g];
   const int L = m->L, D = m->D, d = m->d, rev = g & 1, nl = m->cfg.n_layers, heads = m->cfg.n_heads;
+  bf16* xn = reinterpret_cast<bf16*>(m->xn);
   bf16* q = reinterpret_cast<bf16*>(m->qkv);
   bf16* att = reinterpret_cast<bf16*>(m->att);
   bf16* mlp = reinterpret_cast<bf16*>(m->mlp);
   const size_t layer_stride = (size_t)m->cfg.max_batch * L * d;
   const float scale = 1.0f / sqrtf((float)m->hd);
   const int ethreads = d < 256 ? d : 256;
+  const seq::EpiPartial to_part{m->seq_part, B, d};
   m->cur_rows = B;
   for (int s = 0; s < count; ++s) {
+    const float* pending_bias = nullptr;  // bias of the projection whose partial tiles are not yet in h
+    int pending = 0;
     for (int i = 0; i < nl; ++i) {
       const LayerW& lw = bw.layers[i];
       bf16* kc = reinterpret_cast<bf16*>(m->kcache) + i * layer_stride;
       bf16* vc = reinterpret_cast<bf16*>(m->vcache) + i * layer_stride;
-      TF_TRY((seq_gemm<true>(m, KC_SEQ_GEMM, m->h, lw.ln1_g, lw.ln1_b, lw.w_qkv, B,
-                             seq::EpiQKV{q, kc, vc, lw.b_qkv, d, L, heads}, s)));
-      LAUNCH(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, q, kc, vc, att, L, d, heads,
-             scale * 1.4426950408889634f, m->step_ctr, s, L - 1);
-      TF_TRY((seq_gemm<false>(m, KC_SEQ_GEMM, att, nullptr, nullptr, lw.w_o, B, seq::EpiResidual{m->h, lw.b_o, d}, s)));
-      TF_TRY((seq_gemm<true>(m, KC_SEQ_GEMM, m->h, lw.ln2_g, lw.ln2_b, lw.w_1, B, seq::EpiGelu{mlp, lw.b_1, m->hid}, s)));
-      TF_TRY((seq_gemm<false>(m, KC_SEQ_GEMM, mlp, nullptr, nullptr, lw.w_2, B, seq::EpiResidual{m->h, lw.b_2, d}, s)));
+      TF_TRY(seq_resid_ln(m, pending_bias, pending, lw.ln1_g, lw.ln1_b, B, s));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, lw.w_qkv, B, seq::EpiQKV{q, kc, vc, lw.b_qkv, d, L, heads}, s, false, nullptr));
+      TF_TRY(launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, q, kc, vc, att, L, d, heads,
+                        scale * 1.4426950408889634f, m->step_ctr, s, L - 1));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, att, lw.w_o, B, to_part, s, true, &pending));
+      TF_TRY(seq_resid_ln(m, lw.b_o, pending, lw.ln2_g, lw.ln2_b, B, s));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, lw.w_1, B, seq::EpiGelu{mlp, lw.b_1, m->hid}, s, false, nullptr));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, mlp, lw.w_2, B, to_part, s, true, &pending));
+      pending_bias = lw.b_2;
     }
-    TF_TRY((seq_gemm<true>(m, KC_SEQ_GEMM, m->h, bw.lnf_g, bw.lnf_b, bw.w_out, B, seq::EpiHead{m->o, bw.b_out, 2 * D}, s)));
-    LAUNCH(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, B, ethreads, D * sizeof(float), m->o, v, u, labels, bw.w_in_t,
-           bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 0, m->step_ctr, s, L - 1);
+    TF_TRY(seq_resid_ln(m, pending_bias, pending, bw.lnf_g, bw.lnf_b, B, s));
+    TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, bw.w_out, B, seq::EpiHead{m->o, bw.b_out, 2 * D}, s, false, nullptr));
+    TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B), ethreads, (int)(D * sizeof(float)), m->o, v, u,
+                      labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 0, m->step_ctr, s, L - 1));
   }
   return check_launch("sequential step kernels");
 }
@@ -455,15 +506,15 @@ static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* label
   const int L = m->L, D = m->D, d = m->d, rev = g & 1, n_steps = L - 1;
   const int ethreads = d < 256 ? d : 256;
   cudaStream_t user = m->stream;
+  m->seq_check_steps = (m->prof_on || !m->use_graphs) ? 0 : (n_steps % seq_unroll(n_steps) != 0);
   CU_OK(cudaMemsetAsync(m->step_ctr, 0, sizeof(int), user));
   m->cur_rows = B;
-  LAUNCH(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, B, ethreads, D * sizeof(float), m->o, v, u, labels, bw.w_in_t,
-         bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 1, m->step_ctr, 0, n_steps);
-  TF_TRY(check_launch("seq_update_embed_kernel"));
+  TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B), ethreads, (int)(D * sizeof(float)), m->o, v, u,
+                    labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 1, m->step_ctr, 0, n_steps));
   if (m->prof_on || !m->use_graphs) {  // direct launches (per-kernel events need them)
     for (int t = 0; t < n_steps; ++t) {
       TF_TRY(seq_enqueue_steps(m, g, B, labels, v, u, 1));
-      LAUNCH(m, KC_CTRL, seq::seq_advance_kernel, 1, 32, 0, m->step_ctr, 1);
+      TF_TRY(launch_seq(m, KC_CTRL, seq::seq_advance_kernel, dim3(1), 32, 0, m->step_ctr, 1));
     }
     return check_launch("sequential block");
   }
@@ -479,7 +530,7 @@ static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* label
     int r = TF_OK;
     if (e == cudaSuccess) {
       r = seq_enqueue_steps(m, g, B, labels, v, u, sg.unroll);
-      LAUNCH(m, KC_CTRL, seq::seq_advance_kernel, 1, 32, 0, m->step_ctr, sg.unroll);
+      if (r == TF_OK) r = launch_seq(m, KC_CTRL, seq::seq_advance_kernel, dim3(1), 32, 0, m->step_ctr, sg.unroll);
       e = cudaStreamEndCapture(m->cap_stream, &graph);
     }
     m->stream = user;
@@ -768,6 +819,7 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
   TF_TRY(dev_alloc(m, &m->io_labels, B));
   TF_TRY(dev_alloc(m, &m->labels_own, B));
   TF_TRY(dev_alloc(m, &m->step_ctr, 1));
+  if (c.dtype == 1) TF_TRY(dev_alloc(m, &m->seq_part, (size_t)16 * B * d));
   CU_OK(cudaMemset(m->step_ctr, 0, sizeof(int)));
   CU_OK(cudaMemset(m->ctrl, 0, 8 * sizeof(int)));
   CU_OK(cudaMemset(m->err, 0, sizeof(int)));
@@ -784,10 +836,10 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
                                attn::smem_bytes<true>()));
     CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                attn::smem_bytes<false>()));
-    TF_TRY((seq_gemm_configure<true, seq::EpiQKV>()));
-    TF_TRY((seq_gemm_configure<true, seq::EpiGelu>()));
-    TF_TRY((seq_gemm_configure<true, seq::EpiHead>()));
-    TF_TRY((seq_gemm_configure<false, seq::EpiResidual>()));
+    TF_TRY(seq_gemm_configure<seq::EpiQKV>());
+    TF_TRY(seq_gemm_configure<seq::EpiGelu>());
+    TF_TRY(seq_gemm_configure<seq::EpiHead>());
+    TF_TRY(seq_gemm_configure<seq::EpiPartial>());
     CU_OK(cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking));
   }
   CU_OK(cudaDeviceSynchronize());
@@ -821,6 +873,7 @@ int tf_load(const tf_config* cfg, const void* weights_host, size_t nbytes, tf_mo
   if (c.dtype == 1 && (c.width % 64 || c.width / c.n_heads != 64))
     return fail(TF_EINVAL, "bf16 engine needs width %% 64 == 0 and head_dim == 64");
   if (c.width > 2048) return fail(TF_EINVAL, "width > 2048 not supported");
+  if (c.dtype == 1 && c.width > 1024) return fail(TF_EINVAL, "bf16 engine: width > 1024 not supported");
   tf_model* m = new (std::nothrow) tf_model();
   if (!m) return fail(TF_ENOMEM, "host allocation failed");
   m->cfg = c;
