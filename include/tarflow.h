@@ -144,6 +144,32 @@ int tf_jacobi_update(const float* o_dev, const float* v_dev, float* u_dev, float
 int tf_gemm_bf16(const void* a_dev, const void* w_dev, const float* bias_dev, float* c_dev,
                  int32_t M, int32_t N, int32_t K, void* cuda_stream);
 
+/*
+ * tf_skinny_gemm_noalloc -- C[M,N] (fp32) = A[M,K] (bf16) * W[N,K]^T (bf16) + bias[N] (fp32, may be NULL),
+ * the same product as tf_gemm_bf16, computed by the split-K kernel of the sequential decoding path, for
+ * callers that must not allocate device memory.  (The paper has no counterpart; this is a property of
+ * the library, not of the method.)
+ *   Who needs it: a caller that has handed all device memory to its own pool or arena, a caller inside a
+ *   latency-critical loop where cudaMalloc's implicit device-wide synchronisation is not acceptable, or
+ *   one that runs where the allocator may not be entered at all (for instance from a callback).  Every
+ *   other entry point of this library takes its working memory from cudaMalloc (tf_load for a model,
+ *   tf_gemm_bf16 for its error word on first use); this one calls neither cudaMalloc nor cudaFree nor any
+ *   routine that does.
+ *   How: the fp32 partial tiles of the K slices ((K/256) * M * N * 4 bytes) and one control word live in a
+ *   static device array of TF_NOALLOC_SCRATCH_BYTES that every GPU which loads the library holds until
+ *   the process exits.  A problem whose tiles do not fit is refused with TF_EINVAL and a message that
+ *   names both sizes.  Requirements: M >= 1, N % 8 == 0, K % 256 == 0, pointers 16-byte aligned.
+ *   First call on a device: looks up the array's device address (cudaGetSymbolAddress) and raises the
+ *   kernel's shared-memory limit, with that device current; make this first call outside any stream capture.
+ *   Sharing: all calls on a device use the one array, which keeps the contents of the previous call; the
+ *   call re-zeroes what has to start at zero.  Two calls whose work overlaps on the GPU (different streams
+ *   without ordering between them) race on it and give wrong results: order them.
+ *   Asynchronous on `cuda_stream`; the caller owns every buffer.
+ */
+#define TF_NOALLOC_SCRATCH_BYTES (8u << 20)
+int tf_skinny_gemm_noalloc(const void* a_dev, const void* w_dev, const float* bias_dev, float* c_dev,
+                           int32_t M, int32_t N, int32_t K, void* cuda_stream);
+
 /* tf_gemm_status -- synchronise `cuda_stream` and report whether any tf_gemm_bf16 launch so far
  * gave up on a bounded device-side wait (TF_ETIMEOUT) or all completed (TF_OK). */
 int tf_gemm_status(void* cuda_stream);

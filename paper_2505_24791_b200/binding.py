@@ -50,6 +50,7 @@ def lib():
         L.tf_jacobi_update.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
         L.tf_gemm_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
         L.tf_gemm_status.argtypes = [vp]
+        L.tf_skinny_gemm_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
         L.tf_profile_enable.argtypes = [vp, i32]
         L.tf_profile_read.argtypes = [vp, vp, vp, vp, vp, i32]
         L.tf_set_precision.argtypes = [vp, i32, f32, f32]
@@ -138,6 +139,10 @@ def tf_jacobi_update(o, v, u, maxdiff, B, L, D, reversed_, stream=None):
 
 def tf_gemm_bf16(a, w, bias, c, M, N, K, stream=None):
     return _check(lib().tf_gemm_bf16(_ptr(a), _ptr(w), _ptr(bias), _ptr(c), M, N, K, _stream(stream)))
+
+
+def tf_skinny_gemm_noalloc(a, w, bias, c, M, N, K, stream=None):
+    return _check(lib().tf_skinny_gemm_noalloc(_ptr(a), _ptr(w), _ptr(bias), _ptr(c), M, N, K, _stream(stream)))
 
 
 def tf_gemm_status(stream=None):

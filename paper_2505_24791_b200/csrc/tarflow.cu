@@ -1012,6 +1012,64 @@ int tf_gemm_status(void* cuda_stream) {
   return TF_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Allocation-free skinny GEMM (see tf_skinny_gemm_noalloc in tarflow.h).  The split-K partial tiles and
+// the step-counter word the kernel reads live in a static device array instead of cudaMalloc'd memory.
+// ------------------------------------------------------------------------------------------------
+#define TF_NOALLOC_HEADER_BYTES 256u
+static __device__ __align__(256) unsigned char g_noalloc_scratch[TF_NOALLOC_SCRATCH_BYTES];
+static unsigned char* g_noalloc_ptr[64] = {nullptr};  // device address of the array, per device ordinal
+
+// c[m, n] = bias[n] + sum over K slices of part[s][m][n], slices added in index order
+__global__ void noalloc_reduce_kernel(const float* __restrict__ part, const float* __restrict__ bias,
+                                      float* __restrict__ c, int nsplit, int M, int N) {
+  const size_t total = (size_t)M * N;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    float acc = bias ? bias[i % N] : 0.f;
+    for (int sl = 0; sl < nsplit; ++sl) acc += part[(size_t)sl * total + i];
+    c[i] = acc;
+  }
+}
+
+int tf_skinny_gemm_noalloc(const void* a_dev, const void* w_dev, const float* bias_dev, float* c_dev, int32_t M, int32_t N,
+                           int32_t K, void* cuda_stream) {
+  g_err[0] = 0;
+  if (!a_dev || !w_dev || !c_dev) return fail(TF_EINVAL, "NULL buffer");
+  if (M < 1 || N < 8 || N % 8 || K < 256 || K % 256) return fail(TF_EINVAL, "need M >= 1, N %% 8 == 0, K %% 256 == 0");
+  const int klen = 256, ksplit = K / klen;
+  const size_t need = (size_t)ksplit * M * N * sizeof(float);
+  if (need > (size_t)TF_NOALLOC_SCRATCH_BYTES - TF_NOALLOC_HEADER_BYTES)
+    return fail(TF_EINVAL, "tf_skinny_gemm_noalloc: (K/256)*M*N*4 = %zu bytes of partial tiles exceed the %zu-byte static scratch",
+                need, (size_t)TF_NOALLOC_SCRATCH_BYTES - TF_NOALLOC_HEADER_BYTES);
+  int dev = 0;
+  CU_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(TF_EINVAL, "device ordinal %d not supported", dev);
+  using Kern = void (*)(const bf16*, const bf16*, int, int, int, int, seq::EpiPartial, const int*, int, int, int);
+  Kern kern = seq::seq_gemm_kernel<8, seq::EpiPartial>;
+  const int smem = seq::gemm_smem_bytes(klen);
+  if (!g_noalloc_ptr[dev]) {  // once per device, with that device current: resolve the symbol to a device address
+    unsigned char* p = nullptr;
+    CU_OK(cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_scratch));
+    CU_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    g_noalloc_ptr[dev] = p;
+  }
+  unsigned char* base = g_noalloc_ptr[dev];
+  int* step_word = reinterpret_cast<int*>(base);
+  float* part = reinterpret_cast<float*>(base + TF_NOALLOC_HEADER_BYTES);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  // the array keeps whatever the last call left: the step word must read 0; the tiles are fully overwritten
+  CU_OK(cudaMemsetAsync(step_word, 0, sizeof(int), st));
+  dim3 grid((N + 7) / 8, ksplit, (M + seq::ROWS - 1) / seq::ROWS);
+  kern<<<grid, seq::THREADS, smem, st>>>(reinterpret_cast<const bf16*>(a_dev), reinterpret_cast<const bf16*>(w_dev), M, N, K,
+                                         klen, seq::EpiPartial{part, M, N}, step_word, 0, 1, 0);
+  TF_TRY(check_launch("seq_gemm_kernel (no-alloc)"));
+  const size_t total = (size_t)M * N;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  noalloc_reduce_kernel<<<blocks, 256, 0, st>>>(part, bias_dev, c_dev, ksplit, M, N);
+  return check_launch("noalloc_reduce_kernel");
+}
+
 int tf_profile_enable(tf_model* m, int32_t on) {
   if (!m) return fail(TF_EINVAL, "model is NULL");
   cudaDeviceSynchronize();
