@@ -6,6 +6,9 @@
 //     columns of ONE row and every global access of a warp is a contiguous row segment.
 //     col_const is evaluated once per chunk (the bias of the lane's column), store once per row.
 //     All 32 lanes call store together (it may shuffle); lanes with col >= N pass col_ok = false.
+//   * kRowwise functors (bf16 outputs) skip the transpose: rowwise(row, col0, v, nv, sbias) gets the 32
+//     accumulator columns of the lane's own row and the chunk's bias in shared memory, and writes the
+//     row segment with 16-byte stores (64 contiguous bytes per lane: whole sectors).
 #pragma once
 #include "common.cuh"
 
@@ -18,6 +21,25 @@ struct EpiStore {
   const float* bias;  // may be null
   int ldc;
   OutT* out_lo = nullptr;
+  static constexpr bool kRowwise = sizeof(OutT) == 2;
+  // sbias: the 32 biases of columns col0.. (zeros without a bias), warp-private shared memory
+  __device__ __forceinline__ void rowwise(int row, int col0, float (&v)[32], int nv, const float* sbias) const {
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {
+      const float4 b = *reinterpret_cast<const float4*>(sbias + j);
+      v[j] += b.x; v[j + 1] += b.y; v[j + 2] += b.z; v[j + 3] += b.w;
+    }
+    if (GELU) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = gelu_erf_fast(v[j]);
+    }
+    store_bf16<32>(out + (size_t)row * ldc + col0, v, nv);
+    if (out_lo != nullptr) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] -= __bfloat162float(__float2bfloat16_rn(v[j]));
+      store_bf16<32>(out_lo + (size_t)row * ldc + col0, v, nv);
+    }
+  }
   template <int NC>
   __device__ __forceinline__ void apply(int row, int col0, const float (&v)[NC], int nv) const {
     OutT* p = out + (size_t)row * ldc + col0;
@@ -98,6 +120,7 @@ struct EpiResid {  // h[row, col] += acc + bias[col]   (fp32 residual stream, in
   float* h;
   const float* bias;
   int ldc;
+  static constexpr bool kRowwise = false;
   __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
   __device__ __forceinline__ void store(int row, int col, float acc, float cc, bool col_ok, int) const {
     if (col_ok) {
@@ -173,6 +196,7 @@ struct EpiHeadUpdate {
   const int* idx;      // [n_slots] slot -> sample (null = identity)
   const float* bias;   // [2D] interleaved
   int L, D, reversed;
+  static constexpr bool kRowwise = false;
   __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
   // lane-per-column form: even lanes hold mu~_c, the next lane alpha~_c
   __device__ __forceinline__ void store(int row, int col, float acc, float cc, bool col_ok, int lane) const {

@@ -267,25 +267,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (col0 >= N) break;  // uniform across the warp
         float v[32];
         tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c * 32), v);
-        // transpose through shared memory: lane = row on the way in, lane = column on the way out
-#pragma unroll
-        for (int j = 0; j < 32; ++j) stage_out[lane * 33 + j] = v[j];
-        __syncwarp();
         const int col = col0 + lane;
         const bool col_ok = col < N;
         const float cc = epi.col_const(col, col_ok);
-        if (nrows == 32) {
-#pragma unroll
-          for (int r0 = 0; r0 < 32; r0 += 8) {
-            float a[8];
-#pragma unroll
-            for (int r = 0; r < 8; ++r) a[r] = stage_out[(r0 + r) * 33 + lane];
-            epi.template store_rows<8>(row0 + r0, col, a, cc, col_ok, lane);
-          }
+        if constexpr (Epi::kRowwise) {
+          // lane = row: the chunk's biases go through the warp's shared-memory slot (broadcast reads)
+          stage_out[lane] = cc;
+          __syncwarp();
+          const int nv = (N - col0) < 32 ? (N - col0) : 32;
+          if (lane < nrows) epi.rowwise(row0 + lane, col0, v, nv, stage_out);
+          __syncwarp();
         } else {
-          for (int r = 0; r < nrows; ++r) epi.store(row0 + r, col, stage_out[r * 33 + lane], cc, col_ok, lane);
+          // transpose through shared memory: lane = row on the way in, lane = column on the way out
+#pragma unroll
+          for (int j = 0; j < 32; ++j) stage_out[lane * 33 + j] = v[j];
+          __syncwarp();
+          if (nrows == 32) {
+#pragma unroll
+            for (int r0 = 0; r0 < 32; r0 += 8) {
+              float a[8];
+#pragma unroll
+              for (int r = 0; r < 8; ++r) a[r] = stage_out[(r0 + r) * 33 + lane];
+              epi.template store_rows<8>(row0 + r0, col, a, cc, col_ok, lane);
+            }
+          } else {
+            for (int r = 0; r < nrows; ++r) epi.store(row0 + r, col, stage_out[r * 33 + lane], cc, col_ok, lane);
+          }
+          __syncwarp();
         }
-        __syncwarp();
       }
       tcgen05_fence_before();
       __syncwarp();
