@@ -2,21 +2,25 @@
 // block 0 of the selective policy, Sec. 3.5).  One decoding step pushes ONE token per sample through
 // the block's transformer, so every projection is a skinny GEMM  out[B, N] = A[B, K] W[N, K]^T  with
 // B <= a few hundred rows: the cost is streaming W (from L2 or HBM) and the latency of a chain of
-// small dependent kernels, not FLOPs.  The chain per layer is
-//   resid_ln -> gemm(QKV, cache append) -> attention -> gemm(out, partials)
-//   resid_ln -> gemm(MLP up, GELU)      -> gemm(MLP down, partials)
-// where
-//   seq_gemm_kernel      one CTA per (slice of NC output columns, slice of K).  The activation slice is
-//                        staged once in shared memory with asynchronous copies; each warp streams its
-//                        8 rows of W straight from global memory into registers with 16-byte loads
-//                        (nothing of W is shared between warps, so it never touches shared memory) and
-//                        multiplies with mma.sync m16n8k16; the warps of a CTA split its K slice and
-//                        reduce in shared memory in a fixed order.  Projections that feed the residual
-//                        stream are split along K over several CTAs and write fp32 partial tiles;
-//   seq_resid_ln_kernel  h += sum of those partial tiles + bias (fixed order: deterministic), then the
-//                        LayerNorm of the next projection's input, written as bf16;
-//   seq_attention_kernel one CTA per (sample, head): single query against cache rows 0..t;
-//   seq_update_embed_kernel  affine update of token t+1 (Eq. 5) and its embedding for the next step.
+// small dependent kernels, not FLOPs.  Every projection is split along N and K over the grid and writes
+// fp32 partial tiles; the (cheap, per-sample) consumer that follows sums them in a fixed order, so the
+// result does not depend on scheduling.  The chain per layer is
+//   resid_ln -> gemm(QKV) -> attention (sums q, k, v; appends the cache) -> gemm(out)
+//   resid_ln -> gemm(MLP up) -> bias_gelu -> gemm(MLP down)
+// and per step  ... -> resid_ln -> gemm(head) -> update_embed,  where
+//   seq_gemm_kernel      one CTA per (64 output columns, 256-wide slice of K): it multiplies a [64, klen]
+//                        activation slice with a [klen, 64] weight slice, so it reads as many activation
+//                        bytes as weight bytes.  The activation slice is staged in shared memory with
+//                        asynchronous copies; each warp streams its 8 rows of W straight from global
+//                        memory into registers with 16-byte loads (nothing of W is shared between warps,
+//                        so it never touches shared memory) and multiplies with mma.sync m16n8k16;
+//   seq_resid_ln_kernel  h += sum of partial tiles + bias, then the LayerNorm of the next projection's
+//                        input, written as bf16;
+//   seq_attention_kernel one CTA per (sample, head): sums the partial q, k, v of the new token, appends k, v
+//                        to the cache and attends over cache rows 0..t;
+//   seq_bias_gelu_kernel GELU(sum of partial tiles + bias) as bf16;
+//   seq_update_embed_kernel  affine update of token t+1 (Eq. 5) from the head's partial tiles and its
+//                        embedding for the next step.
 // Consecutive kernels are chained with programmatic dependent launch, and the step index is read from
 // device memory (*step_base + step_off), so one captured CUDA graph of a few steps can be replayed
 // for the whole block.
@@ -88,51 +92,15 @@ __device__ __forceinline__ void quad_transpose(const uint4& w, int lane, uint32_
 }
 
 // ---------------------------------------------------------------------------------------------
-// epilogues: apply(row b, column n, value, step t, k-slice index) for one finished output element
-// ---------------------------------------------------------------------------------------------
-struct EpiQKV {  // q -> q[b, :]; k, v -> cache row t of (b, head): cache layout [B][heads][L][64]
-  bf16 *q, *kc, *vc;
-  const float* bias;
-  int d, L, heads;
-  __device__ __forceinline__ void apply(int b, int n, float x, int t, int) const {
-    const bf16 val = __float2bfloat16_rn(x + bias[n]);
-    if (n < d) { q[(size_t)b * d + n] = val; return; }
-    const int nn = n < 2 * d ? n - d : n - 2 * d;
-    bf16* cache = n < 2 * d ? kc : vc;
-    cache[(((size_t)b * heads + (nn >> 6)) * L + t) * HD + (nn & 63)] = val;
-  }
-};
-struct EpiPartial {  // part[ks][b][n] = x : summed (with the bias) by seq_resid_ln_kernel
-  float* part;
-  int B, N;
-  __device__ __forceinline__ void apply(int b, int n, float x, int, int ks) const {
-    part[((size_t)ks * B + b) * N + n] = x;
-  }
-};
-struct EpiGelu {  // out[b, n] = bf16(gelu(x + bias[n]))
-  bf16* out;
-  const float* bias;
-  int ld;
-  __device__ __forceinline__ void apply(int b, int n, float x, int, int) const {
-    out[(size_t)b * ld + n] = __float2bfloat16_rn(gelu_erf(x + bias[n]));
-  }
-};
-struct EpiHead {  // o[b, n] = x + bias[n]  (fp32, interleaved mu~ / alpha~ columns)
-  float* o;
-  const float* bias;
-  int ld;
-  __device__ __forceinline__ void apply(int b, int n, float x, int, int) const { o[(size_t)b * ld + n] = x + bias[n]; }
-};
-
-// ---------------------------------------------------------------------------------------------
-// out[B, N] (or a partial of it) = A[B, k-slice] * W[N, k-slice]^T,  A bf16 [B, K] row-major.
+// part[ks][B, N] = A[B, k-slice ks] * W[N, k-slice ks]^T,  A bf16 [B, K] row-major, part fp32.
 //   grid = (ceil(N / NC), K / klen, ceil(B / 64)),  NC in {8, 16, 32, 64},  klen % (32 * 64 / NC) == 0.
 // Warp w owns the 8-column tile (w % (NC/8)) and the part (w / (NC/8)) of the CTA's K slice.
 // ---------------------------------------------------------------------------------------------
-template <int NC, class Epi>
+template <int NC>
 __global__ void __launch_bounds__(THREADS)
-seq_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W, int B, int N, int K, int klen, Epi epi,
-                const int* __restrict__ step_base, int step_off, int n_steps, int check_steps) {
+seq_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W, int B, int N, int K, int klen,
+                float* __restrict__ part, const int* __restrict__ step_base, int step_off, int n_steps,
+                int check_steps) {
   pdl_launch_dependents();
   extern __shared__ __align__(128) uint8_t smem_seq[];
   const int pitch = klen + 8;
@@ -160,8 +128,7 @@ seq_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W, int B, i
     if (i < ngroups) wreg[i] = ld_stream16(wp + i * 32);
 
   pdl_wait();  // activations and the step counter are complete from here on
-  const int t = *step_base + step_off;  // only the epilogue needs it, unless steps past the end can occur
-  if (check_steps && t >= n_steps) return;
+  if (check_steps && *step_base + step_off >= n_steps) return;
 
   // stage A[row0 .. row0+63][kbase .. kbase+klen) row-major with asynchronous 16-byte copies (one L2 round
   // trip for the whole slice, no registers held); rows past B inside the last m16 tile are zero
@@ -191,38 +158,89 @@ seq_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W, int B, i
       if (g0 + i < ngroups) {
         uint32_t bq[4];
         quad_transpose(wreg[i], lane, bq);
+        // all A fragments of the group first (independent loads), then the MMAs
+        uint32_t af[2][4][4];
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
+        for (int j = 0; j < 2; ++j)
 #pragma unroll
-          for (int mt = 0; mt < 4; ++mt) {
-            if (mt < mtiles) {  // uniform across the CTA
-              uint32_t af[4];
-              ldsm_x4(af, a_lane + mt * 16 * pitch + (g0 + i) * 32 + 16 * j);
-              mma_bf16(acc[mt], af, bq[2 * j], bq[2 * j + 1]);
-            }
-          }
-        }
+          for (int mt = 0; mt < 4; ++mt)
+            if (mt < mtiles) ldsm_x4(af[j][mt], a_lane + mt * 16 * pitch + (g0 + i) * 32 + 16 * j);
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+          for (int mt = 0; mt < 4; ++mt)
+            if (mt < mtiles) mma_bf16(acc[mt], af[j][mt], bq[2 * j], bq[2 * j + 1]);  // mtiles is uniform across the CTA
       }
     }
   }
 
-  // reduction over the CTA's warps in shared memory (fixed order), then the epilogue: thread -> (row, column)
-  float* my = sRed + warp * (ROWS * 8);
+  float* out = part + ((size_t)blockIdx.y * B + row0) * N;
+  if constexpr (KS == 1) {  // every warp holds finished columns: 8-byte stores straight from the fragments
+    const int n = n0 + 2 * tq;
+    if (n < N) {
 #pragma unroll
-  for (int mt = 0; mt < 4; ++mt) {
-    *reinterpret_cast<float2*>(my + (mt * 16 + g) * 8 + 2 * tq) = make_float2(acc[mt][0], acc[mt][1]);
-    *reinterpret_cast<float2*>(my + (mt * 16 + g + 8) * 8 + 2 * tq) = make_float2(acc[mt][2], acc[mt][3]);
-  }
-  __syncthreads();
-  for (int i = threadIdx.x; i < nrows * NC; i += THREADS) {
-    const int r = i / NC, c = i - r * NC;
-    const int tile = c >> 3, cc = c & 7;
-    float s = 0.f;
+      for (int mt = 0; mt < 4; ++mt) {
+        const int r = mt * 16 + g;
+        if (r < nrows) *reinterpret_cast<float2*>(out + (size_t)r * N + n) = make_float2(acc[mt][0], acc[mt][1]);
+        if (r + 8 < nrows) *reinterpret_cast<float2*>(out + (size_t)(r + 8) * N + n) = make_float2(acc[mt][2], acc[mt][3]);
+      }
+    }
+  } else {  // reduction over the CTA's warps in shared memory (fixed order): thread -> (row, column)
+    float* my = sRed + warp * (ROWS * 8);
 #pragma unroll
-    for (int k = 0; k < KS; ++k) s += sRed[(k * NT + tile) * (ROWS * 8) + r * 8 + cc];
-    const int n = blockIdx.x * NC + c;
-    if (n < N) epi.apply(row0 + r, n, s, t, (int)blockIdx.y);
+    for (int mt = 0; mt < 4; ++mt) {
+      *reinterpret_cast<float2*>(my + (mt * 16 + g) * 8 + 2 * tq) = make_float2(acc[mt][0], acc[mt][1]);
+      *reinterpret_cast<float2*>(my + (mt * 16 + g + 8) * 8 + 2 * tq) = make_float2(acc[mt][2], acc[mt][3]);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < nrows * NC; i += THREADS) {
+      const int r = i / NC, c = i - r * NC;
+      const int tile = c >> 3, cc = c & 7;
+      float sum = 0.f;
+#pragma unroll
+      for (int k = 0; k < KS; ++k) sum += sRed[(k * NT + tile) * (ROWS * 8) + r * 8 + cc];
+      const int n = blockIdx.x * NC + c;
+      if (n < N) out[(size_t)r * N + n] = sum;
+    }
   }
+}
+
+// Fixed-order sum of the K-slice partials of 4 consecutive outputs of row b, plus their bias.
+__device__ __forceinline__ float4 sum_partials4(const float* __restrict__ part, const float* __restrict__ bias, int nsplit,
+                                                int B, int N, int b, int n4) {
+  float4 acc = *reinterpret_cast<const float4*>(bias + 4 * n4);
+  float4 p[8];
+  for (int s0 = 0; s0 < nsplit; s0 += 8) {
+#pragma unroll
+    for (int sl = 0; sl < 8; ++sl)
+      if (s0 + sl < nsplit) p[sl] = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)(s0 + sl) * B + b) * N) + n4);
+#pragma unroll
+    for (int sl = 0; sl < 8; ++sl)
+      if (s0 + sl < nsplit) { acc.x += p[sl].x; acc.y += p[sl].y; acc.z += p[sl].z; acc.w += p[sl].w; }
+  }
+  return acc;
+}
+
+// ---------------------------------------------------------------------------------------------
+// out[b, n] = bf16(GELU(bias[n] + sum of partials)) for the MLP hidden layer.  One thread per 4 outputs.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+seq_bias_gelu_kernel(const float* __restrict__ part, int nsplit, const float* __restrict__ bias, bf16* __restrict__ out,
+                     int B, int N, const int* __restrict__ step_base, int step_off, int n_steps, int check_steps) {
+  pdl_launch_dependents();
+  pdl_wait();
+  if (check_steps && *step_base + step_off >= n_steps) return;
+  const int n4s = N >> 2;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B * n4s) return;
+  const int b = i / n4s, n4 = i - b * n4s;
+  const float4 x = sum_partials4(part, bias, nsplit, B, N, b, n4);
+  const __nv_bfloat162 o0 = __floats2bfloat162_rn(gelu_erf(x.x), gelu_erf(x.y));
+  const __nv_bfloat162 o1 = __floats2bfloat162_rn(gelu_erf(x.z), gelu_erf(x.w));
+  uint2 w2;
+  w2.x = *reinterpret_cast<const uint32_t*>(&o0);
+  w2.y = *reinterpret_cast<const uint32_t*>(&o1);
+  reinterpret_cast<uint2*>(out + (size_t)b * N)[n4] = w2;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -239,21 +257,11 @@ seq_resid_ln_kernel(float* __restrict__ h, const float* __restrict__ part, const
   const int b = blockIdx.x, i = threadIdx.x;  // i < d / 4
   const float4 gg = reinterpret_cast<const float4*>(gamma)[i];
   const float4 bb = reinterpret_cast<const float4*>(beta)[i];
-  float4 add = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (nsplit > 0) add = reinterpret_cast<const float4*>(bias)[i];
   pdl_wait();
   if (check_steps && *step_base + step_off >= n_steps) return;
   float4 x = __ldcg(reinterpret_cast<const float4*>(h + (size_t)b * d) + i);
   if (nsplit > 0) {
-    float4 p[8];
-    for (int s0 = 0; s0 < nsplit; s0 += 8) {
-#pragma unroll
-      for (int s = 0; s < 8; ++s)
-        if (s0 + s < nsplit) p[s] = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)(s0 + s) * B + b) * d) + i);
-#pragma unroll
-      for (int s = 0; s < 8; ++s)
-        if (s0 + s < nsplit) { add.x += p[s].x; add.y += p[s].y; add.z += p[s].z; add.w += p[s].w; }
-    }
+    const float4 add = sum_partials4(part, bias, nsplit, B, d, b, i);
     x.x += add.x; x.y += add.y; x.z += add.z; x.w += add.w;
     reinterpret_cast<float4*>(h + (size_t)b * d)[i] = x;
   }
@@ -280,37 +288,50 @@ seq_resid_ln_kernel(float* __restrict__ h, const float* __restrict__ part, const
 }
 
 // ---------------------------------------------------------------------------------------------
-// Single-query attention over cache rows 0..t of one (sample, head).  Cache layout [B][heads][L][64]
-// bf16, so the rows of one (sample, head) are contiguous.  8 lanes share a key (16 bytes = 8 channels
-// each); the 32 lane groups of the CTA take keys j = group (mod 32), four keys per round with the K
-// and V rows of all four in flight together, and keep an online softmax (running max, sum, output)
-// per group in fp32; the groups are merged through shared memory at the end.  q, out: [B, d].
+// Attention of the new token of one (sample, head).  The CTA first finishes that token's q, k, v (64
+// channels each) from the QKV projection's partial tiles (+ bias), appends k and v to the cache
+// (layout [B][heads][L][64] bf16: the rows of one (sample, head) are contiguous) and keeps q in fp32.
+// Then a single query against rows 0..t: 8 lanes share a key (16 bytes = 8 channels each); the 32 lane
+// groups of the CTA take keys j = group (mod 32), four keys per round with the K and V rows of all four in
+// flight together, and keep an online softmax (running max, sum, output) per group in fp32; the groups
+// are merged through shared memory at the end.  Row t itself is taken from shared memory.  out: [B, d].
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-seq_attention_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc, const bf16* __restrict__ vc,
-                     bf16* __restrict__ out, int L, int d, int heads, float scale_log2e,
+seq_attention_kernel(const float* __restrict__ part, int nsplit, const float* __restrict__ bias, bf16* __restrict__ kc,
+                     bf16* __restrict__ vc, bf16* __restrict__ out, int B, int L, int d, int heads, float scale_log2e,
                      const int* __restrict__ step_base, int step_off, int n_steps) {
   pdl_launch_dependents();
   pdl_wait();
   const int t = *step_base + step_off;
   if (t >= n_steps) return;
   __shared__ float s_m[32], s_l[32], s_o[32][HD];
+  __shared__ __align__(16) float s_q[HD];
+  __shared__ __align__(16) bf16 s_k[HD], s_v[HD];
   const int head = blockIdx.x, b = blockIdx.y;
   const int nk = t + 1;
   const int sub = threadIdx.x & 7, grp = threadIdx.x >> 3;
-  const bf16* kb = kc + ((size_t)b * heads + head) * L * HD + sub * 8;
-  const bf16* vb = vc + ((size_t)b * heads + head) * L * HD + sub * 8;
-  float qf[8];
-  {
-    const uint4 qv = *reinterpret_cast<const uint4*>(q + (size_t)b * d + head * HD + sub * 8);
-    const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float2 f = __bfloat1622float2(q2[i]);
-      qf[2 * i] = f.x * scale_log2e;  // scores in base-2 units: softmax via exp2
-      qf[2 * i + 1] = f.y * scale_log2e;
+  bf16* kb = kc + ((size_t)b * heads + head) * L * HD;
+  bf16* vb = vc + ((size_t)b * heads + head) * L * HD;
+  if (threadIdx.x < 48) {  // 3 x 64 channels, 4 per thread
+    const int which = threadIdx.x >> 4, c4 = threadIdx.x & 15;  // 0 = q, 1 = k, 2 = v
+    const float4 x = sum_partials4(part, bias, nsplit, B, 3 * d, b, (which * d + head * HD) / 4 + c4);
+    if (which == 0) {
+      *reinterpret_cast<float4*>(s_q + 4 * c4) = x;
+    } else {
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y), hi = __floats2bfloat162_rn(x.z, x.w);
+      uint2 w2;
+      w2.x = *reinterpret_cast<const uint32_t*>(&lo);
+      w2.y = *reinterpret_cast<const uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>((which == 1 ? s_k : s_v) + 4 * c4) = w2;
+      *reinterpret_cast<uint2*>((which == 1 ? kb : vb) + (size_t)t * HD + 4 * c4) = w2;
     }
   }
+  __syncthreads();
+  float qf[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) qf[i] = s_q[sub * 8 + i] * scale_log2e;  // scores in base-2 units: softmax via exp2
+  const bf16* kr = kb + sub * 8;
+  const bf16* vr = vb + sub * 8;
   float m_run = -INFINITY, l_run = 0.f, o[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) o[i] = 0.f;
@@ -319,9 +340,16 @@ seq_attention_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc, co
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int j = j0 + u * 32 + grp;
-      const bool ok = j < nk;
-      kv[u] = ok ? __ldcg(reinterpret_cast<const uint4*>(kb + (size_t)j * HD)) : make_uint4(0u, 0u, 0u, 0u);
-      vv[u] = ok ? __ldcg(reinterpret_cast<const uint4*>(vb + (size_t)j * HD)) : make_uint4(0u, 0u, 0u, 0u);
+      if (j < t) {
+        kv[u] = __ldcg(reinterpret_cast<const uint4*>(kr + (size_t)j * HD));
+        vv[u] = __ldcg(reinterpret_cast<const uint4*>(vr + (size_t)j * HD));
+      } else if (j == t) {  // the row this CTA has just produced
+        kv[u] = *reinterpret_cast<const uint4*>(s_k + sub * 8);
+        vv[u] = *reinterpret_cast<const uint4*>(s_v + sub * 8);
+      } else {
+        kv[u] = make_uint4(0u, 0u, 0u, 0u);
+        vv[u] = make_uint4(0u, 0u, 0u, 0u);
+      }
     }
     float sc[4];
 #pragma unroll
@@ -380,12 +408,14 @@ seq_attention_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc, co
 }
 
 // ---------------------------------------------------------------------------------------------
-// u[b, t+1, :] = v[b, t+1, :] * exp(alpha~) + mu~ from the head output o [B, 2D] (interleaved), then
+// u[b, t+1, :] = v[b, t+1, :] * exp(alpha~) + mu~ from the head projection's partial tiles [.][B, 2D]
+// (+ bias; columns interleaved mu~_c, alpha~_c), then
 // the embedding of that token for the next step: h[b, :] = u W_in^T + b_in + pos[t+1] (+ cls[y_b]).
 // One CTA per sample.  With first != 0 the step is the block's start: u[b, 0, :] = v[b, 0, :] (Eq. 5,
 // first row) and the embedding of token 0.
 // ---------------------------------------------------------------------------------------------
-__global__ void seq_update_embed_kernel(const float* __restrict__ o, const float* __restrict__ v, float* __restrict__ u,
+__global__ void seq_update_embed_kernel(const float* __restrict__ part, int nsplit, const float* __restrict__ bias,
+                                        int B, const float* __restrict__ v, float* __restrict__ u,
                                         const int* __restrict__ labels, const float* __restrict__ w_in_t,
                                         const float* __restrict__ b_in, const float* __restrict__ pos,
                                         const float* __restrict__ cls, float* __restrict__ h, int L, int D, int d,
@@ -401,7 +431,15 @@ __global__ void seq_update_embed_kernel(const float* __restrict__ o, const float
   const size_t e0 = ((size_t)b * L + tok_index(l_new, L, reversed)) * D;
   for (int c = threadIdx.x; c < D; c += blockDim.x) {
     float val = v[e0 + c];
-    if (!first) val = fmaf(val, expf(o[(size_t)b * 2 * D + 2 * c + 1]), o[(size_t)b * 2 * D + 2 * c]);
+    if (!first) {
+      float mu = bias[2 * c], al = bias[2 * c + 1];
+      for (int sl = 0; sl < nsplit; ++sl) {
+        const float2 p = __ldcg(reinterpret_cast<const float2*>(part + ((size_t)sl * B + b) * 2 * D) + c);
+        mu += p.x;
+        al += p.y;
+      }
+      val = fmaf(val, expf(al), mu);
+    }
     u[e0 + c] = val;
     s_tok[c] = val;
   }

@@ -10,6 +10,7 @@
 
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <string>
@@ -134,7 +135,8 @@ struct tf_model {
   std::map<std::pair<int, int>, SeqGraph> seq_graphs;  // (block g, B)
   bool use_graphs = true;
   int seq_check_steps = 0;    // 1 when a replayed graph can run past the last step (kernels then test the counter)
-  float* seq_part = nullptr;  // [<=16 K slices][max_batch][d] fp32 partial tiles of the residual projections
+  float* seq_part = nullptr;  // fp32 partial tiles [K slices][B][N] of the projection in flight
+  size_t seq_part_floats = 0;
   float *io_z = nullptr, *io_x = nullptr;  // staging for the host-buffer entry point
   int* io_labels = nullptr;
   cudaStream_t stream = nullptr;
@@ -403,34 +405,34 @@ static int launch_seq(tf_model* m, int cls, void (*kern)(KArgs...), dim3 grid, i
   return TF_OK;
 }
 
-// One skinny GEMM of a decoding step.  `partial`: the projection feeds the residual stream, so it is split
-// along K over several CTAs that write fp32 partial tiles (the number of K slices is returned in *nsplit).
-template <class Epi>
-static int seq_gemm(tf_model* m, int cls, const bf16* A, const Matrix& W, int B, const Epi& epi, int step_off,
-                    bool partial, int* nsplit) {
+// One skinny GEMM of a decoding step: part[ks][B, N] = A[B, K slice ks] W[N, K slice ks]^T.  Returns the number of
+// K slices in *nsplit; the kernel that consumes the tiles adds them up.  CTAs of 64 columns x 256 of K read as many
+// activation bytes as weight bytes and give a grid of (N / 64) * (K / 256) CTAs.
+static int seq_gemm(tf_model* m, int cls, const bf16* A, const Matrix& W, int B, int step_off, int* nsplit) {
   const int N = W.N, K = W.K, n_steps = m->L - 1;
   const bf16* w = reinterpret_cast<const bf16*>(W.w);
   const int row_tiles = (B + seq::ROWS - 1) / seq::ROWS;
-  int klen = K;
-  if (partial && K % 256 == 0) {
-    klen = 256;
-    while (((N + 31) / 32) * (K / klen) > 2 * m->num_sms && klen * 2 <= seq::KC && K % (klen * 2) == 0) klen *= 2;
-  }
-  if (klen > seq::KC || (partial && K / klen > 16))
-    return fail(TF_EINVAL, "sequential decoding: reduction length %d not supported", K);
+  int klen = (K % 256 == 0) ? 256 : K;
+  while (K / klen > 16 && K % (klen * 2) == 0) klen *= 2;  // at most 16 partial tiles
+  if (klen > seq::KC || K / klen > 16) return fail(TF_EINVAL, "sequential decoding: reduction length %d not supported", K);
   const int ksplit = K / klen;
-  if (nsplit) *nsplit = ksplit;
-  // column slices: as narrow as the K slice allows (klen % (32 * 64 / NC) == 0) while the grid stays <= 2 waves;
-  // measured on B200, more and smaller CTAs win although every CTA re-reads its activation slice from L2
+  *nsplit = ksplit;
+  if ((size_t)ksplit * B * N > m->seq_part_floats) return fail(TF_EINVAL, "sequential decoding: partial-tile buffer too small");
+  // column slices: the narrowest (most CTAs, shortest per-warp MMA chain) that keeps the grid within two waves; the
+  // warps of a CTA split its K slice, which needs klen % (32 * 64 / NC) == 0
   int nc = 64;
   if (klen % 256 == 0 && ((N + 7) / 8) * ksplit <= 2 * m->num_sms) nc = 8;
   else if (klen % 128 == 0 && ((N + 15) / 16) * ksplit <= 2 * m->num_sms) nc = 16;
   else if (klen % 64 == 0 && ((N + 31) / 32) * ksplit <= 2 * m->num_sms) nc = 32;
+  if (const char* e = getenv("TARFLOW_SEQ_NC")) {  // tuning aid: force the slice width where it is valid
+    const int f = atoi(e);
+    if ((f == 8 && klen % 256 == 0) || (f == 16 && klen % 128 == 0) || (f == 32 && klen % 64 == 0) || f == 64) nc = f;
+  }
   dim3 grid((N + nc - 1) / nc, ksplit, row_tiles);
   const int smem = seq::gemm_smem_bytes(klen);
-#define TF_SEQ_GEMM_CASE(NCV)                                                                                     \
-  if (nc == NCV)                                                                                                  \
-    return launch_seq(m, cls, seq::seq_gemm_kernel<NCV, Epi>, grid, seq::THREADS, smem, A, w, B, N, K, klen, epi, \
+#define TF_SEQ_GEMM_CASE(NCV)                                                                                            \
+  if (nc == NCV)                                                                                                         \
+    return launch_seq(m, cls, seq::seq_gemm_kernel<NCV>, grid, seq::THREADS, smem, A, w, B, N, K, klen, m->seq_part,     \
                       m->step_ctr, step_off, n_steps, m->seq_check_steps);
   TF_SEQ_GEMM_CASE(8)
   TF_SEQ_GEMM_CASE(16)
@@ -438,16 +440,6 @@ static int seq_gemm(tf_model* m, int cls, const bf16* A, const Matrix& W, int B,
   TF_SEQ_GEMM_CASE(64)
 #undef TF_SEQ_GEMM_CASE
   return fail(TF_EINVAL, "no sequential GEMM variant for this shape");
-}
-
-template <class Epi>
-static int seq_gemm_configure() {
-  const int smem = seq::gemm_smem_bytes(seq::KC);
-  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<8, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<16, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<32, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<64, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  return TF_OK;
 }
 
 static int seq_resid_ln(tf_model* m, const float* bias, int nsplit, const float* gamma, const float* beta, int B,
@@ -461,35 +453,36 @@ static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const
   const BlockW& bw = m->blocks[g];
   const int L = m->L, D = m->D, d = m->d, rev = g & 1, nl = m->cfg.n_layers, heads = m->cfg.n_heads;
   bf16* xn = reinterpret_cast<bf16*>(m->xn);
-  bf16* q = reinterpret_cast<bf16*>(m->qkv);
   bf16* att = reinterpret_cast<bf16*>(m->att);
   bf16* mlp = reinterpret_cast<bf16*>(m->mlp);
   const size_t layer_stride = (size_t)m->cfg.max_batch * L * d;
   const float scale = 1.0f / sqrtf((float)m->hd);
   const int ethreads = d < 256 ? d : 256;
-  const seq::EpiPartial to_part{m->seq_part, B, d};
   m->cur_rows = B;
   for (int s = 0; s < count; ++s) {
     const float* pending_bias = nullptr;  // bias of the projection whose partial tiles are not yet in h
-    int pending = 0;
+    int pending = 0, ns = 0;
     for (int i = 0; i < nl; ++i) {
       const LayerW& lw = bw.layers[i];
       bf16* kc = reinterpret_cast<bf16*>(m->kcache) + i * layer_stride;
       bf16* vc = reinterpret_cast<bf16*>(m->vcache) + i * layer_stride;
       TF_TRY(seq_resid_ln(m, pending_bias, pending, lw.ln1_g, lw.ln1_b, B, s));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, lw.w_qkv, B, seq::EpiQKV{q, kc, vc, lw.b_qkv, d, L, heads}, s, false, nullptr));
-      TF_TRY(launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, q, kc, vc, att, L, d, heads,
-                        scale * 1.4426950408889634f, m->step_ctr, s, L - 1));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, att, lw.w_o, B, to_part, s, true, &pending));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, lw.w_qkv, B, s, &ns));
+      TF_TRY(launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, m->seq_part, ns, lw.b_qkv, kc, vc,
+                        att, B, L, d, heads, scale * 1.4426950408889634f, m->step_ctr, s, L - 1));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, att, lw.w_o, B, s, &pending));
       TF_TRY(seq_resid_ln(m, lw.b_o, pending, lw.ln2_g, lw.ln2_b, B, s));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, lw.w_1, B, seq::EpiGelu{mlp, lw.b_1, m->hid}, s, false, nullptr));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, mlp, lw.w_2, B, to_part, s, true, &pending));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, lw.w_1, B, s, &ns));
+      TF_TRY(launch_seq(m, KC_SEQ_LN, seq::seq_bias_gelu_kernel, dim3((B * (m->hid / 4) + 255) / 256), 256, 0, m->seq_part, ns,
+                        lw.b_1, mlp, B, m->hid, m->step_ctr, s, L - 1, m->seq_check_steps));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, mlp, lw.w_2, B, s, &pending));
       pending_bias = lw.b_2;
     }
     TF_TRY(seq_resid_ln(m, pending_bias, pending, bw.lnf_g, bw.lnf_b, B, s));
-    TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, bw.w_out, B, seq::EpiHead{m->o, bw.b_out, 2 * D}, s, false, nullptr));
-    TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B), ethreads, (int)(D * sizeof(float)), m->o, v, u,
-                      labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 0, m->step_ctr, s, L - 1));
+    TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, bw.w_out, B, s, &ns));
+    TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B), ethreads, (int)(D * sizeof(float)), m->seq_part,
+                      ns, bw.b_out, B, v, u, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 0, m->step_ctr, s,
+                      L - 1));
   }
   return check_launch("sequential step kernels");
 }
@@ -509,8 +502,9 @@ static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* label
   m->seq_check_steps = (m->prof_on || !m->use_graphs) ? 0 : (n_steps % seq_unroll(n_steps) != 0);
   CU_OK(cudaMemsetAsync(m->step_ctr, 0, sizeof(int), user));
   m->cur_rows = B;
-  TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B), ethreads, (int)(D * sizeof(float)), m->o, v, u,
-                    labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 1, m->step_ctr, 0, n_steps));
+  TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B), ethreads, (int)(D * sizeof(float)), m->seq_part, 0,
+                    bw.b_out, B, v, u, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 1, m->step_ctr, 0,
+                    n_steps));
   if (m->prof_on || !m->use_graphs) {  // direct launches (per-kernel events need them)
     for (int t = 0; t < n_steps; ++t) {
       TF_TRY(seq_enqueue_steps(m, g, B, labels, v, u, 1));
@@ -819,7 +813,13 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
   TF_TRY(dev_alloc(m, &m->io_labels, B));
   TF_TRY(dev_alloc(m, &m->labels_own, B));
   TF_TRY(dev_alloc(m, &m->step_ctr, 1));
-  if (c.dtype == 1) TF_TRY(dev_alloc(m, &m->seq_part, (size_t)16 * B * d));
+  if (c.dtype == 1) {  // partial tiles: up to 16 K slices of a [B, d] output, or d/256 slices of the widest one
+    const size_t wide = (size_t)(hid > 3 * d ? hid : 3 * d);
+    m->seq_part_floats = (size_t)16 * B * d;
+    const size_t per_wide = (size_t)((d % 256 == 0) ? d / 256 : 1) * B * wide;
+    if (per_wide > m->seq_part_floats) m->seq_part_floats = per_wide;
+    TF_TRY(dev_alloc(m, &m->seq_part, m->seq_part_floats));
+  }
   CU_OK(cudaMemset(m->step_ctr, 0, sizeof(int)));
   CU_OK(cudaMemset(m->ctrl, 0, 8 * sizeof(int)));
   CU_OK(cudaMemset(m->err, 0, sizeof(int)));
@@ -836,10 +836,11 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
                                attn::smem_bytes<true>()));
     CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                attn::smem_bytes<false>()));
-    TF_TRY(seq_gemm_configure<seq::EpiQKV>());
-    TF_TRY(seq_gemm_configure<seq::EpiGelu>());
-    TF_TRY(seq_gemm_configure<seq::EpiHead>());
-    TF_TRY(seq_gemm_configure<seq::EpiPartial>());
+    const int gsm = seq::gemm_smem_bytes(seq::KC);
+    CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, gsm));
+    CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, gsm));
+    CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, gsm));
+    CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, gsm));
     CU_OK(cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking));
   }
   CU_OK(cudaDeviceSynchronize());
@@ -1044,8 +1045,8 @@ int tf_skinny_gemm_noalloc(const void* a_dev, const void* w_dev, const float* bi
   int dev = 0;
   CU_OK(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return fail(TF_EINVAL, "device ordinal %d not supported", dev);
-  using Kern = void (*)(const bf16*, const bf16*, int, int, int, int, seq::EpiPartial, const int*, int, int, int);
-  Kern kern = seq::seq_gemm_kernel<8, seq::EpiPartial>;
+  using Kern = void (*)(const bf16*, const bf16*, int, int, int, int, float*, const int*, int, int, int);
+  Kern kern = seq::seq_gemm_kernel<8>;
   const int smem = seq::gemm_smem_bytes(klen);
   if (!g_noalloc_ptr[dev]) {  // once per device, with that device current: resolve the symbol to a device address
     unsigned char* p = nullptr;
@@ -1061,7 +1062,7 @@ int tf_skinny_gemm_noalloc(const void* a_dev, const void* w_dev, const float* bi
   CU_OK(cudaMemsetAsync(step_word, 0, sizeof(int), st));
   dim3 grid((N + 7) / 8, ksplit, (M + seq::ROWS - 1) / seq::ROWS);
   kern<<<grid, seq::THREADS, smem, st>>>(reinterpret_cast<const bf16*>(a_dev), reinterpret_cast<const bf16*>(w_dev), M, N, K,
-                                         klen, seq::EpiPartial{part, M, N}, step_word, 0, 1, 0);
+                                         klen, part, step_word, 0, 1, 0);
   TF_TRY(check_launch("seq_gemm_kernel (no-alloc)"));
   const size_t total = (size_t)M * N;
   int blocks = (int)((total + 255) / 256);
