@@ -26,6 +26,7 @@
 // for the whole block.
 #pragma once
 #include "common.cuh"
+#include "gemm_tc.cuh"
 
 namespace seq {
 
@@ -202,6 +203,108 @@ seq_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W, int B, i
       const int n = blockIdx.x * NC + c;
       if (n < N) out[(size_t)r * N + n] = sum;
     }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same partial product on the 5th-generation tensor cores (legacy mma.sync runs at a fraction of the
+// tcgen05 rate on this architecture).  The roles are swapped so that the weight slice supplies the M = 128
+// dimension of the instruction: D^T[128 columns n, RT batch rows] = W[n0.., k-slice] * A[row0.., k-slice]^T.
+//   * TMA brings kbn (<= 4) slabs of 64 k into shared memory, weights [128 x 64] and activations [RT x 64],
+//     128-byte swizzled, one mbarrier per slab; the weight loads are issued before the wait on the
+//     previous kernel (weights are constants), the activation loads after it;
+//   * one thread issues 4 tcgen05.mma (M=128, N=RT, K=16) per slab into RT columns of tensor memory;
+//   * the four warps read their 32 TMEM lanes (lane = output column n) and store part[ks][b][n], so the
+//     32 lanes of a warp write 32 consecutive floats.
+//   grid = (ceil(N / 128), (K / 64) / kbn, ceil(B / RT)), 128 threads, RT in {16, 32, 64}.
+// Every wait is bounded (see gemm_tc.cuh); a wait that expires records a code in *err and the CTA
+// leaves without storing.
+// ---------------------------------------------------------------------------------------------
+template <int RT>
+__host__ __device__ constexpr int gemm_tc_smem_bytes() { return 4 * (128 * 64 * 2 + RT * 64 * 2) + 64 + 1024; }
+
+template <int RT>
+__global__ void __launch_bounds__(128)
+seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a, int B, int N, int kbn,
+                   float* __restrict__ part, const int* __restrict__ step_base, int step_off, int n_steps, int check_steps,
+                   int* err) {
+  using namespace tc;
+  pdl_launch_dependents();
+  constexpr int W_BYTES = 128 * 64 * 2, A_BYTES = RT * 64 * 2, STAGE = W_BYTES + A_BYTES;
+  constexpr uint32_t TMEM_COLS = RT < 32 ? 32 : RT;
+  extern __shared__ uint8_t smem_seq_tc[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_seq_tc) + 1023) & ~(uintptr_t)1023);
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_base + 4 * STAGE;  // full[0..3], done
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + 4 * STAGE + 48);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * 128, ks = blockIdx.y, row0 = blockIdx.z * RT;
+  const int k0 = ks * kbn * 64;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 5; ++i) mbar_init(bar_base + 8u * i, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (threadIdx.x == 0) {  // weight slabs: constants, requested before the previous kernel has finished
+    for (int kb = 0; kb < kbn; ++kb) {
+      mbar_arrive_expect_tx(bar_base + 8u * kb, STAGE);
+      tma_load_2d(smem_base + kb * STAGE, &map_w, k0 + kb * 64, n0, bar_base + 8u * kb);
+    }
+  }
+  pdl_wait();  // activations and the step counter are complete from here on
+  const bool skip = check_steps && (*step_base + step_off >= n_steps);
+  bool ok = true;
+  if (threadIdx.x == 0) {
+    for (int kb = 0; kb < kbn; ++kb)
+      tma_load_2d(smem_base + kb * STAGE + W_BYTES, &map_a, k0 + kb * 64, row0, bar_base + 8u * kb);
+    constexpr uint32_t idesc = make_idesc(RT);
+    for (int kb = 0; kb < kbn && ok; ++kb) {
+      ok = mbar_wait(bar_base + 8u * kb, 0u, err, TFERR_WAIT_FULL);
+      if (!ok) break;
+      tcgen05_fence_after();
+      const uint64_t wdesc = make_smem_desc(smem_base + kb * STAGE), adesc = make_smem_desc(smem_base + kb * STAGE + W_BYTES);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) umma_f16(tmem_base, wdesc + 2u * k, adesc + 2u * k, idesc, (kb | k) != 0);
+    }
+    if (ok) umma_commit(bar_base + 8u * 4);
+  }
+  ok = mbar_wait(bar_base + 8u * 4, 0u, err, TFERR_WAIT_TMEM_FULL);
+  tcgen05_fence_after();
+  if (ok && !skip) {
+    const int n = n0 + warp * 32 + lane;
+    float* out = part + ((size_t)ks * B + row0) * N + n;
+    const int nrows = (B - row0) < RT ? (B - row0) : RT;
+#pragma unroll 1
+    for (int c = 0; c < (RT + 31) / 32; ++c) {
+      float v[32];
+      tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), v);
+      if (n < N) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (c * 32 + j < nrows) out[(size_t)(c * 32 + j) * N] = v[j];
+      }
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    if (*reinterpret_cast<volatile int*>(err) != 0) {  // a wait gave up: let copies and MMAs in flight drain
+      unsigned long long t0 = globaltimer_ns();
+      while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tcgen05_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 

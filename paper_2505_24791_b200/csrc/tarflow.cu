@@ -96,6 +96,7 @@ struct Matrix {       // a linear layer's weight [N, K]
   int N = 0, K = 0;
   CUtensorMap map;    // bf16 engine: box 64 x bn
   int bn = 0;
+  CUtensorMap map_seq;  // bf16 engine: box 64 x 128 for the sequential-step GEMM
 };
 struct LayerW {
   float *ln1_g, *ln1_b, *b_qkv, *b_o, *ln2_g, *ln2_b, *b_1, *b_2;
@@ -119,6 +120,8 @@ struct tf_model {
   void *xn = nullptr, *qkv = nullptr, *att = nullptr, *mlp = nullptr, *kcache = nullptr, *vcache = nullptr;
   void *xn_lo = nullptr, *qkv_lo = nullptr, *att_lo = nullptr, *mlp_lo = nullptr;  // second terms (bf16 engine)
   CUtensorMap map_xn, map_att, map_mlp, map_xn_lo, map_att_lo, map_mlp_lo;
+  CUtensorMap map_seq_a[3][3];  // sequential-step GEMM operands {xn, att, mlp} x row tile {16, 32, 64}
+  bool seq_use_tc = true;       // sequential-step GEMMs on tcgen05 (false: the mma.sync kernel)
   int *idx = nullptr, *idx_tmp = nullptr, *phase = nullptr, *ctrl = nullptr, *iters_sample = nullptr, *err = nullptr;
   // precision policy of Jacobi blocks on the bf16 engine: 0 = escalate per sample, 1 = single bf16
   // operands only, 2 = two-term operands for every sweep
@@ -408,9 +411,35 @@ static int launch_seq(tf_model* m, int cls, void (*kern)(KArgs...), dim3 grid, i
 // One skinny GEMM of a decoding step: part[ks][B, N] = A[B, K slice ks] W[N, K slice ks]^T.  Returns the number of
 // K slices in *nsplit; the kernel that consumes the tiles adds them up.  CTAs of 64 columns x 256 of K read as many
 // activation bytes as weight bytes and give a grid of (N / 64) * (K / 256) CTAs.
-static int seq_gemm(tf_model* m, int cls, const bf16* A, const Matrix& W, int B, int step_off, int* nsplit) {
+static int seq_gemm(tf_model* m, int cls, int abuf, const Matrix& W, int B, int step_off, int* nsplit) {
   const int N = W.N, K = W.K, n_steps = m->L - 1;
+  const bf16* A = reinterpret_cast<const bf16*>(abuf == 0 ? m->xn : abuf == 1 ? m->att : m->mlp);
   const bf16* w = reinterpret_cast<const bf16*>(W.w);
+  if (m->seq_use_tc) {  // tcgen05 kernel: CTAs of 128 columns x kbn slabs of 64 k
+    const int slabs = K / 64;
+    int kbn = slabs % 4 == 0 ? 4 : slabs % 2 == 0 ? 2 : 1;
+    // more, smaller CTAs while the grid is below one wave and the partial tiles stay <= 16
+    while (kbn > 1 && ((N + 127) / 128) * (slabs / kbn) < m->num_sms && slabs / (kbn / 2) <= 16) kbn /= 2;
+    if (const char* e = getenv("TARFLOW_SEQ_KBN")) {
+      const int f = atoi(e);
+      if ((f == 1 || f == 2 || f == 4) && slabs % f == 0 && slabs / f <= 16) kbn = f;
+    }
+    const int ksplit = slabs / kbn;
+    if (ksplit > 16) return fail(TF_EINVAL, "sequential decoding: reduction length %d not supported", K);
+    *nsplit = ksplit;
+    if ((size_t)ksplit * B * N > m->seq_part_floats) return fail(TF_EINVAL, "sequential decoding: partial-tile buffer too small");
+    const int ri = B <= 16 ? 0 : B <= 32 ? 1 : 2, rt = 16 << ri;
+    dim3 grid((N + 127) / 128, ksplit, (B + rt - 1) / rt);
+#define TF_SEQ_TC_CASE(RTV)                                                                                              \
+  if (rt == RTV)                                                                                                         \
+    return launch_seq(m, cls, seq::seq_gemm_tc_kernel<RTV>, grid, 128, seq::gemm_tc_smem_bytes<RTV>(), W.map_seq,         \
+                      m->map_seq_a[abuf][ri], B, N, kbn, m->seq_part, m->step_ctr, step_off, n_steps, m->seq_check_steps, \
+                      m->err);
+    TF_SEQ_TC_CASE(16)
+    TF_SEQ_TC_CASE(32)
+    TF_SEQ_TC_CASE(64)
+#undef TF_SEQ_TC_CASE
+  }
   const int row_tiles = (B + seq::ROWS - 1) / seq::ROWS;
   int klen = (K % 256 == 0) ? 256 : K;
   while (K / klen > 16 && K % (klen * 2) == 0) klen *= 2;  // at most 16 partial tiles
@@ -452,7 +481,6 @@ static int seq_resid_ln(tf_model* m, const float* bias, int nsplit, const float*
 static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const float* v, float* u, int count) {
   const BlockW& bw = m->blocks[g];
   const int L = m->L, D = m->D, d = m->d, rev = g & 1, nl = m->cfg.n_layers, heads = m->cfg.n_heads;
-  bf16* xn = reinterpret_cast<bf16*>(m->xn);
   bf16* att = reinterpret_cast<bf16*>(m->att);
   bf16* mlp = reinterpret_cast<bf16*>(m->mlp);
   const size_t layer_stride = (size_t)m->cfg.max_batch * L * d;
@@ -467,19 +495,19 @@ static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const
       bf16* kc = reinterpret_cast<bf16*>(m->kcache) + i * layer_stride;
       bf16* vc = reinterpret_cast<bf16*>(m->vcache) + i * layer_stride;
       TF_TRY(seq_resid_ln(m, pending_bias, pending, lw.ln1_g, lw.ln1_b, B, s));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, lw.w_qkv, B, s, &ns));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 0, lw.w_qkv, B, s, &ns));
       TF_TRY(launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, m->seq_part, ns, lw.b_qkv, kc, vc,
                         att, B, L, d, heads, scale * 1.4426950408889634f, m->step_ctr, s, L - 1));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, att, lw.w_o, B, s, &pending));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 1, lw.w_o, B, s, &pending));
       TF_TRY(seq_resid_ln(m, lw.b_o, pending, lw.ln2_g, lw.ln2_b, B, s));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, lw.w_1, B, s, &ns));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 0, lw.w_1, B, s, &ns));
       TF_TRY(launch_seq(m, KC_SEQ_LN, seq::seq_bias_gelu_kernel, dim3((B * (m->hid / 4) + 255) / 256), 256, 0, m->seq_part, ns,
                         lw.b_1, mlp, B, m->hid, m->step_ctr, s, L - 1, m->seq_check_steps));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, mlp, lw.w_2, B, s, &pending));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 2, lw.w_2, B, s, &pending));
       pending_bias = lw.b_2;
     }
     TF_TRY(seq_resid_ln(m, pending_bias, pending, bw.lnf_g, bw.lnf_b, B, s));
-    TF_TRY(seq_gemm(m, KC_SEQ_GEMM, xn, bw.w_out, B, s, &ns));
+    TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 0, bw.w_out, B, s, &ns));
     TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B), ethreads, (int)(D * sizeof(float)), m->seq_part,
                       ns, bw.b_out, B, v, u, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 0, m->step_ctr, s,
                       L - 1));
@@ -705,6 +733,7 @@ static int upload_matrix(tf_model* m, Matrix* W, const float* src, int N, int K,
   CU_OK(cudaDeviceSynchronize());
   W->w = w;
   W->bn = (N % 256 == 0) ? 256 : 128;
+  TF_TRY(make_map_bf16(&W->map_seq, w, (uint64_t)N, (uint64_t)K, 128u));
   return make_map_bf16(&W->map, w, (uint64_t)N, (uint64_t)K, (uint32_t)W->bn);
 }
 
@@ -816,7 +845,7 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
   if (c.dtype == 1) {  // partial tiles: up to 16 K slices of a [B, d] output, or d/256 slices of the widest one
     const size_t wide = (size_t)(hid > 3 * d ? hid : 3 * d);
     m->seq_part_floats = (size_t)16 * B * d;
-    const size_t per_wide = (size_t)((d % 256 == 0) ? d / 256 : 1) * B * wide;
+    const size_t per_wide = (size_t)(d / 64 < 16 ? d / 64 : 16) * B * wide;
     if (per_wide > m->seq_part_floats) m->seq_part_floats = per_wide;
     TF_TRY(dev_alloc(m, &m->seq_part, m->seq_part_floats));
   }
@@ -832,6 +861,16 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     TF_TRY(make_map_bf16(&m->map_xn_lo, m->xn_lo, M, d, tc::BM));
     TF_TRY(make_map_bf16(&m->map_att_lo, m->att_lo, M, d, tc::BM));
     TF_TRY(make_map_bf16(&m->map_mlp_lo, m->mlp_lo, M, hid, tc::BM));
+    for (int r = 0; r < 3; ++r) {
+      const uint32_t rt = 16u << r;
+      TF_TRY(make_map_bf16(&m->map_seq_a[0][r], m->xn, M, d, rt));
+      TF_TRY(make_map_bf16(&m->map_seq_a[1][r], m->att, M, d, rt));
+      TF_TRY(make_map_bf16(&m->map_seq_a[2][r], m->mlp, M, hid, rt));
+    }
+    CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<16>()));
+    CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<32>()));
+    CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<64>()));
+    if (const char* e = getenv("TARFLOW_SEQ_MMA")) m->seq_use_tc = atoi(e) == 0;
     CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                attn::smem_bytes<true>()));
     CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
