@@ -214,8 +214,8 @@ seq_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W, int B, i
 //     128-byte swizzled, one mbarrier per slab; the weight loads are issued before the wait on the
 //     previous kernel (weights are constants), the activation loads after it;
 //   * one thread issues 4 tcgen05.mma (M=128, N=RT, K=16) per slab into RT columns of tensor memory;
-//   * the four warps read their 32 TMEM lanes (lane = output column n) and store part[ks][b][n], so the
-//     32 lanes of a warp write 32 consecutive floats.
+//   * the four warps read their 32 TMEM lanes (lane = output column n), transpose through shared memory
+//     and store part[ks][b][n] with 16-byte stores, 512 contiguous bytes per warp.
 //   grid = (ceil(N / 128), (K / 64) / kbn, ceil(B / RT)), 128 threads, RT in {16, 32, 64}.
 // Every wait is bounded (see gemm_tc.cuh); a wait that expires records a code in *err and the CTA
 // leaves without storing.
@@ -281,18 +281,33 @@ seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   }
   ok = mbar_wait(bar_base + 8u * 4, 0u, err, TFERR_WAIT_TMEM_FULL);
   tcgen05_fence_after();
-  if (ok && !skip) {
-    const int n = n0 + warp * 32 + lane;
-    float* out = part + ((size_t)ks * B + row0) * N + n;
-    const int nrows = (B - row0) < RT ? (B - row0) : RT;
+  // TMEM (lane = output column) -> shared memory tile [RT rows][128 columns] in the operand stages, which are
+  // free once the MMAs have completed -> 16-byte stores, 512 contiguous bytes per warp
+  constexpr int TP = 128 + 4;  // tile pitch in floats
+  float* tile = reinterpret_cast<float*>(smem);
+  if (ok) {
 #pragma unroll 1
     for (int c = 0; c < (RT + 31) / 32; ++c) {
       float v[32];
       tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), v);
-      if (n < N) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (c * 32 + j < nrows) out[(size_t)(c * 32 + j) * N] = v[j];
+      for (int j = 0; j < 32; ++j)
+        if (c * 32 + j < RT) tile[(c * 32 + j) * TP + warp * 32 + lane] = v[j];
+    }
+  }
+  __syncthreads();
+  if (ok && !skip) {
+    const int nrows = (B - row0) < RT ? (B - row0) : RT;
+    const int n = n0 + 4 * lane;
+    float* out = part + ((size_t)ks * B + row0) * N + n;
+    for (int r = warp; r < nrows; r += 4) {
+      const float4 x = *reinterpret_cast<const float4*>(tile + r * TP + 4 * lane);
+      if (n + 3 < N) {
+        *reinterpret_cast<float4*>(out + (size_t)r * N) = x;
+      } else {
+        if (n < N) out[(size_t)r * N] = x.x;
+        if (n + 1 < N) out[(size_t)r * N + 1] = x.y;
+        if (n + 2 < N) out[(size_t)r * N + 2] = x.z;
       }
     }
   }

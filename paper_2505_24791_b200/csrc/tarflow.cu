@@ -418,8 +418,8 @@ static int seq_gemm(tf_model* m, int cls, int abuf, const Matrix& W, int B, int 
   if (m->seq_use_tc) {  // tcgen05 kernel: CTAs of 128 columns x kbn slabs of 64 k
     const int slabs = K / 64;
     int kbn = slabs % 4 == 0 ? 4 : slabs % 2 == 0 ? 2 : 1;
-    // more, smaller CTAs while the grid is below one wave and the partial tiles stay <= 16
-    while (kbn > 1 && ((N + 127) / 128) * (slabs / kbn) < m->num_sms && slabs / (kbn / 2) <= 16) kbn /= 2;
+    // two slabs per CTA (more CTAs) while the grid is below one wave and the partial tiles stay <= 16
+    if (kbn == 4 && ((N + 127) / 128) * (slabs / 4) < m->num_sms && slabs / 2 <= 16) kbn = 2;
     if (const char* e = getenv("TARFLOW_SEQ_KBN")) {
       const int f = atoi(e);
       if ((f == 1 || f == 2 || f == 4) && slabs % f == 0 && slabs / f <= 16) kbn = f;
