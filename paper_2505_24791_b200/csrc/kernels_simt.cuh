@@ -49,6 +49,56 @@ __global__ void embed_kernel(const float* __restrict__ u, const int* __restrict_
   }
 }
 
+// The same embedding for the rows of a full pass, R rows per CTA: every weight element a thread loads is
+// used for R rows (the one-row kernel re-reads the whole [D, d] matrix per row).  The R tokens sit in
+// shared memory transposed, [D][R], so that four rows come with one broadcast 16-byte read.
+template <int R>
+__global__ void __launch_bounds__(256)
+embed_rows_kernel(const float* __restrict__ u, const int* __restrict__ idx, const int* __restrict__ labels,
+                  const float* __restrict__ w_in_t, const float* __restrict__ b_in, const float* __restrict__ pos,
+                  const float* __restrict__ cls, float* __restrict__ h, int L, int D, int d, int reversed, int n_rows) {
+  extern __shared__ __align__(16) float s_ut[];  // [D][R]
+  const int row0 = blockIdx.x * R;
+  for (int e = threadIdx.x; e < R * D; e += blockDim.x) {
+    const int r = e / D, c = e - r * D, row = row0 + r;
+    float val = 0.f;
+    if (row < n_rows) {
+      const int s = row / L, l = row - s * L;
+      const int b = idx ? idx[s] : s;
+      val = u[((size_t)b * L + tok_index(l, L, reversed)) * D + c];
+    }
+    s_ut[c * R + r] = val;
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < d; j += blockDim.x) {
+    float acc[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) acc[r] = 0.f;
+    for (int c = 0; c < D; ++c) {
+      const float w = w_in_t[(size_t)c * d + j];
+#pragma unroll
+      for (int r4 = 0; r4 < R; r4 += 4) {
+        const float4 x = *reinterpret_cast<const float4*>(s_ut + c * R + r4);
+        acc[r4] = fmaf(x.x, w, acc[r4]);
+        acc[r4 + 1] = fmaf(x.y, w, acc[r4 + 1]);
+        acc[r4 + 2] = fmaf(x.z, w, acc[r4 + 2]);
+        acc[r4 + 3] = fmaf(x.w, w, acc[r4 + 3]);
+      }
+    }
+    const float bj = b_in[j];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const int row = row0 + r;
+      if (row < n_rows) {
+        const int s = row / L, l = row - s * L;
+        float a = acc[r] + (bj + pos[(size_t)l * d + j]);
+        if (cls != nullptr) a += cls[(size_t)labels[idx ? idx[s] : s] * d + j];
+        h[(size_t)row * d + j] = a;
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // LayerNorm over the last dimension (eps 1e-5), fp32 in, T out.  One warp per row, the row is
 // held in registers (d <= 32*4*MAXV).

@@ -529,8 +529,10 @@ seq_attention_kernel(const float* __restrict__ part, int nsplit, const float* __
 // u[b, t+1, :] = v[b, t+1, :] * exp(alpha~) + mu~ from the head projection's partial tiles [.][B, 2D]
 // (+ bias; columns interleaved mu~_c, alpha~_c), then
 // the embedding of that token for the next step: h[b, :] = u W_in^T + b_in + pos[t+1] (+ cls[y_b]).
-// One CTA per sample.  With first != 0 the step is the block's start: u[b, 0, :] = v[b, 0, :] (Eq. 5,
-// first row) and the embedding of token 0.
+// grid = (B, ceil(d / blockDim.x)): every CTA of a sample recomputes the D values of the token (cheap) and
+// embeds blockDim.x channels, one per thread; the CTA with blockIdx.y == 0 stores the token.  With
+// first != 0 the step is the block's start: u[b, 0, :] = v[b, 0, :] (Eq. 5, first row) and the
+// embedding of token 0.
 // ---------------------------------------------------------------------------------------------
 __global__ void seq_update_embed_kernel(const float* __restrict__ part, int nsplit, const float* __restrict__ bias,
                                         int B, const float* __restrict__ v, float* __restrict__ u,
@@ -558,19 +560,25 @@ __global__ void seq_update_embed_kernel(const float* __restrict__ part, int nspl
       }
       val = fmaf(val, expf(al), mu);
     }
-    u[e0 + c] = val;
+    if (blockIdx.y == 0) u[e0 + c] = val;
     s_tok[c] = val;
   }
   __syncthreads();
   if (l_new >= L - 1) return;  // the last token is never fed back
-  const float* cl = (cls != nullptr) ? cls + (size_t)labels[b] * d : nullptr;
-  for (int j = threadIdx.x; j < d; j += blockDim.x) {
-    float acc = 0.f;
-    for (int c = 0; c < D; ++c) acc = fmaf(s_tok[c], w_in_t[(size_t)c * d + j], acc);
-    acc += b_in[j] + pos[(size_t)l_new * d + j];
-    if (cl) acc += cl[j];
-    h[(size_t)b * d + j] = acc;
+  const int j = blockIdx.y * blockDim.x + threadIdx.x;
+  if (j >= d) return;
+  float acc = b_in[j] + pos[(size_t)l_new * d + j];
+  if (cls != nullptr) acc += cls[(size_t)labels[b] * d + j];
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;  // four independent chains over the token's values
+  int c = 0;
+  for (; c + 4 <= D; c += 4) {
+    a0 = fmaf(s_tok[c], w_in_t[(size_t)c * d + j], a0);
+    a1 = fmaf(s_tok[c + 1], w_in_t[(size_t)(c + 1) * d + j], a1);
+    a2 = fmaf(s_tok[c + 2], w_in_t[(size_t)(c + 2) * d + j], a2);
+    a3 = fmaf(s_tok[c + 3], w_in_t[(size_t)(c + 3) * d + j], a3);
   }
+  for (; c < D; ++c) a0 = fmaf(s_tok[c], w_in_t[(size_t)c * d + j], a0);
+  h[(size_t)b * d + j] = acc + ((a0 + a1) + (a2 + a3));
 }
 
 __global__ void seq_advance_kernel(int* step_base, int by) {

@@ -308,8 +308,8 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
   const CUtensorMap* mml = hp ? &m->map_mlp_lo : nullptr;
   int ethreads = d < 256 ? d : 256;
   m->cur_rows = M;
-  LAUNCH(m, KC_EMBED, embed_kernel, M, ethreads, D * sizeof(float), u_src, idx, labels, bw.w_in_t, bw.b_in, bw.pos,
-         bw.cls, m->h, L, D, d, rev, -1);
+  LAUNCH(m, KC_EMBED, embed_rows_kernel<16>, (M + 15) / 16, ethreads, 16 * D * sizeof(float), u_src, idx, labels, bw.w_in_t,
+         bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, M);
   TF_TRY(check_launch("embed_kernel"));
   for (const LayerW& lw : bw.layers) {
     TF_TRY(layernorm<T>(m, KC_LN, m->h, lw.ln1_g, lw.ln1_b, xn, xn_lo, M));
@@ -485,7 +485,7 @@ static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const
   bf16* mlp = reinterpret_cast<bf16*>(m->mlp);
   const size_t layer_stride = (size_t)m->cfg.max_batch * L * d;
   const float scale = 1.0f / sqrtf((float)m->hd);
-  const int ethreads = d < 256 ? d : 256;
+  const int ethreads = d < 128 ? d : 128;
   m->cur_rows = B;
   for (int s = 0; s < count; ++s) {
     const float* pending_bias = nullptr;  // bias of the projection whose partial tiles are not yet in h
@@ -508,8 +508,8 @@ static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const
     }
     TF_TRY(seq_resid_ln(m, pending_bias, pending, bw.lnf_g, bw.lnf_b, B, s));
     TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 0, bw.w_out, B, s, &ns));
-    TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B), ethreads, (int)(D * sizeof(float)), m->seq_part,
-                      ns, bw.b_out, B, v, u, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 0, m->step_ctr, s,
+    TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B, (d + ethreads - 1) / ethreads), ethreads,
+                      (int)(D * sizeof(float)), m->seq_part, ns, bw.b_out, B, v, u, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 0, m->step_ctr, s,
                       L - 1));
   }
   return check_launch("sequential step kernels");
@@ -525,12 +525,13 @@ static int seq_unroll(int n_steps) {  // steps per graph: a divisor of n_steps c
 static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* labels, const float* v, float* u) {
   const BlockW& bw = m->blocks[g];
   const int L = m->L, D = m->D, d = m->d, rev = g & 1, n_steps = L - 1;
-  const int ethreads = d < 256 ? d : 256;
+  const int ethreads = d < 128 ? d : 128;
   cudaStream_t user = m->stream;
   m->seq_check_steps = (m->prof_on || !m->use_graphs) ? 0 : (n_steps % seq_unroll(n_steps) != 0);
   CU_OK(cudaMemsetAsync(m->step_ctr, 0, sizeof(int), user));
   m->cur_rows = B;
-  TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B), ethreads, (int)(D * sizeof(float)), m->seq_part, 0,
+  TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B, (d + ethreads - 1) / ethreads), ethreads,
+                    (int)(D * sizeof(float)), m->seq_part, 0,
                     bw.b_out, B, v, u, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 1, m->step_ctr, 0,
                     n_steps));
   if (m->prof_on || !m->use_graphs) {  // direct launches (per-kernel events need them)
