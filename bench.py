@@ -242,6 +242,10 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--no-policies", action="store_true", help="skip the all-sequential / all-Jacobi legs")
     ap.add_argument("--kernels", action="store_true", help="add the per-kernel-class table to the JSON line")
+    ap.add_argument("--probe", default=None, choices=["sweep", "seq"],
+                    help="small single-block run for ncu captures: 'sweep' = --sweeps fixed Jacobi sweeps of one block, "
+                         "'seq' = one sequentially decoded block; run twice, the second call timed; not a bench value")
+    ap.add_argument("--sweeps", type=int, default=2)
     ap.add_argument("--launch-list", action="store_true",
                     help="for an ncu launch-list capture: one warm-up and one step of the timed leg only; the line it "
                          "prints is marked as a profiling run and is not a bench value")
@@ -281,6 +285,32 @@ def main():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
+
+    if args.probe:
+        cfg1 = synth.config(args.workload, n_blocks=1)
+        m1 = binding.tf_load(cfg1, synth.pack_blob(cfg1, synth.make_weights(cfg1)), B)
+        z = torch.from_numpy(synth.make_latents(cfg1, 1, B=B)).cuda()
+        lab = synth.make_labels(cfg1, B=B)
+        lab = None if lab is None else torch.from_numpy(lab).cuda()
+        x = torch.empty_like(z)
+        it = np.zeros(1, dtype=np.int32)
+        ms = 0.0
+        for _ in range(2):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            if args.probe == "sweep":
+                binding.tf_inverse_jacobi(m1, z, lab, B, [1], -1.0, args.sweeps, 0, x, it)
+            else:
+                binding.tf_inverse_jacobi(m1, z, lab, B, [0], 0.0, 1, 0, x, it)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+        per = ms / args.sweeps if args.probe == "sweep" else ms
+        print(json.dumps({"profiling_run": True, "note": "not a bench value", "probe": args.probe, "workload": args.workload,
+                          "batch": B, "ms_per_sweep" if args.probe == "sweep" else "ms_per_sequential_block": per,
+                          "finite": bool(torch.isfinite(x).all())}), flush=True)
+        binding.tf_free(m1)
+        return
 
     blocks = synth.make_weights(cfg)
     blob = synth.pack_blob(cfg, blocks)

@@ -22,6 +22,10 @@
  *     passed the stopping test (x holds the last iterate; not an error); negative = error, with a
  *     message available from tf_last_error().  Nothing aborts, throws or traps.
  *   - A tf_model is not thread-safe: it owns one workspace; use it from one thread/stream at a time.
+ *   - Tuning aids read from the environment (bf16 engine, sequential decoding only; results are unchanged
+ *     up to summation order): TARFLOW_SEQ_MMA=1 selects the mma.sync step GEMM instead of the tcgen05 one,
+ *     TARFLOW_SEQ_KBN=1|2|4 the 64-wide k slabs per CTA of the tcgen05 step GEMM, TARFLOW_SEQ_NC=8|16|32|64
+ *     the column-slice width of the mma.sync step GEMM.
  */
 #ifndef TARFLOW_H_
 #define TARFLOW_H_
