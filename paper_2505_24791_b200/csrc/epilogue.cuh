@@ -10,7 +10,18 @@
 //     accumulator columns of the lane's own row and the chunk's bias in shared memory, and writes the
 //     row segment with 16-byte stores (64 contiguous bytes per lane: whole sectors).
 #pragma once
+#include <cuda.h>
+
 #include "common.cuh"
+
+namespace tc {  // defined in gemm_tc.cuh
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src);
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, int x, int y, uint32_t src);
+__device__ __forceinline__ void tma_store_commit();
+__device__ __forceinline__ void tma_store_wait_read();
+__device__ __forceinline__ void fence_proxy_async_smem();
+__device__ __forceinline__ uint32_t swz128(int r, int k);
+}  // namespace tc
 
 // out[row, col] = act(acc + bias[col]).  With `out_lo` set (bf16 only) the value is stored as an
 // error-compensated pair: out = bf16(x), out_lo = bf16(x - out), so that out + out_lo carries about
@@ -22,6 +33,7 @@ struct EpiStore {
   int ldc;
   OutT* out_lo = nullptr;
   static constexpr bool kRowwise = sizeof(OutT) == 2;
+  static constexpr int kTmaCols = 0;
   // sbias: the 32 biases of columns col0.. (zeros without a bias), warp-private shared memory
   __device__ __forceinline__ void rowwise(int row, int col0, float (&v)[32], int nv, const float* sbias) const {
 #pragma unroll
@@ -121,6 +133,7 @@ struct EpiResid {  // h[row, col] += acc + bias[col]   (fp32 residual stream, in
   const float* bias;
   int ldc;
   static constexpr bool kRowwise = false;
+  static constexpr int kTmaCols = 0;
   __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
   __device__ __forceinline__ void store(int row, int col, float acc, float cc, bool col_ok, int) const {
     if (col_ok) {
@@ -197,6 +210,7 @@ struct EpiHeadUpdate {
   const float* bias;   // [2D] interleaved
   int L, D, reversed;
   static constexpr bool kRowwise = false;
+  static constexpr int kTmaCols = 0;
   __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
   // lane-per-column form: even lanes hold mu~_c, the next lane alpha~_c
   __device__ __forceinline__ void store(int row, int col, float acc, float cc, bool col_ok, int lane) const {
@@ -260,5 +274,90 @@ struct EpiHeadUpdate {
       }
     }
     atomic_max_nonneg(maxdiff + b, m);
+  }
+};
+
+// ---- bulk-store forms for the tcgen05 GEMM (kTmaCols > 0): tma_box<CPG>(first chunk, last chunk, biases of the box's
+// columns in shared memory, first column, first row, staging box, its shared address, lane).  The lane owns row
+// `row0 + lane`; it writes its 128 bytes of the box as eight 16-byte pieces in the swizzled order of the tensor map.
+
+// bf16 activations: out[row, col..col+63] = bf16(act(acc + bias)), optionally with the second (error) term.
+template <bool GELU>
+struct EpiStoreTma {
+  const float* bias;  // may be null
+  const CUtensorMap* tmap;
+  const CUtensorMap* tmap_lo;  // null = single term
+  static constexpr bool kRowwise = false;
+  static constexpr int kTmaCols = 64;
+  __device__ __forceinline__ float col_const(int col, bool col_ok) const { return (bias != nullptr && col_ok) ? bias[col] : 0.f; }
+  template <int CPG>
+  __device__ __forceinline__ void tma_box(float (&v0)[32], float (&v1)[32], const float* sbias, int col0, int row0, uint8_t* box,
+                                          uint32_t box_addr, int lane) const {
+    static_assert(CPG == 2, "a bf16 box is two 32-column chunks");
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {
+      const float4 b0 = *reinterpret_cast<const float4*>(sbias + j), b1 = *reinterpret_cast<const float4*>(sbias + 32 + j);
+      v0[j] += b0.x; v0[j + 1] += b0.y; v0[j + 2] += b0.z; v0[j + 3] += b0.w;
+      v1[j] += b1.x; v1[j + 1] += b1.y; v1[j + 2] += b1.z; v1[j + 3] += b1.w;
+    }
+    if (GELU) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) { v0[j] = gelu_erf_fast(v0[j]); v1[j] = gelu_erf_fast(v1[j]); }
+    }
+    write_box(v0, v1, box, lane);
+    tc::fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) { tc::tma_store_2d(tmap, col0, row0, box_addr); tc::tma_store_commit(); }
+    if (tmap_lo != nullptr) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        v0[j] -= __bfloat162float(__float2bfloat16_rn(v0[j]));
+        v1[j] -= __bfloat162float(__float2bfloat16_rn(v1[j]));
+      }
+      if (lane == 0) tc::tma_store_wait_read();  // the engine has read the first box
+      __syncwarp();
+      write_box(v0, v1, box, lane);
+      tc::fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) { tc::tma_store_2d(tmap_lo, col0, row0, box_addr); tc::tma_store_commit(); }
+    }
+    if (lane == 0) tc::tma_store_wait_read();  // the box may be overwritten by the next call
+    __syncwarp();
+  }
+  __device__ __forceinline__ void write_box(const float (&v0)[32], const float (&v1)[32], uint8_t* box, int lane) const {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {  // 16-byte piece k = columns 8k .. 8k+7 of the box
+      const float* src = k < 4 ? &v0[8 * k] : &v1[8 * (k - 4)];
+      const __nv_bfloat162 a = __floats2bfloat162_rn(src[0], src[1]), b = __floats2bfloat162_rn(src[2], src[3]);
+      const __nv_bfloat162 c = __floats2bfloat162_rn(src[4], src[5]), d = __floats2bfloat162_rn(src[6], src[7]);
+      uint4 u;
+      u.x = *reinterpret_cast<const uint32_t*>(&a); u.y = *reinterpret_cast<const uint32_t*>(&b);
+      u.z = *reinterpret_cast<const uint32_t*>(&c); u.w = *reinterpret_cast<const uint32_t*>(&d);
+      *reinterpret_cast<uint4*>(box + tc::swz128(lane, k)) = u;
+    }
+  }
+};
+
+// fp32 residual stream: h[row, col..col+31] += acc + bias, added in memory by the TMA engine (no read by the SM).
+struct EpiResidTma {
+  const float* bias;
+  const CUtensorMap* tmap;  // fp32 [rows, d], box 32 columns x 32 rows, 128-byte swizzle
+  static constexpr bool kRowwise = false;
+  static constexpr int kTmaCols = 32;
+  __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
+  template <int CPG>
+  __device__ __forceinline__ void tma_box(float (&v)[32], float (&)[32], const float* sbias, int col0, int row0, uint8_t* box,
+                                          uint32_t box_addr, int lane) const {
+    static_assert(CPG == 1, "an fp32 box is one 32-column chunk");
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float4 b = *reinterpret_cast<const float4*>(sbias + 4 * k);
+      *reinterpret_cast<float4*>(box + tc::swz128(lane, k)) =
+          make_float4(v[4 * k] + b.x, v[4 * k + 1] + b.y, v[4 * k + 2] + b.z, v[4 * k + 3] + b.w);
+    }
+    tc::fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) { tc::tma_reduce_add_2d(tmap, col0, row0, box_addr); tc::tma_store_commit(); tc::tma_store_wait_read(); }
+    __syncwarp();
   }
 };

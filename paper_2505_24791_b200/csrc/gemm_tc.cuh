@@ -80,6 +80,28 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// Bulk tensor stores from shared memory (the TMA engine writes whole row segments; the SM issues one
+// instruction per box).  `tma_reduce_add_2d` adds the fp32 box into global memory instead of storing it.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x), "r"(y), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x),
+               "r"(y), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+// Byte offset of 16-byte chunk `k` (0..7) of row `r` inside a [rows][128 bytes] staging box with the
+// 128-byte swizzle the tensor maps use (box base 1024-byte aligned).
+__device__ __forceinline__ uint32_t swz128(int r, int k) { return (uint32_t)(r * 128 + ((k ^ (r & 7)) << 4)); }
+
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -117,6 +139,24 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// Issue only: the registers are valid after tmem_ld_wait().
+__device__ __forceinline__ void tmem_ld_32x32b_x32_issue(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, float (&v)[32]) {
   uint32_t r[32];
   asm volatile(
@@ -139,17 +179,23 @@ struct SmemLayout {
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+  // after the operand ring (a multiple of 1024 bytes): the epilogue staging area, per warp either a padded 32x33
+  // fp32 transpose tile (4224 B stride) or a swizzled [32][128 B] box for bulk stores (4096 B stride) followed by
+  // the tile's 256 biases; then the mbarriers and the TMEM slot
+  static constexpr int STAGE_OUT_OFFSET = STAGES * STAGE_BYTES;
+  static constexpr int STAGE_OUT_BYTES = NUM_EPI_WARPS * 32 * 33 * 4;
+  static constexpr int TILE_BIAS_OFFSET = STAGE_OUT_OFFSET + NUM_EPI_WARPS * 4096;
+  static constexpr int BAR_OFFSET = STAGE_OUT_OFFSET + STAGE_OUT_BYTES;
   static constexpr int NUM_BARS = 2 * STAGES + 4;
-  static constexpr int STAGE_OUT_OFFSET = BAR_OFFSET + NUM_BARS * 8 + 16;  // after barriers + tmem slot
-  static constexpr int STAGE_OUT_BYTES = NUM_EPI_WARPS * 32 * 33 * 4;  // one padded 32x32 fp32 chunk per epilogue warp
-  static constexpr int TOTAL = STAGE_OUT_OFFSET + STAGE_OUT_BYTES + 1024;  // + alignment slack
+  static constexpr int TOTAL = BAR_OFFSET + NUM_BARS * 8 + 16 + 1024;  // + tmem slot + alignment slack
 };
 
 template <int BN, int STAGES, class Epi>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_a_lo,
                const __grid_constant__ CUtensorMap map_w, int M, int N, int K, int split, Epi epi, int* err) {
+  static_assert(SmemLayout<BN, STAGES>::TILE_BIAS_OFFSET + 1024 <= SmemLayout<BN, STAGES>::STAGE_OUT_OFFSET +
+                SmemLayout<BN, STAGES>::STAGE_OUT_BYTES, "bias tile must fit behind the store boxes");
   using SL = SmemLayout<BN, STAGES>;
   extern __shared__ uint8_t smem_raw[];
   __shared__ int s_prev_err;
@@ -253,6 +299,50 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     float* stage_out = reinterpret_cast<float*>(smem + SL::STAGE_OUT_OFFSET) + (warp - 2) * (32 * 33);
     bool ok = true;
     int it = 0;
+    if constexpr (Epi::kTmaCols > 0) {
+      // Bulk-store epilogue: each warp owns NCH adjacent 32-column chunks of its 32 rows; values leave the
+      // registers row-per-lane as 16-byte shared-memory writes into a swizzled [32][128 B] box, and one lane
+      // hands the box to the TMA engine (store, or fp32 add into the residual stream).
+      constexpr int NCH = BN / 32 / (NUM_EPI_WARPS / 4);
+      constexpr int CPG = Epi::kTmaCols / 32;  // chunks per box: 2 (bf16, 64 columns) or 1 (fp32, 32 columns)
+      static_assert(NCH % CPG == 0, "box width must divide the warp's columns");
+      const int etid = threadIdx.x - 64;       // 0 .. 32 * NUM_EPI_WARPS - 1
+      uint8_t* box = smem + SL::STAGE_OUT_OFFSET + (warp - 2) * 4096;
+      const uint32_t box_addr = smem_u32(box);
+      float* tile_bias = reinterpret_cast<float*>(smem + SL::TILE_BIAS_OFFSET);
+      for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+        const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1;
+        // the tile's biases, once, while the mainloop still runs
+        named_bar_sync(1, 32 * NUM_EPI_WARPS);
+        if (etid < BN) tile_bias[etid] = epi.col_const(n0 + etid, n0 + etid < N);
+        named_bar_sync(1, 32 * NUM_EPI_WARPS);
+        // a warp whose wait gave up keeps walking the tile list (without work), so the named barrier above
+        // is always reached by all epilogue warps
+        if (ok && !mbar_wait(tfull_bar(acc), acc_phase, err, TFERR_WAIT_TMEM_FULL)) ok = false;
+        if (!ok) continue;
+        tcgen05_fence_after();
+        const int row0 = m0 + quad * 32;
+        float v[NCH][32];
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch)
+          tmem_ld_32x32b_x32_issue(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + (cgroup * NCH + ch) * 32),
+                                   v[ch]);
+        tmem_ld_wait();
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));  // the accumulator is in registers: free it for the next tile
+        if (row0 < M) {
+#pragma unroll
+          for (int g = 0; g < NCH / CPG; ++g) {
+            const int cl = (cgroup * NCH + g * CPG) * 32;  // first column of the box inside the tile
+            if (n0 + cl < N) epi.template tma_box<CPG>(v[g * CPG], v[g * CPG + CPG - 1], tile_bias + cl, n0 + cl, row0, box, box_addr, lane);
+          }
+        }
+      }
+      if (lane == 0) tma_store_wait_all();
+    } else {
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
       const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
       const int acc = it & 1;
@@ -299,6 +389,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
+    }
     }
   }
 

@@ -79,6 +79,23 @@ static int make_map_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, uint6
   return TF_OK;
 }
 
+// Store map for the bulk-store epilogues: matrix [rows, cols] row-major of 2-byte (bf16) or 4-byte (fp32) elements,
+// box = 128 bytes of a row x 32 rows, 128-byte swizzle.
+static int make_map_store(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, int elem_bytes) {
+  encode_tiled_fn fn = get_encode_fn();
+  if (!fn) return fail(TF_ECUDA, "cuTensorMapEncodeTiled entry point not available");
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || (cols * elem_bytes) % 16) return fail(TF_EINVAL, "TMA operand not 16-byte aligned");
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
+  cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                  const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(TF_ECUDA, "cuTensorMapEncodeTiled (store map) failed (%d)", (int)r);
+  return TF_OK;
+}
+
 // ------------------------------------------------------------------------------------------------
 // model
 // ------------------------------------------------------------------------------------------------
@@ -120,6 +137,8 @@ struct tf_model {
   void *xn = nullptr, *qkv = nullptr, *att = nullptr, *mlp = nullptr, *kcache = nullptr, *vcache = nullptr;
   void *xn_lo = nullptr, *qkv_lo = nullptr, *att_lo = nullptr, *mlp_lo = nullptr;  // second terms (bf16 engine)
   CUtensorMap map_xn, map_att, map_mlp, map_xn_lo, map_att_lo, map_mlp_lo;
+  enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_COUNT };
+  CUtensorMap* store_maps = nullptr;  // device copy of the bulk-store maps of qkv, qkv_lo, mlp, mlp_lo, h
   CUtensorMap map_seq_a[3][3];  // sequential-step GEMM operands {xn, att, mlp} x row tile {16, 32, 64}
   bool seq_use_tc = true;       // sequential-step GEMMs on tcgen05 (false: the mma.sync kernel)
   int *idx = nullptr, *idx_tmp = nullptr, *phase = nullptr, *ctrl = nullptr, *iters_sample = nullptr, *err = nullptr;
@@ -313,7 +332,13 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
   TF_TRY(check_launch("embed_kernel"));
   for (const LayerW& lw : bw.layers) {
     TF_TRY(layernorm<T>(m, KC_LN, m->h, lw.ln1_g, lw.ln1_b, xn, xn_lo, M));
-    TF_TRY(gemm<T>(m, KC_GEMM_QKV, xn, &m->map_xn, mxl, lw.w_qkv, M, EpiStore<T, false>{qkv, lw.b_qkv, 3 * d, qkv_lo}));
+    if constexpr (sizeof(T) == 2) {
+      const CUtensorMap* sm = m->store_maps;
+      TF_TRY(gemm<T>(m, KC_GEMM_QKV, xn, &m->map_xn, mxl, lw.w_qkv, M,
+                     EpiStoreTma<false>{lw.b_qkv, sm + tf_model::SM_QKV, hp ? sm + tf_model::SM_QKV_LO : nullptr}));
+    } else {
+      TF_TRY(gemm<T>(m, KC_GEMM_QKV, xn, &m->map_xn, mxl, lw.w_qkv, M, EpiStore<T, false>{qkv, lw.b_qkv, 3 * d, qkv_lo}));
+    }
     if constexpr (sizeof(T) == 2) {
       dim3 grid((L + attn::BQ - 1) / attn::BQ, m->cfg.n_heads, n_slots);
       const float sl2 = 1.4426950408889634f / sqrtf((float)m->hd);
@@ -331,10 +356,20 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
              1.0f / sqrtf((float)m->hd));
     }
     TF_TRY(check_launch("attention kernel"));
-    TF_TRY(gemm<T>(m, KC_GEMM_O, att, &m->map_att, mal, lw.w_o, M, EpiResid{m->h, lw.b_o, d}));
+    if constexpr (sizeof(T) == 2)
+      TF_TRY(gemm<T>(m, KC_GEMM_O, att, &m->map_att, mal, lw.w_o, M, EpiResidTma{lw.b_o, m->store_maps + tf_model::SM_H}));
+    else
+      TF_TRY(gemm<T>(m, KC_GEMM_O, att, &m->map_att, mal, lw.w_o, M, EpiResid{m->h, lw.b_o, d}));
     TF_TRY(layernorm<T>(m, KC_LN, m->h, lw.ln2_g, lw.ln2_b, xn, xn_lo, M));
-    TF_TRY(gemm<T>(m, KC_GEMM_MLP1, xn, &m->map_xn, mxl, lw.w_1, M, EpiStore<T, true>{mlp, lw.b_1, m->hid, mlp_lo}));
-    TF_TRY(gemm<T>(m, KC_GEMM_MLP2, mlp, &m->map_mlp, mml, lw.w_2, M, EpiResid{m->h, lw.b_2, d}));
+    if constexpr (sizeof(T) == 2) {
+      const CUtensorMap* sm = m->store_maps;
+      TF_TRY(gemm<T>(m, KC_GEMM_MLP1, xn, &m->map_xn, mxl, lw.w_1, M,
+                     EpiStoreTma<true>{lw.b_1, sm + tf_model::SM_MLP, hp ? sm + tf_model::SM_MLP_LO : nullptr}));
+      TF_TRY(gemm<T>(m, KC_GEMM_MLP2, mlp, &m->map_mlp, mml, lw.w_2, M, EpiResidTma{lw.b_2, sm + tf_model::SM_H}));
+    } else {
+      TF_TRY(gemm<T>(m, KC_GEMM_MLP1, xn, &m->map_xn, mxl, lw.w_1, M, EpiStore<T, true>{mlp, lw.b_1, m->hid, mlp_lo}));
+      TF_TRY(gemm<T>(m, KC_GEMM_MLP2, mlp, &m->map_mlp, mml, lw.w_2, M, EpiResid{m->h, lw.b_2, d}));
+    }
   }
   TF_TRY(layernorm<T>(m, KC_LN, m->h, bw.lnf_g, bw.lnf_b, xn, xn_lo, M));
   if (mode == PASS_JACOBI) {
@@ -862,6 +897,16 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     TF_TRY(make_map_bf16(&m->map_xn_lo, m->xn_lo, M, d, tc::BM));
     TF_TRY(make_map_bf16(&m->map_att_lo, m->att_lo, M, d, tc::BM));
     TF_TRY(make_map_bf16(&m->map_mlp_lo, m->mlp_lo, M, hid, tc::BM));
+    {
+      CUtensorMap sm[tf_model::SM_COUNT];
+      TF_TRY(make_map_store(&sm[tf_model::SM_QKV], m->qkv, M, 3 * d, 2));
+      TF_TRY(make_map_store(&sm[tf_model::SM_QKV_LO], m->qkv_lo, M, 3 * d, 2));
+      TF_TRY(make_map_store(&sm[tf_model::SM_MLP], m->mlp, M, hid, 2));
+      TF_TRY(make_map_store(&sm[tf_model::SM_MLP_LO], m->mlp_lo, M, hid, 2));
+      TF_TRY(make_map_store(&sm[tf_model::SM_H], m->h, M, d, 4));
+      TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->store_maps), sizeof(sm)));
+      CU_OK(cudaMemcpy(m->store_maps, sm, sizeof(sm), cudaMemcpyHostToDevice));
+    }
     for (int r = 0; r < 3; ++r) {
       const uint32_t rt = 16u << r;
       TF_TRY(make_map_bf16(&m->map_seq_a[0][r], m->xn, M, d, rt));
