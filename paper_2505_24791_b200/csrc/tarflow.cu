@@ -21,6 +21,7 @@
 #include "common.cuh"
 #include "epilogue.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_tc2.cuh"
 #include "kernels_simt.cuh"
 #include "seq_decode.cuh"
 
@@ -140,6 +141,7 @@ struct tf_model {
   enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_COUNT };
   CUtensorMap* store_maps = nullptr;  // device copy of the bulk-store maps of qkv, qkv_lo, mlp, mlp_lo, h
   CUtensorMap map_seq_a[3][3];  // sequential-step GEMM operands {xn, att, mlp} x row tile {16, 32, 64}
+  bool use_pair_gemm = true;    // sweep GEMMs on 2-CTA tile pairs (false: one CTA per tile)
   bool seq_use_tc = true;       // sequential-step GEMMs on tcgen05 (false: the mma.sync kernel)
   int *idx = nullptr, *idx_tmp = nullptr, *phase = nullptr, *ctrl = nullptr, *iters_sample = nullptr, *err = nullptr;
   // precision policy of Jacobi blocks on the bf16 engine: 0 = escalate per sample, 1 = single bf16
@@ -269,6 +271,38 @@ static int launch_gemm_tc(tf_model* m, int cls, cudaStream_t stream, const CUten
   return check_launch("gemm_tc_kernel");
 }
 
+// pair kernel: 256 x 256 tiles on clusters of two CTAs (N % 256 == 0, bulk-store epilogues)
+template <class Epi>
+static int launch_gemm_tc2(tf_model* m, int cls, const CUtensorMap& ma, const CUtensorMap* ma_lo, const CUtensorMap& mw, int M,
+                           int N, int K, const Epi& epi) {
+  auto kern = tc2::gemm_tc2_kernel<Epi>;
+  static bool configured = false;  // per instantiation
+  if (!configured) {
+    CU_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::Smem2::TOTAL));
+    configured = true;
+  }
+  const int tiles = ((M + 2 * tc::BM - 1) / (2 * tc::BM)) * (N / tc2::BN2);
+  int pairs = m->num_sms / 2;
+  if (tiles < pairs) pairs = tiles;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(2 * pairs);
+  lc.blockDim = dim3(tc::NUM_THREADS);
+  lc.dynamicSmemBytes = tc2::Smem2::TOTAL;
+  lc.stream = m->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 2;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  m->pre(cls);
+  cudaError_t e = cudaLaunchKernelEx(&lc, kern, ma, ma_lo ? *ma_lo : ma, mw, M, N, K, ma_lo ? 1 : 0, epi, m->err);
+  m->post(cls);
+  if (e != cudaSuccess) return fail(TF_ECUDA, "gemm_tc2_kernel launch failed: %s", cudaGetErrorString(e));
+  return TF_OK;
+}
+
 template <class T, class Epi>
 static int launch_gemm_simt(tf_model* m, int cls, const T* A, const Matrix& W, int M, const Epi& epi) {
   dim3 grid((W.N + 63) / 64, (M + 63) / 64);
@@ -282,6 +316,10 @@ template <class T, class Epi>
 static int gemm(tf_model* m, int cls, const T* A, const CUtensorMap* map_a, const CUtensorMap* map_a_lo,
                 const Matrix& W, int M, const Epi& epi) {
   if constexpr (sizeof(T) == 2) {
+    if constexpr (Epi::kTmaCols > 0) {
+      if (m->use_pair_gemm && W.N % 256 == 0 && M >= 256)
+        return launch_gemm_tc2<Epi>(m, cls, *map_a, map_a_lo, W.map_seq, M, W.N, W.K, epi);
+    }
     if (W.bn == 256)
       return launch_gemm_tc<256, 4, Epi>(m, cls, m->stream, *map_a, map_a_lo, W.map, M, W.N, W.K, epi, m->err,
                                          m->num_sms, nullptr);
@@ -917,6 +955,7 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<32>()));
     CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<64>()));
     if (const char* e = getenv("TARFLOW_SEQ_MMA")) m->seq_use_tc = atoi(e) == 0;
+    if (const char* e = getenv("TARFLOW_PAIR_GEMM")) m->use_pair_gemm = atoi(e) != 0;
     CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                attn::smem_bytes<true>()));
     CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
