@@ -18,6 +18,7 @@
 
 #include "../../include/tarflow.h"
 #include "attention_mma.cuh"
+#include "attention_tc.cuh"
 #include "common.cuh"
 #include "epilogue.cuh"
 #include "gemm_tc.cuh"
@@ -97,6 +98,23 @@ static int make_map_store(CUtensorMap* map, const void* ptr, uint64_t rows, uint
   return TF_OK;
 }
 
+// bf16 tensor [slots][L][cols] seen as 3-D, box = 64 columns x box_rows positions of one slot, 128-byte swizzle:
+// positions >= L read as zeros and are not written, whatever L is.
+static int make_map_3d(CUtensorMap* map, const void* ptr, uint64_t slots, uint64_t L, uint64_t cols, uint32_t box_rows) {
+  encode_tiled_fn fn = get_encode_fn();
+  if (!fn) return fail(TF_ECUDA, "cuTensorMapEncodeTiled entry point not available");
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || (cols * 2) % 16) return fail(TF_EINVAL, "TMA operand not 16-byte aligned");
+  cuuint64_t dims[3] = {cols, L, slots};
+  cuuint64_t strides[2] = {cols * 2, L * cols * 2};
+  cuuint32_t box[3] = {64, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(TF_ECUDA, "cuTensorMapEncodeTiled (3-D map) failed (%d)", (int)r);
+  return TF_OK;
+}
+
 // ------------------------------------------------------------------------------------------------
 // model
 // ------------------------------------------------------------------------------------------------
@@ -138,7 +156,9 @@ struct tf_model {
   void *xn = nullptr, *qkv = nullptr, *att = nullptr, *mlp = nullptr, *kcache = nullptr, *vcache = nullptr;
   void *xn_lo = nullptr, *qkv_lo = nullptr, *att_lo = nullptr, *mlp_lo = nullptr;  // second terms (bf16 engine)
   CUtensorMap map_xn, map_att, map_mlp, map_xn_lo, map_att_lo, map_mlp_lo;
-  enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_COUNT };
+  enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_ATT3, SM_COUNT };
+  CUtensorMap map_qkv3;        // qkv as [slot][position][3d] for the tensor-core attention
+  bool use_tc_attention = false;  // measured slower than the mma.sync kernel so far: opt-in (TARFLOW_ATTN_TC=1)
   CUtensorMap* store_maps = nullptr;  // device copy of the bulk-store maps of qkv, qkv_lo, mlp, mlp_lo, h
   CUtensorMap map_seq_a[3][3];  // sequential-step GEMM operands {xn, att, mlp} x row tile {16, 32, 64}
   bool use_pair_gemm = true;    // sweep GEMMs on 2-CTA tile pairs (false: one CTA per tile)
@@ -383,6 +403,9 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
       if (hp)
         LAUNCH(m, KC_ATTN, attn::attention_mma_kernel<true>, grid, 128, attn::smem_bytes<true>(), qkv, qkv_lo, att,
                att_lo, L, d, sl2);
+      else if (m->use_tc_attention)
+        LAUNCH(m, KC_ATTN, attn_tc::attention_tc_kernel, dim3((L + attn_tc::BQ - 1) / attn_tc::BQ, m->cfg.n_heads, n_slots),
+               attn_tc::NUM_THREADS_ATTN, attn_tc::SMEM_BYTES, m->map_qkv3, m->store_maps + tf_model::SM_ATT3, L, d, sl2, m->err);
       else
         LAUNCH(m, KC_ATTN, attn::attention_mma_kernel<false>, grid, 128, attn::smem_bytes<false>(), qkv, qkv_lo, att,
                att_lo, L, d, sl2);
@@ -942,6 +965,10 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
       TF_TRY(make_map_store(&sm[tf_model::SM_MLP], m->mlp, M, hid, 2));
       TF_TRY(make_map_store(&sm[tf_model::SM_MLP_LO], m->mlp_lo, M, hid, 2));
       TF_TRY(make_map_store(&sm[tf_model::SM_H], m->h, M, d, 4));
+      TF_TRY(make_map_3d(&sm[tf_model::SM_ATT3], m->att, B, L, d, 32));
+      TF_TRY(make_map_3d(&m->map_qkv3, m->qkv, B, L, 3 * (uint64_t)d, 128));
+      CU_OK(cudaFuncSetAttribute(attn_tc::attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_tc::SMEM_BYTES));
+      if (const char* e = getenv("TARFLOW_ATTN_TC")) m->use_tc_attention = atoi(e) != 0;
       TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->store_maps), sizeof(sm)));
       CU_OK(cudaMemcpy(m->store_maps, sm, sizeof(sm), cudaMemcpyHostToDevice));
     }

@@ -228,3 +228,23 @@ def test_bf16_ragged_sequence_length_and_classes():
     lab = synth.make_labels(cfg, B=3)
     m, x, xo, its, ito, rc = _bf16_case(cfg, 3, 5, [0, 1], 1e-3, labels=lab)
     assert rc == 0 and rel_l2(x, xo) <= BF16_REL_L2 and np.abs(its - ito).max() <= 1
+
+
+def test_bf16_optional_kernel_paths_agree(monkeypatch):
+    """The opt-in tcgen05 attention and the one-CTA-per-tile GEMM give the same sweep as the default kernels."""
+    cfg = synth.config("cfg2", n_blocks=1, n_layers=2)
+    z = synth.make_latents(cfg, 17, B=3)
+    outs = {}
+    for name, env in (("default", {}), ("attn_tc", {"TARFLOW_ATTN_TC": "1"}), ("single_cta", {"TARFLOW_PAIR_GEMM": "0"})):
+        for k in ("TARFLOW_ATTN_TC", "TARFLOW_PAIR_GEMM"):
+            monkeypatch.delenv(k, raising=False)
+        for k, v in env.items():
+            monkeypatch.setenv(k, v)
+        with Model(cfg, max_batch=3) as m:      # the switches are read when the model is loaded
+            outs[name], _, _, rc = m.inverse(z, None, [1], -1.0, 3)
+            assert rc == 0 and np.isfinite(outs[name]).all()
+    xo, _ = O.model_inverse(synth.make_weights(cfg), z, None, cfg, [1], -1.0, 3)
+    for name, x in outs.items():
+        assert rel_l2(x, xo) <= BF16_REL_L2, name
+    assert rel_l2(outs["attn_tc"], outs["default"]) <= 5e-3
+    assert rel_l2(outs["single_cta"], outs["default"]) <= 1e-4
