@@ -1,19 +1,20 @@
 // Causal self-attention on the 5th-generation tensor cores (head_dim 64, single bf16 operands).
 //
-// One CTA = one (slot, head, tile of 128 queries); key/value tiles of 128 keys 0 .. query tile (causal).
+// One CTA = one (slot, head, tile of 128 queries); key/value tiles of 64 keys from 0 up to the query tile (causal).
 // Per key tile j:
-//   S  = Q K_j^T                 tcgen05.mma M=128 N=128 K=64, both operands K-major from TMA tiles, S in TMEM
+//   S  = Q K_j^T                 tcgen05.mma M=128 N=64 K=64, both operands K-major from TMA tiles, S in TMEM
 //   softmax                      4 warps, one query row per thread (TMEM lane = row, so row maximum and row sum
 //                                need no shuffles): running maximum / sum in fp32, P_j = exp2(S - m) written as
 //                                bf16 into a swizzled shared-memory tile (the A operand of the second MMA)
-//   O_j = P_j V_j                tcgen05.mma M=128 N=64 K=128; V_j is used as it arrives from TMA ([key][channel],
+//   O_j = P_j V_j                tcgen05.mma M=128 N=64 K=64; V_j is used as it arrives from TMA ([key][channel],
 //                                i.e. an MN-major B operand), no transposition anywhere
 //   o += O_j (rescaled)          the running output stays in registers of the row's thread
 // K and V each have one buffer: K_{j+1} is loaded as soon as the first MMA of tile j has completed, V_{j+1} after
 // the second, so loads overlap the softmax; two CTAs fit on an SM and fill each other's bubbles.
 // Rows are addressed through 3-D tensor maps [slot][position][column], so positions >= L read as zeros and are
 // never written (ragged L).  Every mbarrier wait is bounded as in gemm_tc.cuh.
-// qkv rows are [q | k | v] (3d wide); out is [slot, L, d] bf16.
+// qkv rows are [q | k | v] (3d wide); out is [slot, L, d] bf16.  map_qkv has a box of 128 positions (queries),
+// map_kv one of 64 positions (keys / values), both 64 columns wide.
 #pragma once
 #include "gemm_tc.cuh"
 
@@ -21,11 +22,11 @@ namespace attn_tc {
 
 using namespace tc;
 
-constexpr int BQ = 128, BKV = 128, HD = 64;
+constexpr int BQ = 128, BKV = 64, HD = 64;
 constexpr int NUM_THREADS_ATTN = 192;  // warp 0 TMA, warp 1 MMA + TMEM, warps 2..5 softmax / epilogue
 constexpr int Q_BYTES = BQ * HD * 2, K_BYTES = BKV * HD * 2, V_BYTES = BKV * HD * 2, P_BYTES = BQ * BKV * 2;
 constexpr int SMEM_BYTES = Q_BYTES + K_BYTES + V_BYTES + P_BYTES + 128 + 1024;
-constexpr uint32_t TMEM_COLS_ATTN = 256;  // S: columns 0..127, O_j: columns 128..191
+constexpr uint32_t TMEM_COLS_ATTN = 128;  // S: columns 0..63, O_j: columns 64..127
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
   asm volatile(
@@ -55,7 +56,8 @@ __host__ __device__ constexpr uint32_t make_idesc_attn(int m, int n, int b_mn) {
 }
 
 __global__ void __launch_bounds__(NUM_THREADS_ATTN, 2)
-attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const CUtensorMap* __restrict__ map_out, int L, int d,
+attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_kv,
+                    const CUtensorMap* __restrict__ map_out, int L, int d,
                     float scale_log2e, int* err) {
   extern __shared__ uint8_t smem_attn_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_attn_raw) + 1023) & ~(uintptr_t)1023);
@@ -68,7 +70,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const CUtensorM
   const int n_qt = (L + BQ - 1) / BQ;
   const int qt = n_qt - 1 - (int)blockIdx.x;  // longest tiles first
   const int head = blockIdx.y, slot = blockIdx.z;
-  const int q0 = qt * BQ, n_kv = qt + 1;
+  const int q0 = qt * BQ;
+  const int n_kv = ((q0 + BQ < L ? q0 + BQ : L) + BKV - 1) / BKV;  // key tiles that hold a visible key
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 4 : 1);
@@ -96,10 +99,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const CUtensorM
         const uint32_t ph = j & 1;
         if (!mbar_wait(bar(2), ph ^ 1u, err, TFERR_WAIT_EMPTY)) { ok = false; break; }
         mbar_arrive_expect_tx(bar(1), K_BYTES);
-        tma_load_3d(sK, &map_qkv, d + head * HD, j * BKV, slot, bar(1));
+        tma_load_3d(sK, &map_kv, d + head * HD, j * BKV, slot, bar(1));
         if (!mbar_wait(bar(4), ph ^ 1u, err, TFERR_WAIT_EMPTY)) { ok = false; break; }
         mbar_arrive_expect_tx(bar(3), V_BYTES);
-        tma_load_3d(sV, &map_qkv, 2 * d + head * HD, j * BKV, slot, bar(3));
+        tma_load_3d(sV, &map_kv, 2 * d + head * HD, j * BKV, slot, bar(3));
       }
     }
   } else if (warp == 1) {
@@ -121,8 +124,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const CUtensorM
         tcgen05_fence_after();
 #pragma unroll
         for (int k = 0; k < BKV / UMMA_K; ++k) {
-          // P: two 64-key halves of [128 rows][128 B]; 16 keys = 32 bytes inside a half.  V: 16 keys = 2048 bytes.
-          const uint64_t pdesc = make_smem_desc(sP + (k >> 2) * (BQ * 128)) + 2u * (k & 3);
+          // P: [128 rows][128 B] (64 keys), 16 keys = 32 bytes along a row.  V: 16 keys = 2048 bytes.
+          const uint64_t pdesc = make_smem_desc(sP) + 2u * k;
           const uint64_t vdesc = make_smem_desc_mn(sV + k * (UMMA_K * 128));
           umma_f16(tmem_base + BKV, pdesc, vdesc, idesc_o, k != 0);
         }
@@ -146,19 +149,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const CUtensorM
       const uint32_t ph = j & 1;
       if (!mbar_wait(bar(5), ph, err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
       tcgen05_fence_after();
-      const bool diag = (j == n_kv - 1);
       const int kv0 = j * BKV;
-      // pass 1: row maximum
+      const bool diag = kv0 + BKV - 1 > q0;  // some key of this tile lies after some query of the tile
+      // the whole score row in one round of tensor-memory loads
+      float s[BKV];
+      tmem_ld_32x32b_x32_issue(t_row, *reinterpret_cast<float(*)[32]>(&s[0]));
+      tmem_ld_32x32b_x32_issue(t_row + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
+      tmem_ld_wait();
       float mx = -INFINITY;
-#pragma unroll 1
-      for (int c = 0; c < BKV / 32; ++c) {
-        float s[32];
-        tmem_ld_32x32b_x32(t_row + c * 32, s);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const bool masked = diag && (kv0 + c * 32 + i > qpos);
-          mx = masked ? mx : fmaxf(mx, s[i]);
-        }
+      for (int i = 0; i < BKV; ++i) {
+        if (diag && kv0 + i > qpos) s[i] = -INFINITY;
+        mx = fmaxf(mx, s[i]);
       }
       const float m_new = fmaxf(m_run, mx);  // finite from the first tile on: key 0 is visible to every row
       const float corr = exp2f((m_run - m_new) * scale_log2e);
@@ -167,38 +169,29 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const CUtensorM
       if (j > 0) {
         if (!mbar_wait(bar(7), ph ^ 1u, err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
         tcgen05_fence_after();
+        float t[HD];
+        tmem_ld_32x32b_x32_issue(t_row + BKV, *reinterpret_cast<float(*)[32]>(&t[0]));
+        tmem_ld_32x32b_x32_issue(t_row + BKV + 32, *reinterpret_cast<float(*)[32]>(&t[32]));
+        tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < HD / 32; ++c) {
-          float t[32];
-          tmem_ld_32x32b_x32(t_row + BKV + c * 32, t);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o[c * 32 + i] += t[i];
-        }
+        for (int i = 0; i < HD; ++i) o[i] = (o[i] + t[i]) * corr;
       }
-#pragma unroll
-      for (int i = 0; i < HD; ++i) o[i] *= corr;
       l_run *= corr;
-      // pass 2: probabilities -> bf16 P tile (swizzled rows of 128 bytes, two 64-key halves)
-#pragma unroll 1
-      for (int c = 0; c < BKV / 32; ++c) {
-        float s[32];
-        tmem_ld_32x32b_x32(t_row + c * 32, s);
-        uint32_t pk[16];
+      // probabilities -> bf16 P tile (swizzled rows of 128 bytes)
+      const float mb = m_new * scale_log2e;
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const bool m0 = diag && (kv0 + c * 32 + i > qpos), m1 = diag && (kv0 + c * 32 + i + 1 > qpos);
-          const float p0 = m0 ? 0.f : exp2f((s[i] - m_new) * scale_log2e);
-          const float p1 = m1 ? 0.f : exp2f((s[i + 1] - m_new) * scale_log2e);
+      for (int q = 0; q < 8; ++q) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float p0 = exp2f(fmaf(s[8 * q + 2 * i], scale_log2e, -mb));      // exp2(-inf) = 0 for masked keys
+          const float p1 = exp2f(fmaf(s[8 * q + 2 * i + 1], scale_log2e, -mb));
           const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-          // the sum uses the rounded probabilities that the second MMA will see
-          const float2 pf = __bfloat1622float2(pb);
+          const float2 pf = __bfloat1622float2(pb);  // the sum uses the rounded probabilities the second MMA sees
           l_run += pf.x + pf.y;
-          pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+          pk[i] = *reinterpret_cast<const uint32_t*>(&pb);
         }
-        uint8_t* half = sPg + (c >> 1) * (BQ * 128);
-#pragma unroll
-        for (int q = 0; q < 4; ++q)  // 16-byte piece (c & 1) * 4 + q of this row's 128 bytes in the half
-          *reinterpret_cast<uint4*>(half + swz128(r, (c & 1) * 4 + q)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+        *reinterpret_cast<uint4*>(sPg + swz128(r, q)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }
       fence_proxy_async_smem();
       tcgen05_fence_before();
@@ -209,13 +202,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const CUtensorM
     // which nobody reads any more)
     if (ok && mbar_wait(bar(7), (uint32_t)((n_kv - 1) & 1), err, TFERR_WAIT_TMEM_FULL)) {
       tcgen05_fence_after();
+      float t[HD];
+      tmem_ld_32x32b_x32_issue(t_row + BKV, *reinterpret_cast<float(*)[32]>(&t[0]));
+      tmem_ld_32x32b_x32_issue(t_row + BKV + 32, *reinterpret_cast<float(*)[32]>(&t[32]));
+      tmem_ld_wait();
 #pragma unroll
-      for (int c = 0; c < HD / 32; ++c) {
-        float t[32];
-        tmem_ld_32x32b_x32(t_row + BKV + c * 32, t);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o[c * 32 + i] += t[i];
-      }
+      for (int i = 0; i < HD; ++i) o[i] += t[i];
       const float inv = 1.f / l_run;
       uint8_t* box = sPg + quad * 4096;
 #pragma unroll

@@ -157,7 +157,7 @@ struct tf_model {
   void *xn_lo = nullptr, *qkv_lo = nullptr, *att_lo = nullptr, *mlp_lo = nullptr;  // second terms (bf16 engine)
   CUtensorMap map_xn, map_att, map_mlp, map_xn_lo, map_att_lo, map_mlp_lo;
   enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_ATT3, SM_COUNT };
-  CUtensorMap map_qkv3;        // qkv as [slot][position][3d] for the tensor-core attention
+  CUtensorMap map_qkv3, map_kv3;  // qkv as [slot][position][3d] for the tensor-core attention (query / key boxes)
   bool use_tc_attention = false;  // measured slower than the mma.sync kernel so far: opt-in (TARFLOW_ATTN_TC=1)
   CUtensorMap* store_maps = nullptr;  // device copy of the bulk-store maps of qkv, qkv_lo, mlp, mlp_lo, h
   CUtensorMap map_seq_a[3][3];  // sequential-step GEMM operands {xn, att, mlp} x row tile {16, 32, 64}
@@ -405,7 +405,8 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
                att_lo, L, d, sl2);
       else if (m->use_tc_attention)
         LAUNCH(m, KC_ATTN, attn_tc::attention_tc_kernel, dim3((L + attn_tc::BQ - 1) / attn_tc::BQ, m->cfg.n_heads, n_slots),
-               attn_tc::NUM_THREADS_ATTN, attn_tc::SMEM_BYTES, m->map_qkv3, m->store_maps + tf_model::SM_ATT3, L, d, sl2, m->err);
+               attn_tc::NUM_THREADS_ATTN, attn_tc::SMEM_BYTES, m->map_qkv3, m->map_kv3, m->store_maps + tf_model::SM_ATT3, L, d, sl2,
+               m->err);
       else
         LAUNCH(m, KC_ATTN, attn::attention_mma_kernel<false>, grid, 128, attn::smem_bytes<false>(), qkv, qkv_lo, att,
                att_lo, L, d, sl2);
@@ -966,7 +967,8 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
       TF_TRY(make_map_store(&sm[tf_model::SM_MLP_LO], m->mlp_lo, M, hid, 2));
       TF_TRY(make_map_store(&sm[tf_model::SM_H], m->h, M, d, 4));
       TF_TRY(make_map_3d(&sm[tf_model::SM_ATT3], m->att, B, L, d, 32));
-      TF_TRY(make_map_3d(&m->map_qkv3, m->qkv, B, L, 3 * (uint64_t)d, 128));
+      TF_TRY(make_map_3d(&m->map_qkv3, m->qkv, B, L, 3 * (uint64_t)d, attn_tc::BQ));
+      TF_TRY(make_map_3d(&m->map_kv3, m->qkv, B, L, 3 * (uint64_t)d, attn_tc::BKV));
       CU_OK(cudaFuncSetAttribute(attn_tc::attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_tc::SMEM_BYTES));
       if (const char* e = getenv("TARFLOW_ATTN_TC")) m->use_tc_attention = atoi(e) != 0;
       TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->store_maps), sizeof(sm)));
