@@ -6,11 +6,14 @@
 //   softmax                      4 warps, one query row per thread (TMEM lane = row, so row maximum and row sum
 //                                need no shuffles): running maximum / sum in fp32, P_j = exp2(S - m) written as
 //                                bf16 into a swizzled shared-memory tile (the A operand of the second MMA)
-//   O_j = P_j V_j                tcgen05.mma M=128 N=64 K=64; V_j is used as it arrives from TMA ([key][channel],
-//                                i.e. an MN-major B operand), no transposition anywhere
-//   o += O_j (rescaled)          the running output stays in registers of the row's thread
-// K and V each have one buffer: K_{j+1} is loaded as soon as the first MMA of tile j has completed, V_{j+1} after
-// the second, so loads overlap the softmax; two CTAs fit on an SM and fill each other's bubbles.
+//   O += P_j V_j                 tcgen05.mma M=128 N=64 K=64, accumulating in TMEM over the key tiles; V_j is used as
+//                                it arrives from TMA ([key][channel], i.e. an MN-major B operand), no transposition
+//   rescale (rare)               the reference maximum of a row moves only when the true maximum has grown by more
+//                                than 2^8; only then is the accumulator read, scaled and written back
+// S and P are double-buffered, so the first MMA of tile j+1 is issued before the softmax of tile j has
+// finished and the tensor core never waits for the softmax warps of its own CTA (and vice versa, apart from
+// true data dependences two tiles back).  K and V tiles travel through rings of three buffers each, so the TMA
+// round trip of a tile is hidden behind the two tiles before it.  Two CTAs fit on an SM.
 // Rows are addressed through 3-D tensor maps [slot][position][column], so positions >= L read as zeros and are
 // never written (ragged L).  Every mbarrier wait is bounded as in gemm_tc.cuh.
 // qkv rows are [q | k | v] (3d wide); out is [slot, L, d] bf16.  map_qkv has a box of 128 positions (queries),
@@ -25,8 +28,10 @@ using namespace tc;
 constexpr int BQ = 128, BKV = 64, HD = 64;
 constexpr int NUM_THREADS_ATTN = 192;  // warp 0 TMA, warp 1 MMA + TMEM, warps 2..5 softmax / epilogue
 constexpr int Q_BYTES = BQ * HD * 2, K_BYTES = BKV * HD * 2, V_BYTES = BKV * HD * 2, P_BYTES = BQ * BKV * 2;
-constexpr int SMEM_BYTES = Q_BYTES + K_BYTES + V_BYTES + P_BYTES + 128 + 1024;
-constexpr uint32_t TMEM_COLS_ATTN = 128;  // S: columns 0..63, O_j: columns 64..127
+constexpr int KV_STAGES = 3;  // K and V tiles in flight ahead of the tensor core
+constexpr int KV_RING = KV_STAGES * (K_BYTES + V_BYTES);
+constexpr int SMEM_BYTES = Q_BYTES + KV_RING + 2 * P_BYTES + 256 + 1024;  // P is double-buffered
+constexpr uint32_t TMEM_COLS_ATTN = 256;  // S buffers at columns 0 and 64, the output accumulator at column 128
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
   asm volatile(
@@ -39,6 +44,49 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, int x, int 
                "r"(z), "r"(src)
                : "memory");
 }
+// Packed fp32 arithmetic (two lanes per instruction), three-input maximum and the bare exp2 unit.
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;"
+      : "=l"(d)
+      : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)),
+        "l"(*reinterpret_cast<unsigned long long*>(&c)));
+  return *reinterpret_cast<float2*>(&d);
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;"
+      : "=l"(d)
+      : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
+  return *reinterpret_cast<float2*>(&d);
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float ex2_approx(float a) {
+  float d;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(d) : "f"(a));
+  return d;
+}
+__device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const float (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])),
+        "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])),
+        "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])),
+        "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])),
+        "r"(__float_as_uint(v[31]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // MN-major B operand tile [keys][64 channels] with 128-byte rows and 128-byte swizzle (what TMA delivers for V):
 // 8 keys x 128 bytes per swizzle atom, atoms 1024 bytes apart along the key (K) direction.
 __device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t saddr) {
@@ -61,11 +109,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
                     float scale_log2e, int* err) {
   extern __shared__ uint8_t smem_attn_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_attn_raw) + 1023) & ~(uintptr_t)1023);
-  const uint32_t sQ = smem_u32(smem), sK = sQ + Q_BYTES, sV = sK + K_BYTES, sP = sV + V_BYTES;
-  const uint32_t bar_base = sP + P_BYTES;
-  // barriers: 0 q_full, 1 k_full, 2 k_empty, 3 v_full, 4 v_empty, 5 s_full, 6 p_ready, 7 o_done
+  const uint32_t sQ = smem_u32(smem), sK = sQ + Q_BYTES, sV = sK + KV_STAGES * K_BYTES, sP = sV + KV_STAGES * V_BYTES;
+  const uint32_t bar_base = sP + 2 * P_BYTES;
+  // barriers: 0 q_full, then k_full[st], k_empty[st], v_full[st], v_empty[st], s_full[2], p_ready[2], o_done[2]
+  constexpr int B_KFULL = 1, B_KEMPTY = B_KFULL + KV_STAGES, B_VFULL = B_KEMPTY + KV_STAGES, B_VEMPTY = B_VFULL + KV_STAGES,
+                B_SFULL = B_VEMPTY + KV_STAGES, B_PREADY = B_SFULL + 2, B_ODONE = B_PREADY + 2, NUM_BARS = B_ODONE + 2;
+  static_assert(NUM_BARS * 8 <= 192, "barrier area");
   auto bar = [&](int i) { return bar_base + 8u * i; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + Q_BYTES + K_BYTES + V_BYTES + P_BYTES + 64);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + Q_BYTES + KV_RING + 2 * P_BYTES + 192);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_qt = (L + BQ - 1) / BQ;
   const int qt = n_qt - 1 - (int)blockIdx.x;  // longest tiles first
@@ -74,7 +125,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
   const int n_kv = ((q0 + BQ < L ? q0 + BQ : L) + BKV - 1) / BKV;  // key tiles that hold a visible key
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 4 : 1);
+    for (int i = 0; i < NUM_BARS; ++i) mbar_init(bar(i), (i == B_PREADY || i == B_PREADY + 1) ? 4 : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -95,14 +146,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
       mbar_arrive_expect_tx(bar(0), Q_BYTES);
       tma_load_3d(sQ, &map_qkv, head * HD, q0, slot, bar(0));
       bool ok = true;
+      int st = 0;
+      uint32_t ph = 0;
       for (int j = 0; j < n_kv && ok; ++j) {
-        const uint32_t ph = j & 1;
-        if (!mbar_wait(bar(2), ph ^ 1u, err, TFERR_WAIT_EMPTY)) { ok = false; break; }
-        mbar_arrive_expect_tx(bar(1), K_BYTES);
-        tma_load_3d(sK, &map_kv, d + head * HD, j * BKV, slot, bar(1));
-        if (!mbar_wait(bar(4), ph ^ 1u, err, TFERR_WAIT_EMPTY)) { ok = false; break; }
-        mbar_arrive_expect_tx(bar(3), V_BYTES);
-        tma_load_3d(sV, &map_kv, 2 * d + head * HD, j * BKV, slot, bar(3));
+        if (!mbar_wait(bar(B_KEMPTY + st), ph ^ 1u, err, TFERR_WAIT_EMPTY)) { ok = false; break; }
+        mbar_arrive_expect_tx(bar(B_KFULL + st), K_BYTES);
+        tma_load_3d(sK + st * K_BYTES, &map_kv, d + head * HD, j * BKV, slot, bar(B_KFULL + st));
+        if (!mbar_wait(bar(B_VEMPTY + st), ph ^ 1u, err, TFERR_WAIT_EMPTY)) { ok = false; break; }
+        mbar_arrive_expect_tx(bar(B_VFULL + st), V_BYTES);
+        tma_load_3d(sV + st * V_BYTES, &map_kv, 2 * d + head * HD, j * BKV, slot, bar(B_VFULL + st));
+        if (++st == KV_STAGES) { st = 0; ph ^= 1u; }
       }
     }
   } else if (warp == 1) {
@@ -110,27 +163,36 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
     if (lane == 0 && !dead) {
       constexpr uint32_t idesc_s = make_idesc_attn(BQ, BKV, 0), idesc_o = make_idesc_attn(BQ, HD, 1);
       bool ok = mbar_wait(bar(0), 0u, err, TFERR_WAIT_FULL);
-      for (int j = 0; j < n_kv && ok; ++j) {
-        const uint32_t ph = j & 1;
-        if (!mbar_wait(bar(1), ph, err, TFERR_WAIT_FULL)) { ok = false; break; }
+      const uint64_t qdesc = make_smem_desc(sQ);
+      auto scores = [&](int j) {  // S[j & 1] = Q K_j^T
+        const int st = j % KV_STAGES;
+        if (!mbar_wait(bar(B_KFULL + st), (uint32_t)((j / KV_STAGES) & 1), err, TFERR_WAIT_FULL)) return false;
         tcgen05_fence_after();
-        const uint64_t qdesc = make_smem_desc(sQ), kdesc = make_smem_desc(sK);
+        const uint64_t kdesc = make_smem_desc(sK + st * K_BYTES);
 #pragma unroll
-        for (int k = 0; k < HD / UMMA_K; ++k) umma_f16(tmem_base, qdesc + 2u * k, kdesc + 2u * k, idesc_s, k != 0);
-        umma_commit(bar(2));  // K buffer free
-        umma_commit(bar(5));  // S complete
-        if (!mbar_wait(bar(6), ph, err, TFERR_WAIT_TMEM_EMPTY)) { ok = false; break; }  // P written, O_{j-1} consumed
-        if (!mbar_wait(bar(3), ph, err, TFERR_WAIT_FULL)) { ok = false; break; }
+        for (int k = 0; k < HD / UMMA_K; ++k) umma_f16(tmem_base + (j & 1) * BKV, qdesc + 2u * k, kdesc + 2u * k, idesc_s, k != 0);
+        umma_commit(bar(B_KEMPTY + st));      // K buffer free
+        umma_commit(bar(B_SFULL + (j & 1)));  // S[j & 1] complete
+        return true;
+      };
+      if (ok) ok = scores(0);
+      for (int j = 0; j < n_kv && ok; ++j) {
+        // the next tile's scores are issued before this tile's probabilities are awaited: its S buffer was last
+        // read by the softmax of tile j-1, which had finished when p_ready of tile j-1 was seen
+        if (j + 1 < n_kv && !scores(j + 1)) { ok = false; break; }
+        const int st = j % KV_STAGES;
+        if (!mbar_wait(bar(B_PREADY + (j & 1)), (uint32_t)((j >> 1) & 1), err, TFERR_WAIT_TMEM_EMPTY)) { ok = false; break; }
+        if (!mbar_wait(bar(B_VFULL + st), (uint32_t)((j / KV_STAGES) & 1), err, TFERR_WAIT_FULL)) { ok = false; break; }
         tcgen05_fence_after();
 #pragma unroll
         for (int k = 0; k < BKV / UMMA_K; ++k) {
           // P: [128 rows][128 B] (64 keys), 16 keys = 32 bytes along a row.  V: 16 keys = 2048 bytes.
-          const uint64_t pdesc = make_smem_desc(sP) + 2u * k;
-          const uint64_t vdesc = make_smem_desc_mn(sV + k * (UMMA_K * 128));
-          umma_f16(tmem_base + BKV, pdesc, vdesc, idesc_o, k != 0);
+          const uint64_t pdesc = make_smem_desc(sP + (j & 1) * P_BYTES) + 2u * k;
+          const uint64_t vdesc = make_smem_desc_mn(sV + st * V_BYTES + k * (UMMA_K * 128));
+          umma_f16(tmem_base + 2 * BKV, pdesc, vdesc, idesc_o, (j | k) != 0);
         }
-        umma_commit(bar(4));  // V buffer (and P) free
-        umma_commit(bar(7));  // O_j complete
+        umma_commit(bar(B_VEMPTY + st));      // V buffer free
+        umma_commit(bar(B_ODONE + (j & 1)));  // products up to tile j complete (and P[j & 1] free)
       }
     }
   } else {
@@ -139,75 +201,94 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
     const int r = quad * 32 + lane;            // row of this thread inside the query tile
     const int qpos = q0 + r;                   // position in the sequence
     const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint8_t* sPg = smem + Q_BYTES + K_BYTES + V_BYTES;
-    float o[HD];
-#pragma unroll
-    for (int i = 0; i < HD; ++i) o[i] = 0.f;
+    const uint32_t t_o = t_row + 2 * BKV;      // this row's slice of the output accumulator
+    uint8_t* sPg = smem + Q_BYTES + KV_RING;
+    // m_run is the reference maximum of the row (in raw score units); it trails the true running maximum by at
+    // most kLazy / scale_log2e, so probabilities stay below 2^kLazy and the accumulator is rescaled only rarely
+    constexpr float kLazy = 8.f;
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = !dead;
     for (int j = 0; j < n_kv && ok; ++j) {
-      const uint32_t ph = j & 1;
-      if (!mbar_wait(bar(5), ph, err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
+      const uint32_t ph2 = (j >> 1) & 1;  // phase of the per-buffer barriers
+      if (!mbar_wait(bar(B_SFULL + (j & 1)), ph2, err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
       tcgen05_fence_after();
       const int kv0 = j * BKV;
       const bool diag = kv0 + BKV - 1 > q0;  // some key of this tile lies after some query of the tile
       // the whole score row in one round of tensor-memory loads
       float s[BKV];
-      tmem_ld_32x32b_x32_issue(t_row, *reinterpret_cast<float(*)[32]>(&s[0]));
-      tmem_ld_32x32b_x32_issue(t_row + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
+      tmem_ld_32x32b_x32_issue(t_row + (j & 1) * BKV, *reinterpret_cast<float(*)[32]>(&s[0]));
+      tmem_ld_32x32b_x32_issue(t_row + (j & 1) * BKV + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
       tmem_ld_wait();
-      float mx = -INFINITY;
+      if (diag) {
 #pragma unroll
-      for (int i = 0; i < BKV; ++i) {
-        if (diag && kv0 + i > qpos) s[i] = -INFINITY;
-        mx = fmaxf(mx, s[i]);
+        for (int i = 0; i < BKV; ++i)
+          if (kv0 + i > qpos) s[i] = -INFINITY;
       }
-      const float m_new = fmaxf(m_run, mx);  // finite from the first tile on: key 0 is visible to every row
-      const float corr = exp2f((m_run - m_new) * scale_log2e);
-      m_run = m_new;
-      // the previous tile's P V product: add it (it is at the previous maximum), then move everything to the new one
-      if (j > 0) {
-        if (!mbar_wait(bar(7), ph ^ 1u, err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
-        tcgen05_fence_after();
-        float t[HD];
-        tmem_ld_32x32b_x32_issue(t_row + BKV, *reinterpret_cast<float(*)[32]>(&t[0]));
-        tmem_ld_32x32b_x32_issue(t_row + BKV + 32, *reinterpret_cast<float(*)[32]>(&t[32]));
-        tmem_ld_wait();
+      float mx0 = s[0], mx1 = s[1];
 #pragma unroll
-        for (int i = 0; i < HD; ++i) o[i] = (o[i] + t[i]) * corr;
+      for (int i = 2; i < BKV; i += 4) {
+        mx0 = fmax3(mx0, s[i], s[i + 1]);
+        if (i + 3 < BKV) mx1 = fmax3(mx1, s[i + 2], s[i + 3]);
       }
-      l_run *= corr;
-      // probabilities -> bf16 P tile (swizzled rows of 128 bytes)
-      const float mb = m_new * scale_log2e;
+      const float mx = fmaxf(mx0, mx1);  // finite from the first tile on: key 0 is visible to every row
+      float corr = 1.f;
+      const bool bump = (mx - m_run) * scale_log2e > kLazy;  // also true on the first tile (m_run = -inf)
+      if (bump) {
+        corr = ex2_approx((m_run - mx) * scale_log2e);
+        m_run = mx;
+        l_run *= corr;
+      }
+      // P[j & 1] was the A operand of the product two tiles back: that product must have completed
+      if (j >= 2 && !mbar_wait(bar(B_ODONE + (j & 1)), ph2 ^ 1u, err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
+      // probabilities -> bf16 P tile (swizzled rows of 128 bytes); two values per instruction where the
+      // hardware has packed fp32 arithmetic
+      const float mb = -m_run * scale_log2e;
+      const float2 sc2 = make_float2(scale_log2e, scale_log2e), mb2 = make_float2(mb, mb);
+      float2 lsum = make_float2(0.f, 0.f);
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
         uint32_t pk[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const float p0 = exp2f(fmaf(s[8 * q + 2 * i], scale_log2e, -mb));      // exp2(-inf) = 0 for masked keys
-          const float p1 = exp2f(fmaf(s[8 * q + 2 * i + 1], scale_log2e, -mb));
-          const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-          const float2 pf = __bfloat1622float2(pb);  // the sum uses the rounded probabilities the second MMA sees
-          l_run += pf.x + pf.y;
+          float2 e = ffma2(make_float2(s[8 * q + 2 * i], s[8 * q + 2 * i + 1]), sc2, mb2);
+          e.x = ex2_approx(e.x);  // exp2(-inf) = 0 for masked keys
+          e.y = ex2_approx(e.y);
+          lsum = fadd2(lsum, e);
+          const __nv_bfloat162 pb = __floats2bfloat162_rn(e.x, e.y);
           pk[i] = *reinterpret_cast<const uint32_t*>(&pb);
         }
-        *reinterpret_cast<uint4*>(sPg + swz128(r, q)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        *reinterpret_cast<uint4*>(sPg + (j & 1) * P_BYTES + swz128(r, q)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }
+      l_run += lsum.x + lsum.y;
       fence_proxy_async_smem();
+      // the accumulator in tensor memory is at the old reference maximum: bring this warp's rows to the new one
+      // before the tensor core adds this tile's product (rare after the first tile)
+      if (j > 0 && __any_sync(0xffffffffu, bump)) {
+        if (!mbar_wait(bar(B_ODONE + ((j - 1) & 1)), (uint32_t)(((j - 1) >> 1) & 1), err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
+        tcgen05_fence_after();
+        float t[HD];
+        tmem_ld_32x32b_x32_issue(t_o, *reinterpret_cast<float(*)[32]>(&t[0]));
+        tmem_ld_32x32b_x32_issue(t_o + 32, *reinterpret_cast<float(*)[32]>(&t[32]));
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < HD; ++i) t[i] *= corr;
+        tmem_st_32x32b_x32(t_o, *reinterpret_cast<float(*)[32]>(&t[0]));
+        tmem_st_32x32b_x32(t_o + 32, *reinterpret_cast<float(*)[32]>(&t[32]));
+        tmem_st_wait();
+      }
       tcgen05_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(6));
+      if (lane == 0) mbar_arrive(bar(B_PREADY + (j & 1)));
     }
-    // last product, normalisation, store through a swizzled [32 rows][128 B] box per warp (inside the P tile,
-    // which nobody reads any more)
-    if (ok && mbar_wait(bar(7), (uint32_t)((n_kv - 1) & 1), err, TFERR_WAIT_TMEM_FULL)) {
+    // normalisation and store through a swizzled [32 rows][128 B] box per warp (inside the P tile, which nobody
+    // reads any more once the last product has completed)
+    const int lb = (n_kv - 1) & 1;
+    if (ok && mbar_wait(bar(B_ODONE + lb), (uint32_t)(((n_kv - 1) >> 1) & 1), err, TFERR_WAIT_TMEM_FULL)) {
       tcgen05_fence_after();
-      float t[HD];
-      tmem_ld_32x32b_x32_issue(t_row + BKV, *reinterpret_cast<float(*)[32]>(&t[0]));
-      tmem_ld_32x32b_x32_issue(t_row + BKV + 32, *reinterpret_cast<float(*)[32]>(&t[32]));
+      float o[HD];
+      tmem_ld_32x32b_x32_issue(t_o, *reinterpret_cast<float(*)[32]>(&o[0]));
+      tmem_ld_32x32b_x32_issue(t_o + 32, *reinterpret_cast<float(*)[32]>(&o[32]));
       tmem_ld_wait();
-#pragma unroll
-      for (int i = 0; i < HD; ++i) o[i] += t[i];
       const float inv = 1.f / l_run;
       uint8_t* box = sPg + quad * 4096;
 #pragma unroll
