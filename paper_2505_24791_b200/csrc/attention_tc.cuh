@@ -10,10 +10,11 @@
 //                                it arrives from TMA ([key][channel], i.e. an MN-major B operand), no transposition
 //   rescale (rare)               the reference maximum of a row moves only when the true maximum has grown by more
 //                                than 2^8; only then is the accumulator read, scaled and written back
-// S and P are double-buffered, so the first MMA of tile j+1 is issued before the softmax of tile j has
-// finished and the tensor core never waits for the softmax warps of its own CTA (and vice versa, apart from
-// true data dependences two tiles back).  K and V tiles travel through rings of three buffers each, so the TMA
-// round trip of a tile is hidden behind the two tiles before it.  Two CTAs fit on an SM.
+// S is released as soon as the softmax warps hold it in registers, so the first MMA of tile j+1 runs under the
+// softmax of tile j; P is free again when the second MMA of the previous tile has completed, long before the
+// next probabilities are ready.  K and V tiles travel through rings of two buffers each.  The CTA needs 128
+// TMEM columns and about 65 KB of shared memory, so three CTAs (twelve softmax warps) share an SM and hide each
+// other's latencies.
 // Rows are addressed through 3-D tensor maps [slot][position][column], so positions >= L read as zeros and are
 // never written (ragged L).  Every mbarrier wait is bounded as in gemm_tc.cuh.
 // qkv rows are [q | k | v] (3d wide); out is [slot, L, d] bf16.  map_qkv has a box of 128 positions (queries),
@@ -28,10 +29,10 @@ using namespace tc;
 constexpr int BQ = 128, BKV = 64, HD = 64;
 constexpr int NUM_THREADS_ATTN = 192;  // warp 0 TMA, warp 1 MMA + TMEM, warps 2..5 softmax / epilogue
 constexpr int Q_BYTES = BQ * HD * 2, K_BYTES = BKV * HD * 2, V_BYTES = BKV * HD * 2, P_BYTES = BQ * BKV * 2;
-constexpr int KV_STAGES = 3;  // K and V tiles in flight ahead of the tensor core
+constexpr int KV_STAGES = 2;  // K and V tiles in flight ahead of the tensor core
 constexpr int KV_RING = KV_STAGES * (K_BYTES + V_BYTES);
-constexpr int SMEM_BYTES = Q_BYTES + KV_RING + 2 * P_BYTES + 256 + 1024;  // P is double-buffered
-constexpr uint32_t TMEM_COLS_ATTN = 256;  // S buffers at columns 0 and 64, the output accumulator at column 128
+constexpr int SMEM_BYTES = Q_BYTES + KV_RING + P_BYTES + 256 + 1024;
+constexpr uint32_t TMEM_COLS_ATTN = 128;  // S at column 0, the output accumulator at column 64
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
   asm volatile(
@@ -103,20 +104,21 @@ __host__ __device__ constexpr uint32_t make_idesc_attn(int m, int n, int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-__global__ void __launch_bounds__(NUM_THREADS_ATTN, 2)
+__global__ void __launch_bounds__(NUM_THREADS_ATTN, 3)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_kv,
                     const CUtensorMap* __restrict__ map_out, int L, int d,
                     float scale_log2e, int* err) {
   extern __shared__ uint8_t smem_attn_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_attn_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sQ = smem_u32(smem), sK = sQ + Q_BYTES, sV = sK + KV_STAGES * K_BYTES, sP = sV + KV_STAGES * V_BYTES;
-  const uint32_t bar_base = sP + 2 * P_BYTES;
-  // barriers: 0 q_full, then k_full[st], k_empty[st], v_full[st], v_empty[st], s_full[2], p_ready[2], o_done[2]
+  const uint32_t bar_base = sP + P_BYTES;
+  // barriers: 0 q_full, then k_full[st], k_empty[st], v_full[st], v_empty[st], s_full, s_free, p_ready, o_done
   constexpr int B_KFULL = 1, B_KEMPTY = B_KFULL + KV_STAGES, B_VFULL = B_KEMPTY + KV_STAGES, B_VEMPTY = B_VFULL + KV_STAGES,
-                B_SFULL = B_VEMPTY + KV_STAGES, B_PREADY = B_SFULL + 2, B_ODONE = B_PREADY + 2, NUM_BARS = B_ODONE + 2;
+                B_SFULL = B_VEMPTY + KV_STAGES, B_SFREE = B_SFULL + 1, B_PREADY = B_SFREE + 1, B_ODONE = B_PREADY + 1,
+                NUM_BARS = B_ODONE + 1;
   static_assert(NUM_BARS * 8 <= 192, "barrier area");
   auto bar = [&](int i) { return bar_base + 8u * i; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + Q_BYTES + KV_RING + 2 * P_BYTES + 192);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + Q_BYTES + KV_RING + P_BYTES + 192);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_qt = (L + BQ - 1) / BQ;
   const int qt = n_qt - 1 - (int)blockIdx.x;  // longest tiles first
@@ -125,7 +127,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
   const int n_kv = ((q0 + BQ < L ? q0 + BQ : L) + BKV - 1) / BKV;  // key tiles that hold a visible key
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < NUM_BARS; ++i) mbar_init(bar(i), (i == B_PREADY || i == B_PREADY + 1) ? 4 : 1);
+    for (int i = 0; i < NUM_BARS; ++i) mbar_init(bar(i), (i == B_PREADY || i == B_SFREE) ? 4 : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -164,35 +166,38 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
       constexpr uint32_t idesc_s = make_idesc_attn(BQ, BKV, 0), idesc_o = make_idesc_attn(BQ, HD, 1);
       bool ok = mbar_wait(bar(0), 0u, err, TFERR_WAIT_FULL);
       const uint64_t qdesc = make_smem_desc(sQ);
-      auto scores = [&](int j) {  // S[j & 1] = Q K_j^T
+      auto scores = [&](int j) {  // S = Q K_j^T
         const int st = j % KV_STAGES;
         if (!mbar_wait(bar(B_KFULL + st), (uint32_t)((j / KV_STAGES) & 1), err, TFERR_WAIT_FULL)) return false;
         tcgen05_fence_after();
         const uint64_t kdesc = make_smem_desc(sK + st * K_BYTES);
 #pragma unroll
-        for (int k = 0; k < HD / UMMA_K; ++k) umma_f16(tmem_base + (j & 1) * BKV, qdesc + 2u * k, kdesc + 2u * k, idesc_s, k != 0);
-        umma_commit(bar(B_KEMPTY + st));      // K buffer free
-        umma_commit(bar(B_SFULL + (j & 1)));  // S[j & 1] complete
+        for (int k = 0; k < HD / UMMA_K; ++k) umma_f16(tmem_base, qdesc + 2u * k, kdesc + 2u * k, idesc_s, k != 0);
+        umma_commit(bar(B_KEMPTY + st));  // K buffer free
+        umma_commit(bar(B_SFULL));        // S complete
         return true;
       };
       if (ok) ok = scores(0);
       for (int j = 0; j < n_kv && ok; ++j) {
-        // the next tile's scores are issued before this tile's probabilities are awaited: its S buffer was last
-        // read by the softmax of tile j-1, which had finished when p_ready of tile j-1 was seen
-        if (j + 1 < n_kv && !scores(j + 1)) { ok = false; break; }
+        // the next tile's scores are issued as soon as the softmax warps hold this tile's scores in registers,
+        // long before this tile's probabilities are ready
+        if (j + 1 < n_kv) {
+          if (!mbar_wait(bar(B_SFREE), (uint32_t)(j & 1), err, TFERR_WAIT_TMEM_EMPTY)) { ok = false; break; }
+          if (!scores(j + 1)) { ok = false; break; }
+        }
         const int st = j % KV_STAGES;
-        if (!mbar_wait(bar(B_PREADY + (j & 1)), (uint32_t)((j >> 1) & 1), err, TFERR_WAIT_TMEM_EMPTY)) { ok = false; break; }
+        if (!mbar_wait(bar(B_PREADY), (uint32_t)(j & 1), err, TFERR_WAIT_TMEM_EMPTY)) { ok = false; break; }
         if (!mbar_wait(bar(B_VFULL + st), (uint32_t)((j / KV_STAGES) & 1), err, TFERR_WAIT_FULL)) { ok = false; break; }
         tcgen05_fence_after();
 #pragma unroll
         for (int k = 0; k < BKV / UMMA_K; ++k) {
           // P: [128 rows][128 B] (64 keys), 16 keys = 32 bytes along a row.  V: 16 keys = 2048 bytes.
-          const uint64_t pdesc = make_smem_desc(sP + (j & 1) * P_BYTES) + 2u * k;
+          const uint64_t pdesc = make_smem_desc(sP) + 2u * k;
           const uint64_t vdesc = make_smem_desc_mn(sV + st * V_BYTES + k * (UMMA_K * 128));
-          umma_f16(tmem_base + 2 * BKV, pdesc, vdesc, idesc_o, (j | k) != 0);
+          umma_f16(tmem_base + BKV, pdesc, vdesc, idesc_o, (j | k) != 0);
         }
-        umma_commit(bar(B_VEMPTY + st));      // V buffer free
-        umma_commit(bar(B_ODONE + (j & 1)));  // products up to tile j complete (and P[j & 1] free)
+        umma_commit(bar(B_VEMPTY + st));  // V buffer free
+        umma_commit(bar(B_ODONE));        // products up to tile j complete (and P free)
       }
     }
   } else {
@@ -201,7 +206,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
     const int r = quad * 32 + lane;            // row of this thread inside the query tile
     const int qpos = q0 + r;                   // position in the sequence
     const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
-    const uint32_t t_o = t_row + 2 * BKV;      // this row's slice of the output accumulator
+    const uint32_t t_o = t_row + BKV;          // this row's slice of the output accumulator
     uint8_t* sPg = smem + Q_BYTES + KV_RING;
     // m_run is the reference maximum of the row (in raw score units); it trails the true running maximum by at
     // most kLazy / scale_log2e, so probabilities stay below 2^kLazy and the accumulator is rescaled only rarely
@@ -209,16 +214,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = !dead;
     for (int j = 0; j < n_kv && ok; ++j) {
-      const uint32_t ph2 = (j >> 1) & 1;  // phase of the per-buffer barriers
-      if (!mbar_wait(bar(B_SFULL + (j & 1)), ph2, err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
+      if (!mbar_wait(bar(B_SFULL), (uint32_t)(j & 1), err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
       tcgen05_fence_after();
       const int kv0 = j * BKV;
       const bool diag = kv0 + BKV - 1 > q0;  // some key of this tile lies after some query of the tile
       // the whole score row in one round of tensor-memory loads
       float s[BKV];
-      tmem_ld_32x32b_x32_issue(t_row + (j & 1) * BKV, *reinterpret_cast<float(*)[32]>(&s[0]));
-      tmem_ld_32x32b_x32_issue(t_row + (j & 1) * BKV + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
+      tmem_ld_32x32b_x32_issue(t_row, *reinterpret_cast<float(*)[32]>(&s[0]));
+      tmem_ld_32x32b_x32_issue(t_row + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
       tmem_ld_wait();
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_SFREE));  // the tensor core may overwrite S with the next tile's scores
       if (diag) {
 #pragma unroll
         for (int i = 0; i < BKV; ++i)
@@ -238,8 +245,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
         m_run = mx;
         l_run *= corr;
       }
-      // P[j & 1] was the A operand of the product two tiles back: that product must have completed
-      if (j >= 2 && !mbar_wait(bar(B_ODONE + (j & 1)), ph2 ^ 1u, err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
+      // P was the A operand of the previous tile's product, which also has to be in the accumulator before a rescale
+      if (j > 0) {
+        if (!mbar_wait(bar(B_ODONE), (uint32_t)((j - 1) & 1), err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
+        tcgen05_fence_after();
+      }
       // probabilities -> bf16 P tile (swizzled rows of 128 bytes); two values per instruction where the
       // hardware has packed fp32 arithmetic
       const float mb = -m_run * scale_log2e;
@@ -257,15 +267,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
           const __nv_bfloat162 pb = __floats2bfloat162_rn(e.x, e.y);
           pk[i] = *reinterpret_cast<const uint32_t*>(&pb);
         }
-        *reinterpret_cast<uint4*>(sPg + (j & 1) * P_BYTES + swz128(r, q)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        *reinterpret_cast<uint4*>(sPg + swz128(r, q)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }
       l_run += lsum.x + lsum.y;
       fence_proxy_async_smem();
       // the accumulator in tensor memory is at the old reference maximum: bring this warp's rows to the new one
       // before the tensor core adds this tile's product (rare after the first tile)
       if (j > 0 && __any_sync(0xffffffffu, bump)) {
-        if (!mbar_wait(bar(B_ODONE + ((j - 1) & 1)), (uint32_t)(((j - 1) >> 1) & 1), err, TFERR_WAIT_TMEM_FULL)) { ok = false; break; }
-        tcgen05_fence_after();
         float t[HD];
         tmem_ld_32x32b_x32_issue(t_o, *reinterpret_cast<float(*)[32]>(&t[0]));
         tmem_ld_32x32b_x32_issue(t_o + 32, *reinterpret_cast<float(*)[32]>(&t[32]));
@@ -278,12 +286,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
       }
       tcgen05_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_PREADY + (j & 1)));
+      if (lane == 0) mbar_arrive(bar(B_PREADY));
     }
     // normalisation and store through a swizzled [32 rows][128 B] box per warp (inside the P tile, which nobody
     // reads any more once the last product has completed)
-    const int lb = (n_kv - 1) & 1;
-    if (ok && mbar_wait(bar(B_ODONE + lb), (uint32_t)(((n_kv - 1) >> 1) & 1), err, TFERR_WAIT_TMEM_FULL)) {
+    if (ok && mbar_wait(bar(B_ODONE), (uint32_t)((n_kv - 1) & 1), err, TFERR_WAIT_TMEM_FULL)) {
       tcgen05_fence_after();
       float o[HD];
       tmem_ld_32x32b_x32_issue(t_o, *reinterpret_cast<float(*)[32]>(&o[0]));

@@ -158,7 +158,7 @@ struct tf_model {
   CUtensorMap map_xn, map_att, map_mlp, map_xn_lo, map_att_lo, map_mlp_lo;
   enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_ATT3, SM_COUNT };
   CUtensorMap map_qkv3, map_kv3;  // qkv as [slot][position][3d] for the tensor-core attention (query / key boxes)
-  bool use_tc_attention = false;  // measured slower than the mma.sync kernel so far: opt-in (TARFLOW_ATTN_TC=1)
+  bool use_tc_attention = true;   // single-operand attention on tcgen05 (TARFLOW_ATTN_TC=0: the mma.sync kernel)
   CUtensorMap* store_maps = nullptr;  // device copy of the bulk-store maps of qkv, qkv_lo, mlp, mlp_lo, h
   CUtensorMap map_seq_a[3][3];  // sequential-step GEMM operands {xn, att, mlp} x row tile {16, 32, 64}
   bool use_pair_gemm = true;    // sweep GEMMs on 2-CTA tile pairs (false: one CTA per tile)

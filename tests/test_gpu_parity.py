@@ -231,11 +231,11 @@ def test_bf16_ragged_sequence_length_and_classes():
 
 
 def test_bf16_optional_kernel_paths_agree(monkeypatch):
-    """The opt-in tcgen05 attention and the one-CTA-per-tile GEMM give the same sweep as the default kernels."""
+    """The mma.sync attention and the one-CTA-per-tile GEMM give the same sweep as the default kernels."""
     cfg = synth.config("cfg2", n_blocks=1, n_layers=2)
     z = synth.make_latents(cfg, 17, B=3)
     outs = {}
-    for name, env in (("default", {}), ("attn_tc", {"TARFLOW_ATTN_TC": "1"}), ("single_cta", {"TARFLOW_PAIR_GEMM": "0"})):
+    for name, env in (("default", {}), ("attn_mma", {"TARFLOW_ATTN_TC": "0"}), ("single_cta", {"TARFLOW_PAIR_GEMM": "0"})):
         for k in ("TARFLOW_ATTN_TC", "TARFLOW_PAIR_GEMM"):
             monkeypatch.delenv(k, raising=False)
         for k, v in env.items():
@@ -246,5 +246,5 @@ def test_bf16_optional_kernel_paths_agree(monkeypatch):
     xo, _ = O.model_inverse(synth.make_weights(cfg), z, None, cfg, [1], -1.0, 3)
     for name, x in outs.items():
         assert rel_l2(x, xo) <= BF16_REL_L2, name
-    assert rel_l2(outs["attn_tc"], outs["default"]) <= 5e-3
+    assert rel_l2(outs["attn_mma"], outs["default"]) <= 5e-3
     assert rel_l2(outs["single_cta"], outs["default"]) <= 1e-4
