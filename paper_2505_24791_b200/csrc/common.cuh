@@ -62,3 +62,11 @@ __device__ __forceinline__ void atomic_max_nonneg(float* addr, float v) {
 
 // Core position l of a block <-> raster token index (block permutation: reversal on odd blocks).
 __device__ __forceinline__ int tok_index(int l, int L, int reversed) { return reversed ? (L - 1 - l) : l; }
+
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may be scheduled
+// while its predecessor in the stream still runs; it must not touch anything the predecessor reads or writes
+// before pdl_wait(), which returns once the predecessor has completed and its writes are visible.
+// pdl_launch_dependents() lets the successor's CTAs be scheduled as soon as every CTA of this kernel has
+// called it.  Both are no-ops in a kernel launched without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

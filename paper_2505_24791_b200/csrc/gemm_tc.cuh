@@ -199,6 +199,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   using SL = SmemLayout<BN, STAGES>;
   extern __shared__ uint8_t smem_raw[];
   __shared__ int s_prev_err;
+  pdl_launch_dependents();
+  pdl_wait();  // the activations (and the error word) of the previous kernel are complete
   if (threadIdx.x == 0) s_prev_err = *reinterpret_cast<volatile int*>(err);
   __syncthreads();
   if (s_prev_err != 0) return;  // an earlier kernel failed: the whole CTA does nothing

@@ -90,6 +90,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   static_assert(Epi::kTmaCols > 0, "the pair kernel has the bulk-store epilogue only");
   using SL = Smem2;
   extern __shared__ uint8_t smem_raw2[];
+  pdl_launch_dependents();
+  pdl_wait();  // the activations (and the error word) of the previous kernel are complete
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw2) + 1023) & ~(uintptr_t)1023);
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_base = smem_base + SL::BAR_OFFSET;

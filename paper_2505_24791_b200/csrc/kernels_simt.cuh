@@ -58,6 +58,8 @@ embed_rows_kernel(const float* __restrict__ u, const int* __restrict__ idx, cons
                   const float* __restrict__ w_in_t, const float* __restrict__ b_in, const float* __restrict__ pos,
                   const float* __restrict__ cls, float* __restrict__ h, int L, int D, int d, int reversed, int n_rows) {
   extern __shared__ __align__(16) float s_ut[];  // [D][R]
+  pdl_launch_dependents();
+  pdl_wait();
   const int row0 = blockIdx.x * R;
   for (int e = threadIdx.x; e < R * D; e += blockDim.x) {
     const int r = e / D, c = e - r * D, row = row0 + r;
@@ -107,6 +109,8 @@ template <class T, int MAXV>
 __global__ void layernorm_kernel(const float* __restrict__ x, const float* __restrict__ gamma,
                                  const float* __restrict__ beta, T* __restrict__ y, T* __restrict__ y_lo, int rows,
                                  int d) {
+  pdl_launch_dependents();
+  pdl_wait();
   int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= rows) return;
   const float4* xr = reinterpret_cast<const float4*>(x + (size_t)warp * d);
@@ -392,7 +396,7 @@ __global__ void __launch_bounds__(256) forward_affine_kernel(const float* __rest
 }
 
 // ------------------------------------------------------------------------------------------------
-// Sweep control (single thread; B is at most a few hundred).  After sweep `t`: record the sweep
+// Sweep control.  After sweep `t`: record the sweep
 // count of every active sample, drop the samples that passed the test, move a sample to the
 // two-term ("hp") phase once its own max|du| <= switch_thresh, and rebuild the slot list as
 // [single-precision samples..., hp samples...] with a stable partition, so the slot order never
@@ -400,31 +404,73 @@ __global__ void __launch_bounds__(256) forward_affine_kernel(const float* __rest
 // ctrl[0] = n_active, ctrl[1] = non-finite flag, ctrl[2] = bits of max over active samples of
 // maxdiff, ctrl[3] = number of active samples in the hp phase (the tail of idx).
 // ------------------------------------------------------------------------------------------------
-__global__ void jacobi_finalize_kernel(float* __restrict__ maxdiff, int* __restrict__ idx, int* __restrict__ idx_tmp,
-                                       int* __restrict__ phase, int* __restrict__ ctrl, int* __restrict__ iters_sample,
-                                       float tau, float switch_thresh, int t) {
-  if (threadIdx.x != 0 || blockIdx.x != 0) return;
-  int n = ctrl[0], keep = 0, bad = ctrl[1];
+// One CTA of 256 threads; the order of the surviving samples is kept (stable compaction), single-term samples first.
+__global__ void __launch_bounds__(256)
+jacobi_finalize_kernel(float* __restrict__ maxdiff, int* __restrict__ idx, int* __restrict__ idx_tmp,
+                       int* __restrict__ phase, int* __restrict__ ctrl, int* __restrict__ iters_sample,
+                       float tau, float switch_thresh, int t) {
+  __shared__ int s_cnt[2][8];
+  __shared__ float s_top[8];
+  __shared__ int s_flag[2][8];
+  pdl_launch_dependents();
+  pdl_wait();
+  if (blockIdx.x != 0) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned below = (1u << lane) - 1u;
+  const int n = ctrl[0];
+  int base0 = 0, base1 = 0;  // survivors so far: single-term phase, two-term phase
   float top = 0.f;
-  for (int s = 0; s < n; ++s) {
-    int b = idx[s];
-    float m = maxdiff[b];
-    maxdiff[b] = 0.f;
-    top = (m > top || m != m) ? m : top;
-    if (iters_sample) iters_sample[b] = t;
-    if (!(m <= 3.0e38f)) bad = 1;
-    if (tau < 0.f || !(m <= tau)) {
-      if (m <= switch_thresh) phase[b] = 1;
-      idx_tmp[keep++] = b;
+  int bad = 0, nan = 0;
+  for (int c0 = 0; c0 < n; c0 += 256) {
+    const int s = c0 + threadIdx.x;
+    int b = 0;
+    bool f0 = false, f1 = false;
+    if (s < n) {
+      b = idx[s];
+      const float m = maxdiff[b];
+      maxdiff[b] = 0.f;
+      if (m != m) nan = 1; else top = fmaxf(top, m);
+      if (iters_sample) iters_sample[b] = t;
+      if (!(m <= 3.0e38f)) bad = 1;
+      if (tau < 0.f || !(m <= tau)) {
+        int ph = phase[b];
+        if (m <= switch_thresh) { phase[b] = 1; ph = 1; }
+        f0 = ph == 0;
+        f1 = !f0;
+      }
     }
+    const unsigned b0 = __ballot_sync(0xffffffffu, f0), b1 = __ballot_sync(0xffffffffu, f1);
+    if (lane == 0) { s_cnt[0][warp] = __popc(b0); s_cnt[1][warp] = __popc(b1); }
+    __syncthreads();  // every idx[s] of this chunk has been read before any slot of the chunk is overwritten
+    int off0 = base0, off1 = base1;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      if (w < warp) { off0 += s_cnt[0][w]; off1 += s_cnt[1][w]; }
+      base0 += s_cnt[0][w];
+      base1 += s_cnt[1][w];
+    }
+    if (f0) idx[off0 + __popc(b0 & below)] = b;      // slot <= s: already read
+    if (f1) idx_tmp[off1 + __popc(b1 & below)] = b;
+    __syncthreads();
   }
-  int k = 0, n_hp = 0;
-  for (int s = 0; s < keep; ++s) if (phase[idx_tmp[s]] == 0) idx[k++] = idx_tmp[s];
-  for (int s = 0; s < keep; ++s) if (phase[idx_tmp[s]] != 0) { idx[k++] = idx_tmp[s]; ++n_hp; }
-  ctrl[0] = keep;
-  ctrl[1] = bad;
-  ctrl[2] = __float_as_int(top);
-  ctrl[3] = n_hp;
+  for (int j = threadIdx.x; j < base1; j += 256) idx[base0 + j] = idx_tmp[j];
+  top = warp_max(top);
+  bad = __any_sync(0xffffffffu, bad != 0);
+  nan = __any_sync(0xffffffffu, nan != 0);
+  if (lane == 0) { s_top[warp] = top; s_flag[0][warp] = bad; s_flag[1][warp] = nan; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int anybad = ctrl[1], anynan = 0;
+    for (int w = 0; w < 8; ++w) {
+      top = fmaxf(top, s_top[w]);
+      anybad |= s_flag[0][w];
+      anynan |= s_flag[1][w];
+    }
+    ctrl[0] = base0 + base1;
+    ctrl[1] = anybad;
+    ctrl[2] = anynan ? 0x7fc00000 : __float_as_int(top);
+    ctrl[3] = base1;
+  }
 }
 
 __global__ void jacobi_begin_kernel(float* __restrict__ maxdiff, int* __restrict__ idx, int* __restrict__ phase,

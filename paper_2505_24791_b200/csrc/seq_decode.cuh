@@ -64,12 +64,10 @@ __device__ __forceinline__ void cp_async_wait_all() {
   asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
 }
 
-// Programmatic dependent launch: a kernel lets its successor in the stream start early (its CTAs are
-// scheduled, fetch weights, and then block in pdl_wait) and itself waits for its predecessor's
-// results only where it first needs them.  Every kernel of the chain calls pdl_wait before it ends,
-// so "kernel k finished" always implies "kernels < k finished".
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Programmatic dependent launch (pdl_launch_dependents / pdl_wait of common.cuh): a kernel lets its successor in
+// the stream start early (its CTAs are scheduled, fetch weights, and then block in pdl_wait) and itself waits for
+// its predecessor's results only where it first needs them.  Every kernel of the chain calls pdl_wait before it
+// ends, so "kernel k finished" always implies "kernels < k finished".
 
 // B fragments from 16-byte weight loads.  Lane (g, t) of a warp loads W[n0 + g][k0 + 8t .. k0 + 8t + 7],
 // i.e. the four lanes of a quad hold the four 16-byte chunks of one 32-wide k group of row g, as pairs

@@ -247,6 +247,29 @@ struct tf_model {
     (m)->post(cls);                                            \
   } while (0)
 
+// Launch with programmatic stream serialization: only for kernels that call pdl_wait() before they touch global
+// memory, so their CTAs may be scheduled while the previous kernel of the stream drains.
+template <class... KArgs, class... Args>
+static void launch_pdl_raw(cudaStream_t stream, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args... args) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = grid;
+  lc.blockDim = block;
+  lc.dynamicSmemBytes = smem;
+  lc.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  cudaLaunchKernelEx(&lc, kern, static_cast<KArgs>(args)...);  // errors surface in check_launch()
+}
+#define LAUNCH_PDL(m, cls, kern, grid, block, smem, ...)                                        \
+  do {                                                                                          \
+    (m)->pre(cls);                                                                              \
+    launch_pdl_raw((m)->stream, kern, dim3(grid), dim3(block), (size_t)(smem), __VA_ARGS__);    \
+    (m)->post(cls);                                                                             \
+  } while (0)
+
 static int check_launch(const char* what) {
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(TF_ECUDA, "%s: %s", what, cudaGetErrorString(e));
@@ -286,7 +309,8 @@ static int launch_gemm_tc(tf_model* m, int cls, cudaStream_t stream, const CUten
   int tiles = ((M + tc::BM - 1) / tc::BM) * ((N + BN - 1) / BN);
   int grid = tiles < num_sms ? tiles : num_sms;
   if (m) m->pre(cls);
-  kern<<<grid, tc::NUM_THREADS, SL::TOTAL, stream>>>(ma, ma_lo ? *ma_lo : ma, mw, M, N, K, ma_lo ? 1 : 0, epi, err);
+  launch_pdl_raw(stream, kern, dim3(grid), dim3(tc::NUM_THREADS), (size_t)SL::TOTAL, ma, ma_lo ? *ma_lo : ma, mw, M, N, K,
+                 ma_lo ? 1 : 0, epi, err);
   if (m) m->post(cls); else if (launches) ++*launches;
   return check_launch("gemm_tc_kernel");
 }
@@ -309,13 +333,15 @@ static int launch_gemm_tc2(tf_model* m, int cls, const CUtensorMap& ma, const CU
   lc.blockDim = dim3(tc::NUM_THREADS);
   lc.dynamicSmemBytes = tc2::Smem2::TOTAL;
   lc.stream = m->stream;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 2;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at;
-  lc.numAttrs = 1;
+  lc.numAttrs = 2;
   m->pre(cls);
   cudaError_t e = cudaLaunchKernelEx(&lc, kern, ma, ma_lo ? *ma_lo : ma, mw, M, N, K, ma_lo ? 1 : 0, epi, m->err);
   m->post(cls);
@@ -357,10 +383,10 @@ template <class T>
 static int layernorm(tf_model* m, int cls, const float* x, const float* g, const float* b, T* y, T* y_lo, int rows) {
   int d = m->d;
   int blocks = (rows * 32 + 255) / 256;
-  if (d <= 128 * 1) LAUNCH(m, cls, (layernorm_kernel<T, 1>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
-  else if (d <= 128 * 4) LAUNCH(m, cls, (layernorm_kernel<T, 4>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
-  else if (d <= 128 * 8) LAUNCH(m, cls, (layernorm_kernel<T, 8>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
-  else LAUNCH(m, cls, (layernorm_kernel<T, 16>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
+  if (d <= 128 * 1) LAUNCH_PDL(m, cls, (layernorm_kernel<T, 1>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
+  else if (d <= 128 * 4) LAUNCH_PDL(m, cls, (layernorm_kernel<T, 4>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
+  else if (d <= 128 * 8) LAUNCH_PDL(m, cls, (layernorm_kernel<T, 8>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
+  else LAUNCH_PDL(m, cls, (layernorm_kernel<T, 16>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
   return check_launch("layernorm_kernel");
 }
 
@@ -385,7 +411,7 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
   const CUtensorMap* mml = hp ? &m->map_mlp_lo : nullptr;
   int ethreads = d < 256 ? d : 256;
   m->cur_rows = M;
-  LAUNCH(m, KC_EMBED, embed_rows_kernel<16>, (M + 15) / 16, ethreads, 16 * D * sizeof(float), u_src, idx, labels, bw.w_in_t,
+  LAUNCH_PDL(m, KC_EMBED, embed_rows_kernel<16>, (M + 15) / 16, ethreads, 16 * D * sizeof(float), u_src, idx, labels, bw.w_in_t,
          bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, M);
   TF_TRY(check_launch("embed_kernel"));
   for (const LayerW& lw : bw.layers) {
@@ -404,7 +430,7 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
         LAUNCH(m, KC_ATTN, attn::attention_mma_kernel<true>, grid, 128, attn::smem_bytes<true>(), qkv, qkv_lo, att,
                att_lo, L, d, sl2);
       else if (m->use_tc_attention)
-        LAUNCH(m, KC_ATTN, attn_tc::attention_tc_kernel, dim3((L + attn_tc::BQ - 1) / attn_tc::BQ, m->cfg.n_heads, n_slots),
+        LAUNCH_PDL(m, KC_ATTN, attn_tc::attention_tc_kernel, dim3((L + attn_tc::BQ - 1) / attn_tc::BQ, m->cfg.n_heads, n_slots),
                attn_tc::NUM_THREADS_ATTN, attn_tc::SMEM_BYTES, m->map_qkv3, m->map_kv3, m->store_maps + tf_model::SM_ATT3, L, d, sl2,
                m->err);
       else
@@ -714,7 +740,7 @@ static int run_jacobi_block(tf_model* m, int g, int B, const int* labels, const 
     const int n_lp = n_active - n_hp;
     if (n_lp > 0) TF_TRY(run_pass<T>(m, g, n_lp, u, m->idx, labels, PASS_JACOBI, v, u, false));
     if (n_hp > 0) TF_TRY(run_pass<T>(m, g, n_hp, u, m->idx + n_lp, labels, PASS_JACOBI, v, u, true));
-    LAUNCH(m, KC_CTRL, jacobi_finalize_kernel, 1, 32, 0, m->maxdiff, m->idx, m->idx_tmp, m->phase, m->ctrl, iters_row,
+    LAUNCH_PDL(m, KC_CTRL, jacobi_finalize_kernel, 1, 256, 0, m->maxdiff, m->idx, m->idx_tmp, m->phase, m->ctrl, iters_row,
            tau, sw, t);
     if (tau >= 0.f || t == max_iters || m->trace_on) {
       const int before = n_active;
