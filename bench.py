@@ -76,7 +76,7 @@ def class_work(cfg, L, D):
         "gemm_head": (bound, 2.0 * 2 * D * d, 0.0),
         "attention": (bound, 2.0 * d * L, 0.0),
         "layernorm": ("hbm", d * (4.0 + esz), 0.0),
-        "embed": ("hbm", D * 4.0 + d * 4.0, 0.0),
+        "embed": ("hbm", D * 4.0 + d * (4.0 + esz), 0.0),  # token in, residual row and first LayerNorm's row out
         "forward_affine": ("hbm", D * (2 * 4.0 + 2 * 4.0), 0.0),
         "layout": ("hbm", 0.0, 0.0),
         "sweep_control": ("hbm", 0.0, 0.0),

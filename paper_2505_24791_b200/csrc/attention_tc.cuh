@@ -109,8 +109,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
                     const CUtensorMap* __restrict__ map_out, int L, int d,
                     float scale_log2e, int* err) {
   extern __shared__ uint8_t smem_attn_raw[];
-  pdl_launch_dependents();
-  pdl_wait();  // q, k, v of the previous kernel are complete
+  pdl_launch_dependents();  // the next kernel of the stream may be scheduled; it waits for this one to complete
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_attn_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sQ = smem_u32(smem), sK = sQ + Q_BYTES, sV = sK + KV_STAGES * K_BYTES, sP = sV + KV_STAGES * V_BYTES;
   const uint32_t bar_base = sP + P_BYTES;
@@ -142,6 +141,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();  // set-up above overlaps the previous kernel's tail; q, k, v and the error word are complete from here on
   const bool dead = *reinterpret_cast<volatile int*>(err) != 0;
 
   if (warp == 0) {

@@ -236,10 +236,69 @@ struct EpiHeadUpdate {
     }
     if (lane == 0) atomic_max_nonneg(maxdiff + b, df);
   }
+  // R consecutive rows at once: all loads of the old iterate and of v are issued before the first store (the rows
+  // of a batch touch distinct tokens), so a warp pays one memory round trip per batch instead of one per row;
+  // rows of the same sample share one reduction and one atomic.
   template <int R>
   __device__ __forceinline__ void store_rows(int row0, int col, const float (&acc)[R], float cc, bool col_ok, int lane) const {
+    const bool active = col_ok && (lane & 1) == 0;
+    const int c = col >> 1;
+    float mine[R], al[R], old[R], vv[R], df[R];
+    size_t e[R];
+    int bs[R], ss[R];
+    bool upd[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) store(row0 + r, col, acc[r], cc, col_ok, lane);
+    for (int r = 0; r < R; ++r) {
+      mine[r] = acc[r] + cc;
+      al[r] = __shfl_down_sync(0xffffffffu, mine[r], 1);
+      const int row = row0 + r;
+      const int s = row / L, l = row - s * L;
+      ss[r] = s;
+      bs[r] = idx ? idx[s] : s;
+      upd[r] = l < L - 1;  // the last position's head output is unused: that row copies token 0
+      e[r] = ((size_t)bs[r] * L + tok_index(upd[r] ? l + 1 : 0, L, reversed)) * D + c;
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      old[r] = 0.f;
+      vv[r] = 0.f;
+      if (active) {
+        old[r] = u[e[r]];
+        vv[r] = v[e[r]];
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      df[r] = 0.f;
+      if (active) {
+        const float nw = upd[r] ? fmaf(vv[r], expf(al[r]), mine[r]) : vv[r];
+        u[e[r]] = nw;
+        df[r] = fabsf(nw - old[r]);
+      }
+    }
+    // NaN-propagating max; the slot index is the same in every lane, so the branch is uniform
+    if (ss[0] == ss[R - 1]) {
+      float m = df[0];
+#pragma unroll
+      for (int r = 1; r < R; ++r) m = (df[r] > m || df[r] != df[r]) ? df[r] : m;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float other = __shfl_xor_sync(0xffffffffu, m, o);
+        m = (other > m || other != other) ? other : m;
+      }
+      if (lane == 0) atomic_max_nonneg(maxdiff + bs[0], m);
+    } else {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        float m = df[r];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float other = __shfl_xor_sync(0xffffffffu, m, o);
+          m = (other > m || other != other) ? other : m;
+        }
+        if (lane == 0) atomic_max_nonneg(maxdiff + bs[r], m);
+      }
+    }
   }
   template <int NC>
   __device__ __forceinline__ void apply(int row, int col0, const float (&acc)[NC], int nv) const {

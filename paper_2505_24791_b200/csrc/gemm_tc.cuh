@@ -198,12 +198,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 SmemLayout<BN, STAGES>::STAGE_OUT_BYTES, "bias tile must fit behind the store boxes");
   using SL = SmemLayout<BN, STAGES>;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ int s_prev_err;
-  pdl_launch_dependents();
-  pdl_wait();  // the activations (and the error word) of the previous kernel are complete
-  if (threadIdx.x == 0) s_prev_err = *reinterpret_cast<volatile int*>(err);
-  __syncthreads();
-  if (s_prev_err != 0) return;  // an earlier kernel failed: the whole CTA does nothing
+  pdl_launch_dependents();  // the next kernel of the stream may be scheduled; it waits for this one to complete
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t smem_base = smem_u32(smem);
@@ -216,7 +211,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN;
-  const int num_tiles = tiles_m * tiles_n;
+  const int num_tiles_all = tiles_m * tiles_n;
   // split != 0: A is an error-compensated pair (hi + lo); the K loop runs over [A_hi | A_lo] against
   // [W | W], i.e. both products accumulate into the same TMEM tile.
   const int kb_per_pass = (K + BK - 1) / BK;
@@ -244,6 +239,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above (barriers, tensor memory) overlaps the previous kernel's tail; its activations and the
+  // error word are complete from here on.  After an earlier failure the CTA walks an empty tile list.
+  pdl_wait();
+  const int num_tiles = *reinterpret_cast<volatile int*>(err) != 0 ? 0 : num_tiles_all;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer

@@ -90,8 +90,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   static_assert(Epi::kTmaCols > 0, "the pair kernel has the bulk-store epilogue only");
   using SL = Smem2;
   extern __shared__ uint8_t smem_raw2[];
-  pdl_launch_dependents();
-  pdl_wait();  // the activations (and the error word) of the previous kernel are complete
+  pdl_launch_dependents();  // the next kernel of the stream may be scheduled; it waits for this one to complete
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw2) + 1023) & ~(uintptr_t)1023);
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_base = smem_base + SL::BAR_OFFSET;
@@ -132,6 +131,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   cluster_sync_all();  // the peer's barriers exist before anything signals them
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above (barriers, tensor memory, cluster handshake) overlaps the previous kernel's tail; its
+  // activations and the error word are complete from here on
+  pdl_wait();
   // an earlier kernel failed: both CTAs skip the work (the leader's view decides, so the pair agrees)
   const bool dead = *reinterpret_cast<volatile int*>(err) != 0;
 

@@ -102,6 +102,140 @@ embed_rows_kernel(const float* __restrict__ u, const int* __restrict__ idx, cons
 }
 
 // ------------------------------------------------------------------------------------------------
+// Embedding of R rows per CTA fused with the first LayerNorm of the block:
+//   h[row, :]  = u[token] W_in^T + b_in + pos[l] (+ cls[y])          (fp32 residual stream)
+//   xn[row, :] = LayerNorm(h[row, :]) * gamma + beta                  (T; plus the "lo" half of a two-term pair)
+// Thread k owns columns 4k..4k+3 of all R rows (blockDim.x = d / 4 rounded up to whole warps, d % 4 == 0): per
+// token value one 16-byte weight load feeds 4 R FMAs, the R tokens sit in shared memory transposed ([D][R]) so
+// four rows come with one broadcast 16-byte read.  The row statistics (two-pass, eps 1e-5) are reduced over the
+// CTA's warps through shared memory.  h is bit-identical to embed_rows_kernel's.
+// ------------------------------------------------------------------------------------------------
+template <class T, int R>
+__global__ void __launch_bounds__(256)
+embed_ln_rows_kernel(const float* __restrict__ u, const int* __restrict__ idx, const int* __restrict__ labels,
+                     const float* __restrict__ w_in_t, const float* __restrict__ b_in, const float* __restrict__ pos,
+                     const float* __restrict__ cls, float* __restrict__ h, const float* __restrict__ gamma,
+                     const float* __restrict__ beta, T* __restrict__ xn, T* __restrict__ xn_lo, int L, int D, int d,
+                     int reversed, int n_rows) {
+  extern __shared__ __align__(16) float s_ut[];  // [D][R]
+  __shared__ float s_red[2][8][R];
+  __shared__ int s_l[R], s_b[R];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int row0 = blockIdx.x * R;
+  if (threadIdx.x < R) {
+    const int row = row0 + threadIdx.x;
+    int l = 0, b = -1;
+    if (row < n_rows) {
+      const int s = row / L;
+      l = row - s * L;
+      b = idx ? idx[s] : s;
+    }
+    s_l[threadIdx.x] = l;
+    s_b[threadIdx.x] = b;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < R * D; e += blockDim.x) {
+    const int r = e / D, c = e - r * D, b = s_b[r];
+    s_ut[c * R + r] = b >= 0 ? u[((size_t)b * L + tok_index(s_l[r], L, reversed)) * D + c] : 0.f;
+  }
+  __syncthreads();
+  const int k = threadIdx.x, dv = d >> 2;
+  const bool act = k < dv;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = (blockDim.x + 31) >> 5;
+  float4 acc[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (act) {
+    const float4* w4 = reinterpret_cast<const float4*>(w_in_t) + k;
+#pragma unroll 4
+    for (int c = 0; c < D; ++c) {
+      const float4 w = __ldg(w4 + (size_t)c * dv);
+#pragma unroll
+      for (int r4 = 0; r4 < R; r4 += 4) {
+        const float4 x = *reinterpret_cast<const float4*>(s_ut + c * R + r4);
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          acc[r4 + q].x = fmaf(xs[q], w.x, acc[r4 + q].x);
+          acc[r4 + q].y = fmaf(xs[q], w.y, acc[r4 + q].y);
+          acc[r4 + q].z = fmaf(xs[q], w.z, acc[r4 + q].z);
+          acc[r4 + q].w = fmaf(xs[q], w.w, acc[r4 + q].w);
+        }
+      }
+    }
+  }
+  // residual stream row, first statistic
+  float4 bj = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (act) bj = reinterpret_cast<const float4*>(b_in)[k];
+  float part[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const int row = row0 + r;
+    part[r] = 0.f;
+    if (act && row < n_rows) {
+      const float4 p = __ldg(reinterpret_cast<const float4*>(pos) + (size_t)s_l[r] * dv + k);
+      float4 a = acc[r];
+      a.x += bj.x + p.x; a.y += bj.y + p.y; a.z += bj.z + p.z; a.w += bj.w + p.w;
+      if (cls != nullptr) {
+        const float4 cl = __ldg(reinterpret_cast<const float4*>(cls) + (size_t)labels[s_b[r]] * dv + k);
+        a.x += cl.x; a.y += cl.y; a.z += cl.z; a.w += cl.w;
+      }
+      acc[r] = a;
+      reinterpret_cast<float4*>(h)[(size_t)row * dv + k] = a;
+      part[r] = (a.x + a.y) + (a.z + a.w);
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const float v = warp_sum(part[r]);
+    if (lane == 0) s_red[0][warp][r] = v;
+  }
+  __syncthreads();
+  const float inv_d = 1.f / (float)d;
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    float tot = 0.f;
+    for (int w = 0; w < nwarps; ++w) tot += s_red[0][w][r];
+    const float mean = tot * inv_d;
+    float sq = 0.f;
+    if (act) {
+      acc[r].x -= mean; acc[r].y -= mean; acc[r].z -= mean; acc[r].w -= mean;
+      sq = (acc[r].x * acc[r].x + acc[r].y * acc[r].y) + (acc[r].z * acc[r].z + acc[r].w * acc[r].w);
+    }
+    part[r] = warp_sum(sq);
+    if (lane == 0) s_red[1][warp][r] = part[r];
+  }
+  __syncthreads();
+  if (!act) return;
+  const float4 g = reinterpret_cast<const float4*>(gamma)[k], bb = reinterpret_cast<const float4*>(beta)[k];
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const int row = row0 + r;
+    if (row >= n_rows) continue;
+    float tot = 0.f;
+    for (int w = 0; w < nwarps; ++w) tot += s_red[1][w][r];
+    const float rstd = rsqrtf(tot * inv_d + 1e-5f);
+    const float o0 = acc[r].x * rstd * g.x + bb.x, o1 = acc[r].y * rstd * g.y + bb.y;
+    const float o2 = acc[r].z * rstd * g.z + bb.z, o3 = acc[r].w * rstd * g.w + bb.w;
+    if constexpr (sizeof(T) == 4) {
+      reinterpret_cast<float4*>(xn)[(size_t)row * dv + k] = make_float4(o0, o1, o2, o3);
+    } else {
+      __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);
+      uint2 w2;
+      w2.x = *reinterpret_cast<uint32_t*>(&p0); w2.y = *reinterpret_cast<uint32_t*>(&p1);
+      reinterpret_cast<uint2*>(xn)[(size_t)row * dv + k] = w2;
+      if (xn_lo != nullptr) {  // second term of the error-compensated pair
+        const float2 f0 = __bfloat1622float2(p0), f1 = __bfloat1622float2(p1);
+        __nv_bfloat162 q0 = __floats2bfloat162_rn(o0 - f0.x, o1 - f0.y), q1 = __floats2bfloat162_rn(o2 - f1.x, o3 - f1.y);
+        w2.x = *reinterpret_cast<uint32_t*>(&q0); w2.y = *reinterpret_cast<uint32_t*>(&q1);
+        reinterpret_cast<uint2*>(xn_lo)[(size_t)row * dv + k] = w2;
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // LayerNorm over the last dimension (eps 1e-5), fp32 in, T out.  One warp per row, the row is
 // held in registers (d <= 32*4*MAXV).
 // ------------------------------------------------------------------------------------------------

@@ -411,11 +411,21 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
   const CUtensorMap* mml = hp ? &m->map_mlp_lo : nullptr;
   int ethreads = d < 256 ? d : 256;
   m->cur_rows = M;
-  LAUNCH_PDL(m, KC_EMBED, embed_rows_kernel<16>, (M + 15) / 16, ethreads, 16 * D * sizeof(float), u_src, idx, labels, bw.w_in_t,
-         bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, M);
+  // embedding fused with the first LayerNorm when a thread can own four columns of a row
+  const bool fused_embed = d % 4 == 0 && d <= 1024 && (size_t)16 * D * sizeof(float) <= 40 * 1024;
+  if (fused_embed) {
+    const LayerW& l0 = bw.layers[0];
+    LAUNCH_PDL(m, KC_EMBED, (embed_ln_rows_kernel<T, 16>), (M + 15) / 16, ((d / 4 + 31) / 32) * 32, 16 * D * sizeof(float), u_src,
+               idx, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, l0.ln1_g, l0.ln1_b, xn, xn_lo, L, D, d, rev, M);
+  } else {
+    LAUNCH_PDL(m, KC_EMBED, embed_rows_kernel<16>, (M + 15) / 16, ethreads, 16 * D * sizeof(float), u_src, idx, labels,
+               bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, M);
+  }
   TF_TRY(check_launch("embed_kernel"));
+  bool first_layer = true;
   for (const LayerW& lw : bw.layers) {
-    TF_TRY(layernorm<T>(m, KC_LN, m->h, lw.ln1_g, lw.ln1_b, xn, xn_lo, M));
+    if (!(first_layer && fused_embed)) TF_TRY(layernorm<T>(m, KC_LN, m->h, lw.ln1_g, lw.ln1_b, xn, xn_lo, M));
+    first_layer = false;
     if constexpr (sizeof(T) == 2) {
       const CUtensorMap* sm = m->store_maps;
       TF_TRY(gemm<T>(m, KC_GEMM_QKV, xn, &m->map_xn, mxl, lw.w_qkv, M,
