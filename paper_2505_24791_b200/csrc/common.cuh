@@ -43,6 +43,64 @@ __device__ __forceinline__ float gelu_erf_fast(float x) {
   return fmaf(fabsf(hx), 1.0f - erfc_abs, hx);   // 0.5 x (1 + erf(x / sqrt 2)) with erf odd
 }
 
+// Packed fp32 arithmetic (two lanes per instruction), three-input maximum and the bare exp2 unit.
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;"
+      : "=l"(d)
+      : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)),
+        "l"(*reinterpret_cast<unsigned long long*>(&c)));
+  return *reinterpret_cast<float2*>(&d);
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;"
+      : "=l"(d)
+      : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
+  return *reinterpret_cast<float2*>(&d);
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float ex2_approx(float a) {
+  float d;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(d) : "f"(a));
+  return d;
+}
+__device__ __forceinline__ float2 fmul2(float2 a, float2 b) {
+  unsigned long long d;
+  asm("mul.rn.f32x2 %0, %1, %2;"
+      : "=l"(d)
+      : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
+  return *reinterpret_cast<float2*>(&d);
+}
+__device__ __forceinline__ float2 fabs2(float2 a) {
+  unsigned long long d = *reinterpret_cast<unsigned long long*>(&a) & 0x7fffffff7fffffffull;
+  return *reinterpret_cast<float2*>(&d);
+}
+
+// gelu_erf_fast on two values at once with the packed instructions: about half the issue slots per value.
+__device__ __forceinline__ float2 gelu_erf_fast2(float2 x) {
+  float2 z = fmul2(fabs2(x), make_float2(0.70710678118654752440f, 0.70710678118654752440f));
+  z.x = fminf(z.x, 4.0f);
+  z.y = fminf(z.y, 4.0f);
+  float2 p = ffma2(make_float2(1.0021848e-4f, 1.0021848e-4f), z, make_float2(-4.6155503e-4f, -4.6155503e-4f));
+  p = ffma2(p, z, make_float2(-2.302284e-3f, -2.302284e-3f));
+  p = ffma2(p, z, make_float2(2.945257e-2f, 2.945257e-2f));
+  p = ffma2(p, z, make_float2(-1.489637e-1f, -1.489637e-1f));
+  p = ffma2(p, z, make_float2(-9.1832864e-1f, -9.1832864e-1f));
+  p = ffma2(p, z, make_float2(-1.6279137f, -1.6279137f));
+  const float2 t = fmul2(p, z);
+  float2 e;  // erfc(|x| / sqrt 2)
+  e.x = ex2_approx(t.x);
+  e.y = ex2_approx(t.y);
+  const float2 hx = fmul2(x, make_float2(0.5f, 0.5f));
+  const float2 erf_abs = ffma2(e, make_float2(-1.0f, -1.0f), make_float2(1.0f, 1.0f));
+  return ffma2(fabs2(hx), erf_abs, hx);
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -354,15 +354,22 @@ struct EpiStoreTma {
                                           uint32_t box_addr, int lane) const {
     static_assert(CPG == 2, "a bf16 box is two 32-column chunks");
 #pragma unroll
-    for (int j = 0; j < 32; j += 4) {
+    for (int j = 0; j < 32; j += 4) {  // bias (+ GELU) two values per instruction
       const float4 b0 = *reinterpret_cast<const float4*>(sbias + j), b1 = *reinterpret_cast<const float4*>(sbias + 32 + j);
-      v0[j] += b0.x; v0[j + 1] += b0.y; v0[j + 2] += b0.z; v0[j + 3] += b0.w;
-      v1[j] += b1.x; v1[j + 1] += b1.y; v1[j + 2] += b1.z; v1[j + 3] += b1.w;
+      float2 a0 = fadd2(make_float2(v0[j], v0[j + 1]), make_float2(b0.x, b0.y));
+      float2 a1 = fadd2(make_float2(v0[j + 2], v0[j + 3]), make_float2(b0.z, b0.w));
+      float2 c0 = fadd2(make_float2(v1[j], v1[j + 1]), make_float2(b1.x, b1.y));
+      float2 c1 = fadd2(make_float2(v1[j + 2], v1[j + 3]), make_float2(b1.z, b1.w));
+      if (GELU) {
+        a0 = gelu_erf_fast2(a0); a1 = gelu_erf_fast2(a1);
+        c0 = gelu_erf_fast2(c0); c1 = gelu_erf_fast2(c1);
+      }
+      v0[j] = a0.x; v0[j + 1] = a0.y; v0[j + 2] = a1.x; v0[j + 3] = a1.y;
+      v1[j] = c0.x; v1[j + 1] = c0.y; v1[j + 2] = c1.x; v1[j + 3] = c1.y;
     }
-    if (GELU) {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) { v0[j] = gelu_erf_fast(v0[j]); v1[j] = gelu_erf_fast(v1[j]); }
-    }
+    // the engine reads the warp's previous box while the values above are computed; only now must it be done
+    if (lane == 0) tc::tma_store_wait_read();
+    __syncwarp();
     write_box(v0, v1, box, lane);
     tc::fence_proxy_async_smem();
     __syncwarp();
@@ -380,8 +387,6 @@ struct EpiStoreTma {
       __syncwarp();
       if (lane == 0) { tc::tma_store_2d(tmap_lo, col0, row0, box_addr); tc::tma_store_commit(); }
     }
-    if (lane == 0) tc::tma_store_wait_read();  // the box may be overwritten by the next call
-    __syncwarp();
   }
   __device__ __forceinline__ void write_box(const float (&v0)[32], const float (&v1)[32], uint8_t* box, int lane) const {
 #pragma unroll
@@ -411,12 +416,15 @@ struct EpiResidTma {
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       const float4 b = *reinterpret_cast<const float4*>(sbias + 4 * k);
-      *reinterpret_cast<float4*>(box + tc::swz128(lane, k)) =
-          make_float4(v[4 * k] + b.x, v[4 * k + 1] + b.y, v[4 * k + 2] + b.z, v[4 * k + 3] + b.w);
+      v[4 * k] += b.x; v[4 * k + 1] += b.y; v[4 * k + 2] += b.z; v[4 * k + 3] += b.w;
     }
+    if (lane == 0) tc::tma_store_wait_read();  // the engine has read the warp's previous box
+    __syncwarp();
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      *reinterpret_cast<float4*>(box + tc::swz128(lane, k)) = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
     tc::fence_proxy_async_smem();
     __syncwarp();
-    if (lane == 0) { tc::tma_reduce_add_2d(tmap, col0, row0, box_addr); tc::tma_store_commit(); tc::tma_store_wait_read(); }
-    __syncwarp();
+    if (lane == 0) { tc::tma_reduce_add_2d(tmap, col0, row0, box_addr); tc::tma_store_commit(); }
   }
 };

@@ -196,13 +196,23 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     float* tile_bias = reinterpret_cast<float*>(smem + SL::TILE_BIAS_OFFSET);
     bool ok = !dead;
     int it = 0;
+    // this thread's bias of the next tile is fetched one tile ahead, so its latency is off the epilogue's path
+    float next_bias = 0.f;
+    if (pair < num_tiles && etid < BN2) {
+      const int nn = (pair % tiles_n) * BN2 + etid;
+      next_bias = epi.col_const(nn, nn < N);
+    }
     for (int tile = pair; tile < num_tiles; tile += num_pairs, ++it) {
       const int m0 = (tile / tiles_n) * (2 * BM) + (int)rank * BM, n0 = (tile % tiles_n) * BN2;
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
       named_bar_sync(1, 32 * NUM_EPI_WARPS);
-      if (etid < BN2) tile_bias[etid] = epi.col_const(n0 + etid, n0 + etid < N);
+      if (etid < BN2) tile_bias[etid] = next_bias;
       named_bar_sync(1, 32 * NUM_EPI_WARPS);
+      if (tile + num_pairs < num_tiles && etid < BN2) {
+        const int nn = ((tile + num_pairs) % tiles_n) * BN2 + etid;
+        next_bias = epi.col_const(nn, nn < N);
+      }
       if (ok && !mbar_wait(tfull_bar(acc), acc_phase, err, TFERR_WAIT_TMEM_FULL)) ok = false;
       if (!ok) continue;
       tcgen05_fence_after();
