@@ -215,17 +215,21 @@ seq_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W, int B, i
 //   * the four warps read their 32 TMEM lanes (lane = output column n), transpose through shared memory
 //     and store part[ks][b][n] with 16-byte stores, 512 contiguous bytes per warp.
 //   grid = (ceil(N / 128), (K / 64) / kbn, ceil(B / RT)), 128 threads, RT in {16, 32, 64}.
+// When the whole reduction fits the CTA's slab buffers (K <= 64 NS, one K slice) the kernel can finish the output
+// itself: bf16(GELU(sum + bias)) for the MLP hidden layer, so no partial tiles and no consumer kernel are needed.
 // Every wait is bounded (see gemm_tc.cuh); a wait that expires records a code in *err and the CTA
 // leaves without storing.
 // ---------------------------------------------------------------------------------------------
-template <int RT>
-__host__ __device__ constexpr int gemm_tc_smem_bytes() { return 4 * (128 * 64 * 2 + RT * 64 * 2) + 64 + 1024; }
+// NS = slab buffers (kbn <= NS).  With gelu_out != null (one K slice only: gridDim.y == 1) the CTA holds finished
+// sums and writes bf16(GELU(sum + bias)) itself instead of a partial tile, which saves the consumer kernel.
+template <int RT, int NS = 4>
+__host__ __device__ constexpr int gemm_tc_smem_bytes() { return NS * (128 * 64 * 2 + RT * 64 * 2) + 128 + 1024; }
 
-template <int RT>
+template <int RT, int NS = 4>
 __global__ void __launch_bounds__(128)
 seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a, int B, int N, int kbn,
                    float* __restrict__ part, const int* __restrict__ step_base, int step_off, int n_steps, int check_steps,
-                   int* err) {
+                   int* err, const float* __restrict__ gelu_bias, bf16* __restrict__ gelu_out) {
   using namespace tc;
   pdl_launch_dependents();
   constexpr int W_BYTES = 128 * 64 * 2, A_BYTES = RT * 64 * 2, STAGE = W_BYTES + A_BYTES;
@@ -233,14 +237,14 @@ seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   extern __shared__ uint8_t smem_seq_tc[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_seq_tc) + 1023) & ~(uintptr_t)1023);
   const uint32_t smem_base = smem_u32(smem);
-  const uint32_t bar_base = smem_base + 4 * STAGE;  // full[0..3], done
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + 4 * STAGE + 48);
+  const uint32_t bar_base = smem_base + NS * STAGE;  // full[0..NS-1], done
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + NS * STAGE + 96);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * 128, ks = blockIdx.y, row0 = blockIdx.z * RT;
   const int k0 = ks * kbn * 64;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 5; ++i) mbar_init(bar_base + 8u * i, 1);
+    for (int i = 0; i < NS + 1; ++i) mbar_init(bar_base + 8u * i, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -275,9 +279,9 @@ seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
 #pragma unroll
       for (int k = 0; k < 4; ++k) umma_f16(tmem_base, wdesc + 2u * k, adesc + 2u * k, idesc, (kb | k) != 0);
     }
-    if (ok) umma_commit(bar_base + 8u * 4);
+    if (ok) umma_commit(bar_base + 8u * NS);
   }
-  ok = mbar_wait(bar_base + 8u * 4, 0u, err, TFERR_WAIT_TMEM_FULL);
+  ok = mbar_wait(bar_base + 8u * NS, 0u, err, TFERR_WAIT_TMEM_FULL);
   tcgen05_fence_after();
   // TMEM (lane = output column) -> shared memory tile [RT rows][128 columns] in the operand stages, which are
   // free once the MMAs have completed -> 16-byte stores, 512 contiguous bytes per warp
@@ -298,14 +302,29 @@ seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     const int nrows = (B - row0) < RT ? (B - row0) : RT;
     const int n = n0 + 4 * lane;
     float* out = part + ((size_t)ks * B + row0) * N + n;
-    for (int r = warp; r < nrows; r += 4) {
-      const float4 x = *reinterpret_cast<const float4*>(tile + r * TP + 4 * lane);
-      if (n + 3 < N) {
-        *reinterpret_cast<float4*>(out + (size_t)r * N) = x;
-      } else {
-        if (n < N) out[(size_t)r * N] = x.x;
-        if (n + 1 < N) out[(size_t)r * N + 1] = x.y;
-        if (n + 2 < N) out[(size_t)r * N + 2] = x.z;
+    if (gelu_out != nullptr) {  // N % 4 == 0 here
+      if (n < N) {
+        const float4 bj = *reinterpret_cast<const float4*>(gelu_bias + n);
+        for (int r = warp; r < nrows; r += 4) {
+          const float4 x = *reinterpret_cast<const float4*>(tile + r * TP + 4 * lane);
+          const __nv_bfloat162 o0 = __floats2bfloat162_rn(gelu_erf(bj.x + x.x), gelu_erf(bj.y + x.y));
+          const __nv_bfloat162 o1 = __floats2bfloat162_rn(gelu_erf(bj.z + x.z), gelu_erf(bj.w + x.w));
+          uint2 w2;
+          w2.x = *reinterpret_cast<const uint32_t*>(&o0);
+          w2.y = *reinterpret_cast<const uint32_t*>(&o1);
+          *reinterpret_cast<uint2*>(gelu_out + (size_t)(row0 + r) * N + n) = w2;
+        }
+      }
+    } else {
+      for (int r = warp; r < nrows; r += 4) {
+        const float4 x = *reinterpret_cast<const float4*>(tile + r * TP + 4 * lane);
+        if (n + 3 < N) {
+          *reinterpret_cast<float4*>(out + (size_t)r * N) = x;
+        } else {
+          if (n < N) out[(size_t)r * N] = x.x;
+          if (n + 1 < N) out[(size_t)r * N + 1] = x.y;
+          if (n + 2 < N) out[(size_t)r * N + 2] = x.z;
+        }
       }
     }
   }

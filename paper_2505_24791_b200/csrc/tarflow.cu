@@ -163,6 +163,8 @@ struct tf_model {
   CUtensorMap map_seq_a[3][3];  // sequential-step GEMM operands {xn, att, mlp} x row tile {16, 32, 64}
   bool use_pair_gemm = true;    // sweep GEMMs on 2-CTA tile pairs (false: one CTA per tile)
   bool seq_use_tc = true;       // sequential-step GEMMs on tcgen05 (false: the mma.sync kernel)
+  bool seq_fuse_gelu = false;   // MLP-up step GEMM with K <= 512 applies bias + GELU itself (no K split): one kernel
+                                // less per layer, but 16 CTAs instead of 64 stream the weights; measured slower
   int *idx = nullptr, *idx_tmp = nullptr, *phase = nullptr, *ctrl = nullptr, *iters_sample = nullptr, *err = nullptr;
   // precision policy of Jacobi blocks on the bf16 engine: 0 = escalate per sample, 1 = single bf16
   // operands only, 2 = two-term operands for every sweep
@@ -544,10 +546,21 @@ static int launch_seq(tf_model* m, int cls, void (*kern)(KArgs...), dim3 grid, i
 // One skinny GEMM of a decoding step: part[ks][B, N] = A[B, K slice ks] W[N, K slice ks]^T.  Returns the number of
 // K slices in *nsplit; the kernel that consumes the tiles adds them up.  CTAs of 64 columns x 256 of K read as many
 // activation bytes as weight bytes and give a grid of (N / 64) * (K / 256) CTAs.
-static int seq_gemm(tf_model* m, int cls, int abuf, const Matrix& W, int B, int step_off, int* nsplit) {
+// gelu_bias / gelu_out non-null: the caller wants bf16(GELU(product + bias)) in gelu_out.  When the whole reduction
+// fits one CTA (K <= 512) the GEMM writes that itself and *nsplit = 0; otherwise it writes partial tiles as usual
+// and the caller runs the bias + GELU kernel.
+static int seq_gemm(tf_model* m, int cls, int abuf, const Matrix& W, int B, int step_off, int* nsplit,
+                    const float* gelu_bias = nullptr, bf16* gelu_out = nullptr) {
   const int N = W.N, K = W.K, n_steps = m->L - 1;
   const bf16* A = reinterpret_cast<const bf16*>(abuf == 0 ? m->xn : abuf == 1 ? m->att : m->mlp);
   const bf16* w = reinterpret_cast<const bf16*>(W.w);
+  if (m->seq_use_tc && gelu_out != nullptr && m->seq_fuse_gelu && K % 64 == 0 && K / 64 <= 8 && N % 4 == 0) {
+    *nsplit = 0;
+    dim3 grid((N + 127) / 128, 1, (B + 63) / 64);
+    return launch_seq(m, cls, seq::seq_gemm_tc_kernel<64, 8>, grid, 128, seq::gemm_tc_smem_bytes<64, 8>(), W.map_seq,
+                      m->map_seq_a[abuf][2], B, N, K / 64, m->seq_part, m->step_ctr, step_off, n_steps, m->seq_check_steps,
+                      m->err, gelu_bias, gelu_out);
+  }
   if (m->seq_use_tc) {  // tcgen05 kernel: CTAs of 128 columns x kbn slabs of 64 k
     const int slabs = K / 64;
     int kbn = slabs % 4 == 0 ? 4 : slabs % 2 == 0 ? 2 : 1;
@@ -567,7 +580,7 @@ static int seq_gemm(tf_model* m, int cls, int abuf, const Matrix& W, int B, int 
   if (rt == RTV)                                                                                                         \
     return launch_seq(m, cls, seq::seq_gemm_tc_kernel<RTV>, grid, 128, seq::gemm_tc_smem_bytes<RTV>(), W.map_seq,         \
                       m->map_seq_a[abuf][ri], B, N, kbn, m->seq_part, m->step_ctr, step_off, n_steps, m->seq_check_steps, \
-                      m->err);
+                      m->err, (const float*)nullptr, (bf16*)nullptr);
     TF_SEQ_TC_CASE(16)
     TF_SEQ_TC_CASE(32)
     TF_SEQ_TC_CASE(64)
@@ -633,9 +646,10 @@ static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const
                         att, B, L, d, heads, scale * 1.4426950408889634f, m->step_ctr, s, L - 1));
       TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 1, lw.w_o, B, s, &pending));
       TF_TRY(seq_resid_ln(m, lw.b_o, pending, lw.ln2_g, lw.ln2_b, B, s));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 0, lw.w_1, B, s, &ns));
-      TF_TRY(launch_seq(m, KC_SEQ_LN, seq::seq_bias_gelu_kernel, dim3((B * (m->hid / 4) + 255) / 256), 256, 0, m->seq_part, ns,
-                        lw.b_1, mlp, B, m->hid, m->step_ctr, s, L - 1, m->seq_check_steps));
+      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 0, lw.w_1, B, s, &ns, lw.b_1, mlp));
+      if (ns > 0)  // the GEMM left partial tiles: sum them, add the bias, apply GELU
+        TF_TRY(launch_seq(m, KC_SEQ_LN, seq::seq_bias_gelu_kernel, dim3((B * (m->hid / 4) + 255) / 256), 256, 0, m->seq_part, ns,
+                          lw.b_1, mlp, B, m->hid, m->step_ctr, s, L - 1, m->seq_check_steps));
       TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 2, lw.w_2, B, s, &pending));
       pending_bias = lw.b_2;
     }
@@ -1020,6 +1034,8 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<32>()));
     CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<64>()));
     if (const char* e = getenv("TARFLOW_SEQ_MMA")) m->seq_use_tc = atoi(e) == 0;
+    if (const char* e = getenv("TARFLOW_SEQ_FUSE_GELU")) m->seq_fuse_gelu = atoi(e) != 0;
+    CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<64, 8>()));
     if (const char* e = getenv("TARFLOW_PAIR_GEMM")) m->use_pair_gemm = atoi(e) != 0;
     CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                attn::smem_bytes<true>()));

@@ -248,3 +248,24 @@ def test_bf16_optional_kernel_paths_agree(monkeypatch):
         assert rel_l2(x, xo) <= BF16_REL_L2, name
     assert rel_l2(outs["attn_mma"], outs["default"]) <= 5e-3
     assert rel_l2(outs["single_cta"], outs["default"]) <= 1e-4
+
+
+@pytest.mark.gpu
+def test_bf16_optional_sequential_paths_agree(monkeypatch):
+    """Sequential decoding: the step GEMM with fused bias + GELU and the mma.sync step GEMM give the default path's result."""
+    cfg = synth.config("cfg2", n_blocks=1, n_layers=2)
+    z = synth.make_latents(cfg, 19, B=5)
+    outs = {}
+    for name, env in (("default", {}), ("gelu_fused", {"TARFLOW_SEQ_FUSE_GELU": "1"}), ("mma_sync", {"TARFLOW_SEQ_MMA": "1"})):
+        for k in ("TARFLOW_SEQ_FUSE_GELU", "TARFLOW_SEQ_MMA"):
+            monkeypatch.delenv(k, raising=False)
+        for k, v in env.items():
+            monkeypatch.setenv(k, v)
+        with Model(cfg, max_batch=5) as m:      # the switches are read when the model is loaded
+            outs[name], _, _, rc = m.inverse(z, None, [0], -1.0, 3)
+            assert rc == 0 and np.isfinite(outs[name]).all()
+    xo, _ = O.model_inverse(synth.make_weights(cfg), z, None, cfg, [0], -1.0, 3)
+    for name, x in outs.items():
+        assert rel_l2(x, xo) <= BF16_REL_L2, name
+    assert rel_l2(outs["gelu_fused"], outs["default"]) <= 5e-3
+    assert rel_l2(outs["mma_sync"], outs["default"]) <= 5e-3
