@@ -37,7 +37,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # dram bytes per launch (read + write) of a kernel class from the committed ncu capture of that class;
 # None = no capture of the current kernel.  {workload: {class: bytes}}
-NCU_TRAFFIC: dict = {}
+# cfg2 / seq_gemm: mean over the 17 step-GEMM launches of one decoding step (27.44 MB read, 0 written), captured with
+# L2 flushed between replays, see profiles/seq_gemm_tc_kernel_cfg2_step.md; the algorithmic figure is 1.48 MB.
+NCU_TRAFFIC: dict = {"cfg2": {"seq_gemm": 27.44e6 / 17}}
 
 
 def peaks():
