@@ -598,6 +598,188 @@ __global__ void seq_update_embed_kernel(const float* __restrict__ part, int nspl
   h[(size_t)b * d + j] = acc + ((a0 + a1) + (a2 + a3));
 }
 
+// ---------------------------------------------------------------------------------------------
+// Tail of a decoding step in one kernel, for heads small enough that one CTA per sample can stream the head
+// matrix (2 D d bf16) itself.  CTA b does, for sample b and step t = *step_base + step_off:
+//   x    = h[b] + bias + partial tiles of the last MLP-down projection        (as seq_resid_ln_kernel)
+//   y    = bf16(LayerNorm_f(x))                                               (the head's input, rounded as xn is)
+//   o[n] = y . w_out[n, :] + b_out[n],  n < 2 D                               (warp per output, fp32 accumulation)
+//   u[b, t+1, c] = v[b, t+1, c] * exp(o[2c+1]) + o[2c]                         (Eq. 5)
+//   h[b] = embedding of that token;  xn[b] = bf16(LayerNorm_1(h[b]))          (layer 0's input of the next step)
+// With first != 0 it is the block's start instead: token 0 is copied (u = v), embedded and normalised.
+// It replaces resid_ln -> head GEMM -> update_embed -> resid_ln(layer 0), i.e. three kernel boundaries per step.
+// blockDim.x = 256, d % 4 == 0, d <= 1024; dynamic shared memory: (d + 2 D + D) floats.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float block_sum_256(float v, float* red /* [8] */, int warp, int lane) {
+  v = warp_sum(v);
+  __syncthreads();  // red free again
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += red[w];
+  return tot;
+}
+
+__global__ void __launch_bounds__(256)
+seq_tail_kernel(float* __restrict__ h, const float* __restrict__ part, const float* __restrict__ bias, int nsplit,
+                const float* __restrict__ lnf_g, const float* __restrict__ lnf_b, const bf16* __restrict__ w_out,
+                const float* __restrict__ b_out, int B, const float* __restrict__ v, float* __restrict__ u,
+                const int* __restrict__ labels, const float* __restrict__ w_in_t, const float* __restrict__ b_in,
+                const float* __restrict__ pos, const float* __restrict__ cls, const float* __restrict__ ln1_g,
+                const float* __restrict__ ln1_b, bf16* __restrict__ xn, int L, int D, int d, int reversed, int first,
+                const int* __restrict__ step_base, int step_off, int n_steps) {
+  pdl_launch_dependents();
+  extern __shared__ __align__(16) float s_tail[];
+  float* s_y = s_tail;          // [d]  head input
+  float* s_o = s_tail + d;      // [2D] head output
+  float* s_tok = s_o + 2 * D;   // [D]  new token
+  __shared__ float red[8];
+  const int b = blockIdx.x, i = threadIdx.x, warp = i >> 5, lane = i & 31;
+  const int dv = d >> 2;
+  const bool act = i < dv;
+  // constants first: they are requested before the previous kernel has finished
+  constexpr int WPRE = 12;  // rows of W_in kept in registers
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 gf = zero4, bf = zero4, g1 = zero4, b1 = zero4, bi = zero4, wpre[WPRE];
+  const float4* w4 = reinterpret_cast<const float4*>(w_in_t) + i;
+  if (act) {
+    gf = reinterpret_cast<const float4*>(lnf_g)[i];
+    bf = reinterpret_cast<const float4*>(lnf_b)[i];
+    g1 = reinterpret_cast<const float4*>(ln1_g)[i];
+    b1 = reinterpret_cast<const float4*>(ln1_b)[i];
+    bi = reinterpret_cast<const float4*>(b_in)[i];
+#pragma unroll
+    for (int c = 0; c < WPRE; ++c)
+      if (c < D) wpre[c] = w4[(size_t)c * dv];
+  }
+  // this warp's head outputs are n = warp, warp + 8, ...; the first HPRE 16-byte weight pieces of its lanes too
+  constexpr int HPRE = 8;
+  const int chunks = (d + 255) >> 8;  // 256-wide k chunks per output
+  uint4 hpre[HPRE];
+  if (!first) {
+#pragma unroll
+    for (int q = 0; q < HPRE; ++q) {
+      const int n = warp + 8 * (q / chunks), k0 = lane * 8 + 256 * (q % chunks);
+      hpre[q] = make_uint4(0u, 0u, 0u, 0u);
+      if (n < 2 * D && k0 < d) hpre[q] = ld_stream16(w_out + (size_t)n * d + k0);
+    }
+  }
+  pdl_wait();
+  const int t = *step_base + step_off;
+  if (!first && t >= n_steps) return;
+  const int l_new = first ? 0 : t + 1;
+  const size_t e0 = ((size_t)b * L + tok_index(l_new, L, reversed)) * D;
+  // everything that depends on the step index only
+  float vtok = 0.f;
+  if (i < D) vtok = v[e0 + i];
+  float4 base = zero4;
+  if (act && l_new < L - 1) {
+    const float4 po = reinterpret_cast<const float4*>(pos)[(size_t)l_new * dv + i];
+    base = make_float4(bi.x + po.x, bi.y + po.y, bi.z + po.z, bi.w + po.w);
+    if (cls != nullptr) {
+      const float4 cl = reinterpret_cast<const float4*>(cls)[(size_t)labels[b] * dv + i];
+      base.x += cl.x; base.y += cl.y; base.z += cl.z; base.w += cl.w;
+    }
+  }
+  if (!first) {
+    // residual + final LayerNorm (two-pass statistics, eps 1e-5)
+    float4 x = zero4;
+    if (act) {
+      x = __ldcg(reinterpret_cast<const float4*>(h + (size_t)b * d) + i);
+      if (nsplit > 0) {
+        const float4 add = sum_partials4(part, bias, nsplit, B, d, b, i);
+        x.x += add.x; x.y += add.y; x.z += add.z; x.w += add.w;
+      }
+    }
+    const float mean = block_sum_256((x.x + x.y) + (x.z + x.w), red, warp, lane) / d;
+    const float a0 = x.x - mean, a1 = x.y - mean, a2 = x.z - mean, a3 = x.w - mean;
+    const float sq = act ? (a0 * a0 + a1 * a1) + (a2 * a2 + a3 * a3) : 0.f;
+    const float rstd = rsqrtf(block_sum_256(sq, red, warp, lane) / d + 1e-5f);
+    if (act) {
+      const __nv_bfloat162 o0 = __floats2bfloat162_rn(a0 * rstd * gf.x + bf.x, a1 * rstd * gf.y + bf.y);
+      const __nv_bfloat162 o1 = __floats2bfloat162_rn(a2 * rstd * gf.z + bf.z, a3 * rstd * gf.w + bf.w);
+      const float2 f0 = __bfloat1622float2(o0), f1 = __bfloat1622float2(o1);
+      *reinterpret_cast<float4*>(s_y + 4 * i) = make_float4(f0.x, f0.y, f1.x, f1.y);
+    }
+    __syncthreads();
+    // head: a lane takes 8 consecutive k per 256-wide chunk of an output row
+    int q = 0;
+    for (int n = warp; n < 2 * D; n += 8) {
+      float acc = 0.f;
+      for (int ch = 0; ch < chunks; ++ch, ++q) {
+        const int k0 = lane * 8 + 256 * ch;
+        if (k0 >= d) continue;
+        uint4 wv;
+        if (q < HPRE) {
+          wv = hpre[0];
+#pragma unroll
+          for (int z = 1; z < HPRE; ++z)
+            if (q == z) wv = hpre[z];
+        } else {
+          wv = ld_stream16(w_out + (size_t)n * d + k0);
+        }
+        const __nv_bfloat162* w2 = reinterpret_cast<const __nv_bfloat162*>(&wv);
+        const float4 y0 = *reinterpret_cast<const float4*>(s_y + k0), y1 = *reinterpret_cast<const float4*>(s_y + k0 + 4);
+        const float2 c0 = __bfloat1622float2(w2[0]), c1 = __bfloat1622float2(w2[1]);
+        const float2 c2 = __bfloat1622float2(w2[2]), c3 = __bfloat1622float2(w2[3]);
+        acc = fmaf(y0.x, c0.x, acc); acc = fmaf(y0.y, c0.y, acc); acc = fmaf(y0.z, c1.x, acc); acc = fmaf(y0.w, c1.y, acc);
+        acc = fmaf(y1.x, c2.x, acc); acc = fmaf(y1.y, c2.y, acc); acc = fmaf(y1.z, c3.x, acc); acc = fmaf(y1.w, c3.y, acc);
+      }
+      acc = warp_sum(acc);
+      if (lane == 0) s_o[n] = acc + b_out[n];
+    }
+    __syncthreads();
+  }
+  // new token (Eq. 5; the first token of a block is copied)
+  for (int c = i; c < D; c += 256) {
+    float val = c == i ? vtok : v[e0 + c];
+    if (!first) val = fmaf(val, expf(s_o[2 * c + 1]), s_o[2 * c]);
+    u[e0 + c] = val;
+    s_tok[c] = val;
+  }
+  __syncthreads();
+  if (l_new >= L - 1) return;  // the last token is never fed back
+  // embedding of the token (same accumulation order as seq_update_embed_kernel) and layer 0's LayerNorm
+  float4 e = zero4;
+  if (act) {
+    float4 q0 = zero4, q1 = zero4, q2 = zero4, q3 = zero4;  // four independent chains over the token's values
+    auto add = [&](float4& acc, float tv, const float4& w) {
+      acc.x = fmaf(tv, w.x, acc.x); acc.y = fmaf(tv, w.y, acc.y); acc.z = fmaf(tv, w.z, acc.z); acc.w = fmaf(tv, w.w, acc.w);
+    };
+    const int d4 = D & ~3;
+#pragma unroll
+    for (int c = 0; c < WPRE; c += 4) {
+      if (c < d4) {
+        add(q0, s_tok[c], wpre[c]); add(q1, s_tok[c + 1], wpre[c + 1]);
+        add(q2, s_tok[c + 2], wpre[c + 2]); add(q3, s_tok[c + 3], wpre[c + 3]);
+      }
+    }
+    for (int c = WPRE; c < d4; c += 4) {
+      add(q0, s_tok[c], w4[(size_t)c * dv]); add(q1, s_tok[c + 1], w4[(size_t)(c + 1) * dv]);
+      add(q2, s_tok[c + 2], w4[(size_t)(c + 2) * dv]); add(q3, s_tok[c + 3], w4[(size_t)(c + 3) * dv]);
+    }
+    for (int c = d4; c < D; ++c) add(q0, s_tok[c], w4[(size_t)c * dv]);
+    e.x = base.x + ((q0.x + q1.x) + (q2.x + q3.x));
+    e.y = base.y + ((q0.y + q1.y) + (q2.y + q3.y));
+    e.z = base.z + ((q0.z + q1.z) + (q2.z + q3.z));
+    e.w = base.w + ((q0.w + q1.w) + (q2.w + q3.w));
+    reinterpret_cast<float4*>(h + (size_t)b * d)[i] = e;
+  }
+  const float mean = block_sum_256((e.x + e.y) + (e.z + e.w), red, warp, lane) / d;
+  const float a0 = e.x - mean, a1 = e.y - mean, a2 = e.z - mean, a3 = e.w - mean;
+  const float sq = act ? (a0 * a0 + a1 * a1) + (a2 * a2 + a3 * a3) : 0.f;
+  const float rstd = rsqrtf(block_sum_256(sq, red, warp, lane) / d + 1e-5f);
+  if (act) {
+    const __nv_bfloat162 o0 = __floats2bfloat162_rn(a0 * rstd * g1.x + b1.x, a1 * rstd * g1.y + b1.y);
+    const __nv_bfloat162 o1 = __floats2bfloat162_rn(a2 * rstd * g1.z + b1.z, a3 * rstd * g1.w + b1.w);
+    uint2 w2;
+    w2.x = *reinterpret_cast<const uint32_t*>(&o0);
+    w2.y = *reinterpret_cast<const uint32_t*>(&o1);
+    reinterpret_cast<uint2*>(xn + (size_t)b * d)[i] = w2;
+  }
+}
+
 __global__ void seq_advance_kernel(int* step_base, int by) {
   pdl_wait();  // every kernel of the replayed steps has finished reading the counter
   if (threadIdx.x == 0 && blockIdx.x == 0) *step_base += by;

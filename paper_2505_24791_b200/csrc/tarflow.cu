@@ -163,6 +163,8 @@ struct tf_model {
   CUtensorMap map_seq_a[3][3];  // sequential-step GEMM operands {xn, att, mlp} x row tile {16, 32, 64}
   bool use_pair_gemm = true;    // sweep GEMMs on 2-CTA tile pairs (false: one CTA per tile)
   bool seq_use_tc = true;       // sequential-step GEMMs on tcgen05 (false: the mma.sync kernel)
+  int seq_fuse_tail = -1;       // step tail (final LN, head, update, embed, next LN) in one kernel: -1 = when the head
+                                // matrix is at most 64 KB, 0 = never, 1 = always
   bool seq_fuse_gelu = false;   // MLP-up step GEMM with K <= 512 applies bias + GELU itself (no K split): one kernel
                                 // less per layer, but 16 CTAs instead of 64 stream the weights; measured slower
   int *idx = nullptr, *idx_tmp = nullptr, *phase = nullptr, *ctrl = nullptr, *iters_sample = nullptr, *err = nullptr;
@@ -623,6 +625,24 @@ static int seq_resid_ln(tf_model* m, const float* bias, int nsplit, const float*
                     beta, reinterpret_cast<bf16*>(m->xn), B, m->d, m->step_ctr, step_off, m->L - 1, m->seq_check_steps);
 }
 
+static bool seq_tail_fused(const tf_model* m) {
+  if (m->d % 8 != 0 || m->d > 1024) return false;
+  if (m->seq_fuse_tail >= 0) return m->seq_fuse_tail != 0;
+  return (size_t)2 * m->D * m->d * sizeof(bf16) <= 64 * 1024;
+}
+
+// the fused tail of step step_off (first = 0) or the block's start (first = 1)
+static int seq_tail(tf_model* m, int g, int B, const int* labels, const float* v, float* u, const float* pending_bias,
+                    int pending, int first, int step_off) {
+  const BlockW& bw = m->blocks[g];
+  const LayerW& l0 = bw.layers[0];
+  const int smem = (m->d + 3 * m->D) * (int)sizeof(float);
+  return launch_seq(m, KC_SEQ_UPDATE, seq::seq_tail_kernel, dim3(B), 256, smem, m->h, m->seq_part, pending_bias, pending,
+                    bw.lnf_g, bw.lnf_b, reinterpret_cast<const bf16*>(bw.w_out.w), bw.b_out, B, v, u, labels, bw.w_in_t,
+                    bw.b_in, bw.pos, bw.cls, l0.ln1_g, l0.ln1_b, reinterpret_cast<bf16*>(m->xn), m->L, m->D, m->d, g & 1, first,
+                    m->step_ctr, step_off, m->L - 1);
+}
+
 // kernels of decoding steps step_off .. step_off+count-1 relative to the device step counter
 static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const float* v, float* u, int count) {
   const BlockW& bw = m->blocks[g];
@@ -633,6 +653,7 @@ static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const
   const float scale = 1.0f / sqrtf((float)m->hd);
   const int ethreads = d < 128 ? d : 128;
   m->cur_rows = B;
+  const bool tail = seq_tail_fused(m);
   for (int s = 0; s < count; ++s) {
     const float* pending_bias = nullptr;  // bias of the projection whose partial tiles are not yet in h
     int pending = 0, ns = 0;
@@ -640,7 +661,8 @@ static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const
       const LayerW& lw = bw.layers[i];
       bf16* kc = reinterpret_cast<bf16*>(m->kcache) + i * layer_stride;
       bf16* vc = reinterpret_cast<bf16*>(m->vcache) + i * layer_stride;
-      TF_TRY(seq_resid_ln(m, pending_bias, pending, lw.ln1_g, lw.ln1_b, B, s));
+      // layer 0's input comes from the fused tail of the previous step (or of the block's start) when that is on
+      if (!(tail && i == 0)) TF_TRY(seq_resid_ln(m, pending_bias, pending, lw.ln1_g, lw.ln1_b, B, s));
       TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 0, lw.w_qkv, B, s, &ns));
       TF_TRY(launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, m->seq_part, ns, lw.b_qkv, kc, vc,
                         att, B, L, d, heads, scale * 1.4426950408889634f, m->step_ctr, s, L - 1));
@@ -652,6 +674,10 @@ static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const
                           lw.b_1, mlp, B, m->hid, m->step_ctr, s, L - 1, m->seq_check_steps));
       TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 2, lw.w_2, B, s, &pending));
       pending_bias = lw.b_2;
+    }
+    if (tail) {
+      TF_TRY(seq_tail(m, g, B, labels, v, u, pending_bias, pending, 0, s));
+      continue;
     }
     TF_TRY(seq_resid_ln(m, pending_bias, pending, bw.lnf_g, bw.lnf_b, B, s));
     TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 0, bw.w_out, B, s, &ns));
@@ -677,10 +703,13 @@ static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* label
   m->seq_check_steps = (m->prof_on || !m->use_graphs) ? 0 : (n_steps % seq_unroll(n_steps) != 0);
   CU_OK(cudaMemsetAsync(m->step_ctr, 0, sizeof(int), user));
   m->cur_rows = B;
-  TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B, (d + ethreads - 1) / ethreads), ethreads,
-                    (int)(D * sizeof(float)), m->seq_part, 0,
-                    bw.b_out, B, v, u, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 1, m->step_ctr, 0,
-                    n_steps));
+  if (seq_tail_fused(m))
+    TF_TRY(seq_tail(m, g, B, labels, v, u, nullptr, 0, 1, 0));
+  else
+    TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B, (d + ethreads - 1) / ethreads), ethreads,
+                      (int)(D * sizeof(float)), m->seq_part, 0,
+                      bw.b_out, B, v, u, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 1, m->step_ctr, 0,
+                      n_steps));
   if (m->prof_on || !m->use_graphs) {  // direct launches (per-kernel events need them)
     for (int t = 0; t < n_steps; ++t) {
       TF_TRY(seq_enqueue_steps(m, g, B, labels, v, u, 1));
@@ -1035,6 +1064,7 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<64>()));
     if (const char* e = getenv("TARFLOW_SEQ_MMA")) m->seq_use_tc = atoi(e) == 0;
     if (const char* e = getenv("TARFLOW_SEQ_FUSE_GELU")) m->seq_fuse_gelu = atoi(e) != 0;
+    if (const char* e = getenv("TARFLOW_SEQ_FUSE_TAIL")) m->seq_fuse_tail = atoi(e) != 0;
     CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<64, 8>()));
     if (const char* e = getenv("TARFLOW_PAIR_GEMM")) m->use_pair_gemm = atoi(e) != 0;
     CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -252,12 +252,13 @@ def test_bf16_optional_kernel_paths_agree(monkeypatch):
 
 @pytest.mark.gpu
 def test_bf16_optional_sequential_paths_agree(monkeypatch):
-    """Sequential decoding: the step GEMM with fused bias + GELU and the mma.sync step GEMM give the default path's result."""
+    """Sequential decoding: fused bias + GELU, the mma.sync step GEMM and the unfused step tail give the default path's result."""
     cfg = synth.config("cfg2", n_blocks=1, n_layers=2)
     z = synth.make_latents(cfg, 19, B=5)
     outs = {}
-    for name, env in (("default", {}), ("gelu_fused", {"TARFLOW_SEQ_FUSE_GELU": "1"}), ("mma_sync", {"TARFLOW_SEQ_MMA": "1"})):
-        for k in ("TARFLOW_SEQ_FUSE_GELU", "TARFLOW_SEQ_MMA"):
+    for name, env in (("default", {}), ("gelu_fused", {"TARFLOW_SEQ_FUSE_GELU": "1"}), ("mma_sync", {"TARFLOW_SEQ_MMA": "1"}),
+                      ("tail_kernels", {"TARFLOW_SEQ_FUSE_TAIL": "0"})):
+        for k in ("TARFLOW_SEQ_FUSE_GELU", "TARFLOW_SEQ_MMA", "TARFLOW_SEQ_FUSE_TAIL"):
             monkeypatch.delenv(k, raising=False)
         for k, v in env.items():
             monkeypatch.setenv(k, v)
@@ -269,3 +270,4 @@ def test_bf16_optional_sequential_paths_agree(monkeypatch):
         assert rel_l2(x, xo) <= BF16_REL_L2, name
     assert rel_l2(outs["gelu_fused"], outs["default"]) <= 5e-3
     assert rel_l2(outs["mma_sync"], outs["default"]) <= 5e-3
+    assert rel_l2(outs["tail_kernels"], outs["default"]) <= 5e-3
