@@ -37,9 +37,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # dram bytes per launch (read + write) of a kernel class from the committed ncu capture of that class;
 # None = no capture of the current kernel.  {workload: {class: bytes}}
-# cfg2 / seq_gemm: mean over the 17 step-GEMM launches of one decoding step (27.44 MB read, 0 written), captured with
-# L2 flushed between replays, see profiles/seq_gemm_tc_kernel_cfg2_step.md; the algorithmic figure is 1.48 MB.
-NCU_TRAFFIC: dict = {"cfg2": {"seq_gemm": 27.44e6 / 17}}
+# cfg2 / seq_gemm: mean over the 16 layer GEMMs of one decoding step (27.33 MB read, 0 written) in the ncu summary of
+# that kernel under profiles/, captured with L2 flushed between replays; the algorithmic figure is 1.57 MB.
+NCU_TRAFFIC: dict = {"cfg2": {"seq_gemm": 27.33e6 / 16}}
 
 
 def peaks():
@@ -67,8 +67,10 @@ def class_work(cfg, L, D):
     esz = 2 if cfg["dtype"] == 1 else 4
     bound = "tensor" if cfg["dtype"] == 1 else "alu"
     w_layer = 3 * d * d + d * d + 2 * hid * d
-    seq_launches = nl * 4 + 1
-    seq_w_bytes = (nl * w_layer + 2 * D * d) * esz / seq_launches  # mean per launch of the class
+    # a small head (<= 64 KB) is part of the one-kernel step tail, not a GEMM launch of its own
+    head_gemm = not (cfg["dtype"] == 1 and 2 * D * d * esz <= 64 * 1024)
+    seq_launches = nl * 4 + (1 if head_gemm else 0)
+    seq_w_bytes = (nl * w_layer + (2 * D * d if head_gemm else 0)) * esz / seq_launches  # mean per launch of the class
     return {
         "gemm_qkv": (bound, 2.0 * 3 * d * d, 0.0),
         "gemm_out": (bound, 2.0 * d * d, 0.0),
@@ -86,7 +88,7 @@ def class_work(cfg, L, D):
         "seq_attention": ("hbm", (L / 2.0) * 2 * d * esz, 0.0),  # mean cache rows read per step: K and V
         "seq_layernorm": ("hbm", d * (4.0 + esz), 0.0),
         "seq_embed": ("hbm", D * 4.0 + d * 4.0, 0.0),
-        "seq_update": ("hbm", D * 4.0 * 4, 0.0),
+        "seq_update": ("hbm", D * 4.0 * 4 + (0.0 if head_gemm else 2 * d * (4.0 + esz) + 2 * D * d * esz), 0.0),
         "seq_step": ("hbm", (L / 2.0) * 2 * d * esz * nl, (nl * w_layer + 2 * D * d) * esz),
     }
 

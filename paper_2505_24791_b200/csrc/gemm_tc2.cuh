@@ -105,8 +105,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const int tiles_m = (M + 2 * BM - 1) / (2 * BM), tiles_n = (N + BN2 - 1) / BN2;
   const int num_tiles = tiles_m * tiles_n;
-  const int kb_per_pass = (K + BK - 1) / BK;
-  const int kblocks = split ? 2 * kb_per_pass : kb_per_pass;
+  // split != 0: A is an error-compensated pair (hi + lo).  A stage then holds [A_hi | A_lo | W] of one k slab
+  // (48 KB, four stages in the same 192 KB), so the weight slab is fetched once for both products.
+  const int kblocks = (K + BK - 1) / BK;
+  const uint32_t stage_bytes = split ? (uint32_t)(2 * SL::A_BYTES + SL::B_BYTES) : (uint32_t)SL::STAGE_BYTES;
+  const int nstages = split ? 4 : STAGES2;
+  const uint32_t w_off = split ? 2u * SL::A_BYTES : (uint32_t)SL::A_BYTES;
   constexpr uint32_t TMEM_COLS = 2 * BN2;
 
   if (threadIdx.x == 0) {
@@ -147,13 +151,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int m0 = (tile / tiles_n) * (2 * BM) + (int)rank * BM, n0 = (tile % tiles_n) * BN2 + (int)rank * (BN2 / 2);
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, err, TFERR_WAIT_EMPTY)) { ok = false; break; }
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * SL::STAGE_BYTES);
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * stage_bytes);
           const uint32_t lead_full = map_to_cta(full_bar(stage), 0);
-          const uint32_t sa = smem_base + stage * SL::STAGE_BYTES;
-          const int kk = (kb >= kb_per_pass ? kb - kb_per_pass : kb) * BK;
-          tma_load_2d_pair(sa, kb >= kb_per_pass ? &map_a_lo : &map_a, kk, m0, lead_full);
-          tma_load_2d_pair(sa + SL::A_BYTES, &map_w, kk, n0, lead_full);
-          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
+          const uint32_t sa = smem_base + stage * stage_bytes;
+          const int kk = kb * BK;
+          tma_load_2d_pair(sa, &map_a, kk, m0, lead_full);
+          if (split) tma_load_2d_pair(sa + SL::A_BYTES, &map_a_lo, kk, m0, lead_full);
+          tma_load_2d_pair(sa + w_off, &map_w, kk, n0, lead_full);
+          if (++stage == nstages) { stage = 0; phase ^= 1u; }
         }
       }
     }
@@ -174,12 +179,17 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, err, TFERR_WAIT_FULL)) { ok = false; break; }
           tcgen05_fence_after();
-          const uint32_t sa = smem_base + stage * SL::STAGE_BYTES;
-          const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sa + SL::A_BYTES);
+          const uint32_t sa = smem_base + stage * stage_bytes;
+          const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sa + w_off);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) umma_f16_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0);
+          if (split) {  // the low halves against the same weight slab, into the same accumulator
+            const uint64_t ldesc = make_smem_desc(sa + SL::A_BYTES);
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k) umma_f16_pair(d_tmem, ldesc + 2u * k, bdesc + 2u * k, idesc, 1u);
+          }
           umma_commit_pair(empty_bar(stage));  // frees the stage in both CTAs
-          if (++stage == STAGES2) { stage = 0; phase ^= 1u; }
+          if (++stage == nstages) { stage = 0; phase ^= 1u; }
         }
         if (ok) umma_commit_pair(tfull_bar(acc));  // accumulator complete, in both CTAs
       }
