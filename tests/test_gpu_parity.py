@@ -206,6 +206,45 @@ def test_bf16_small_model_selective_parity():
     assert np.abs(its - ito).max() <= 1
 
 
+def test_bf16_cfg2_full_batch_sampled_against_oracle():
+    """The benchmark's launch configuration (cfg2, batch 64, selective policy, tau 1e-3): three samples of the
+    batch are checked against the oracle one by one (samples are independent: per-sample stopping test), the
+    rest through properties that hold at any size."""
+    cfg = synth.config("cfg2")
+    B = cfg["B"]
+    policy = [0] + [1] * (cfg["n_blocks"] - 1)
+    with Model(cfg, max_batch=B) as m:
+        z = synth.make_latents(cfg, 1000, B=B)
+        x, ib, its, rc = m.inverse(z, None, policy, cfg["tau"], m.L + 1)
+        assert rc == 0 and np.isfinite(x).all()
+        assert (its[0] == m.L - 1).all()                       # the sequential block reports L - 1 steps
+        assert (its[1:] >= 2).all() and (its[1:] <= m.L).all()  # Jacobi: at least two sweeps, at most L (Prop. 3.2)
+        pick = [0, 37, B - 1]
+        xo, ito = O.model_inverse(m.blocks, z[pick], None, cfg, policy, cfg["tau"], m.L + 1)
+        assert rel_l2(x[pick], xo) <= BF16_REL_L2
+        assert np.abs(its[:, pick] - ito).max() <= 1
+        x2, _, its2, rc2 = m.inverse(z, None, policy, cfg["tau"], m.L + 1)  # run-twice determinism
+        assert rc2 == 0 and np.array_equal(x, x2) and np.array_equal(its, its2)
+
+
+def test_bf16_cfg3_full_batch_sampled_against_oracle():
+    """cfg3 at its full size (8 blocks x 8 layers, width 1024, 1000 classes, batch 64): one sample of the batch
+    against the oracle (about 45 s of CPU), sweep-count properties for all."""
+    cfg = synth.config("cfg3")
+    B = cfg["B"]
+    policy = [0] + [1] * (cfg["n_blocks"] - 1)
+    lab = synth.make_labels(cfg, B=B)
+    with Model(cfg, max_batch=B) as m:
+        z = synth.make_latents(cfg, 1000, B=B)
+        x, ib, its, rc = m.inverse(z, lab, policy, cfg["tau"], m.L + 1)
+        assert rc == 0 and np.isfinite(x).all()
+        assert (its[0] == m.L - 1).all() and (its[1:] >= 2).all() and (its[1:] <= m.L).all()
+        pick = [41]
+        xo, ito = O.model_inverse(m.blocks, z[pick], lab[pick], cfg, policy, cfg["tau"], m.L + 1)
+        assert rel_l2(x[pick], xo) <= BF16_REL_L2
+        assert np.abs(its[:, pick] - ito).max() <= 1
+
+
 def test_bf16_all_jacobi_and_all_sequential_agree_with_oracle():
     cfg = synth.config("cfg2", n_blocks=2, n_layers=2)
     with Model(cfg, max_batch=3) as m:
