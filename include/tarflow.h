@@ -28,8 +28,8 @@
  *     the column-slice width of the mma.sync step GEMM, TARFLOW_SEQ_FUSE_GELU=1 lets the MLP-up step GEMM
  *     apply bias + GELU itself when its reduction fits one CTA (K <= 512), TARFLOW_SEQ_FUSE_TAIL=0|1 switches the one-kernel
  *     step tail (final LayerNorm, head, update, embedding, next LayerNorm) off or on whatever the head's size.  Sweeps: TARFLOW_PAIR_GEMM=0 runs the projections with
- *     one CTA per 128x256 tile instead of 2-CTA pairs; TARFLOW_ATTN_TC=0 runs single-operand attention on the
- *     mma.sync kernel instead of the tcgen05 one.
+ *     one CTA per 128x256 tile instead of 2-CTA pairs; TARFLOW_ATTN_TC=0 runs attention on the mma.sync kernel
+ *     instead of the tcgen05 one, TARFLOW_ATTN_TC_SPLIT=0 does so for two-term operands only.
  */
 #ifndef TARFLOW_H_
 #define TARFLOW_H_

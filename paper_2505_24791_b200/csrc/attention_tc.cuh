@@ -29,9 +29,17 @@ using namespace tc;
 constexpr int BQ = 128, BKV = 64, HD = 64;
 constexpr int NUM_THREADS_ATTN = 192;  // warp 0 TMA, warp 1 MMA + TMEM, warps 2..5 softmax / epilogue
 constexpr int Q_BYTES = BQ * HD * 2, K_BYTES = BKV * HD * 2, V_BYTES = BKV * HD * 2, P_BYTES = BQ * BKV * 2;
-constexpr int KV_STAGES = 2;  // K and V tiles in flight ahead of the tensor core
-constexpr int KV_RING = KV_STAGES * (K_BYTES + V_BYTES);
-constexpr int SMEM_BYTES = Q_BYTES + KV_RING + P_BYTES + 256 + 1024;
+// SPLIT: every operand is an error-compensated bf16 pair (hi + lo) and every product keeps hi*hi + lo*hi + hi*lo;
+// the low halves sit directly behind the high halves of Q, of each K / V ring slot and of P.
+template <bool SPLIT>
+struct Cfg {
+  static constexpr int NT = SPLIT ? 2 : 1;           // tiles per operand
+  static constexpr int KV_STAGES = SPLIT ? 1 : 2;    // K and V tiles in flight ahead of the tensor core
+  static constexpr int Q_ALL = NT * Q_BYTES, K_SLOT = NT * K_BYTES, V_SLOT = NT * V_BYTES, P_ALL = NT * P_BYTES;
+  static constexpr int KV_RING = KV_STAGES * (K_SLOT + V_SLOT);
+  static constexpr int SMEM_BYTES = Q_ALL + KV_RING + P_ALL + 256 + 1024;
+  static constexpr int CTAS_PER_SM = SPLIT ? 2 : 3;
+};
 constexpr uint32_t TMEM_COLS_ATTN = 128;  // S at column 0, the output accumulator at column 64
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
@@ -78,22 +86,26 @@ __host__ __device__ constexpr uint32_t make_idesc_attn(int m, int n, int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-__global__ void __launch_bounds__(NUM_THREADS_ATTN, 3)
+template <bool SPLIT>
+__global__ void __launch_bounds__(NUM_THREADS_ATTN, Cfg<SPLIT>::CTAS_PER_SM)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_kv,
-                    const CUtensorMap* __restrict__ map_out, int L, int d,
+                    const __grid_constant__ CUtensorMap map_qkv_lo, const __grid_constant__ CUtensorMap map_kv_lo,
+                    const CUtensorMap* __restrict__ map_out, const CUtensorMap* __restrict__ map_out_lo, int L, int d,
                     float scale_log2e, int* err) {
+  using C = Cfg<SPLIT>;
+  constexpr int KV_STAGES = C::KV_STAGES, KV_RING = C::KV_RING;
   extern __shared__ uint8_t smem_attn_raw[];
   pdl_launch_dependents();  // the next kernel of the stream may be scheduled; it waits for this one to complete
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_attn_raw) + 1023) & ~(uintptr_t)1023);
-  const uint32_t sQ = smem_u32(smem), sK = sQ + Q_BYTES, sV = sK + KV_STAGES * K_BYTES, sP = sV + KV_STAGES * V_BYTES;
-  const uint32_t bar_base = sP + P_BYTES;
+  const uint32_t sQ = smem_u32(smem), sK = sQ + C::Q_ALL, sV = sK + KV_STAGES * C::K_SLOT, sP = sV + KV_STAGES * C::V_SLOT;
+  const uint32_t bar_base = sP + C::P_ALL;
   // barriers: 0 q_full, then k_full[st], k_empty[st], v_full[st], v_empty[st], s_full, s_free, p_ready, o_done
   constexpr int B_KFULL = 1, B_KEMPTY = B_KFULL + KV_STAGES, B_VFULL = B_KEMPTY + KV_STAGES, B_VEMPTY = B_VFULL + KV_STAGES,
                 B_SFULL = B_VEMPTY + KV_STAGES, B_SFREE = B_SFULL + 1, B_PREADY = B_SFREE + 1, B_ODONE = B_PREADY + 1,
                 NUM_BARS = B_ODONE + 1;
   static_assert(NUM_BARS * 8 <= 192, "barrier area");
   auto bar = [&](int i) { return bar_base + 8u * i; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + Q_BYTES + KV_RING + P_BYTES + 192);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + C::Q_ALL + KV_RING + C::P_ALL + 192);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_qt = (L + BQ - 1) / BQ;
   const int qt = n_qt - 1 - (int)blockIdx.x;  // longest tiles first
@@ -121,18 +133,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0 && !dead) {
-      mbar_arrive_expect_tx(bar(0), Q_BYTES);
+      mbar_arrive_expect_tx(bar(0), C::Q_ALL);
       tma_load_3d(sQ, &map_qkv, head * HD, q0, slot, bar(0));
+      if constexpr (SPLIT) tma_load_3d(sQ + Q_BYTES, &map_qkv_lo, head * HD, q0, slot, bar(0));
       bool ok = true;
       int st = 0;
       uint32_t ph = 0;
       for (int j = 0; j < n_kv && ok; ++j) {
         if (!mbar_wait(bar(B_KEMPTY + st), ph ^ 1u, err, TFERR_WAIT_EMPTY)) { ok = false; break; }
-        mbar_arrive_expect_tx(bar(B_KFULL + st), K_BYTES);
-        tma_load_3d(sK + st * K_BYTES, &map_kv, d + head * HD, j * BKV, slot, bar(B_KFULL + st));
+        mbar_arrive_expect_tx(bar(B_KFULL + st), C::K_SLOT);
+        tma_load_3d(sK + st * C::K_SLOT, &map_kv, d + head * HD, j * BKV, slot, bar(B_KFULL + st));
+        if constexpr (SPLIT) tma_load_3d(sK + st * C::K_SLOT + K_BYTES, &map_kv_lo, d + head * HD, j * BKV, slot, bar(B_KFULL + st));
         if (!mbar_wait(bar(B_VEMPTY + st), ph ^ 1u, err, TFERR_WAIT_EMPTY)) { ok = false; break; }
-        mbar_arrive_expect_tx(bar(B_VFULL + st), V_BYTES);
-        tma_load_3d(sV + st * V_BYTES, &map_kv, 2 * d + head * HD, j * BKV, slot, bar(B_VFULL + st));
+        mbar_arrive_expect_tx(bar(B_VFULL + st), C::V_SLOT);
+        tma_load_3d(sV + st * C::V_SLOT, &map_kv, 2 * d + head * HD, j * BKV, slot, bar(B_VFULL + st));
+        if constexpr (SPLIT) tma_load_3d(sV + st * C::V_SLOT + V_BYTES, &map_kv_lo, 2 * d + head * HD, j * BKV, slot, bar(B_VFULL + st));
         if (++st == KV_STAGES) { st = 0; ph ^= 1u; }
       }
     }
@@ -146,9 +161,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
         const int st = j % KV_STAGES;
         if (!mbar_wait(bar(B_KFULL + st), (uint32_t)((j / KV_STAGES) & 1), err, TFERR_WAIT_FULL)) return false;
         tcgen05_fence_after();
-        const uint64_t kdesc = make_smem_desc(sK + st * K_BYTES);
+        const uint64_t kdesc = make_smem_desc(sK + st * C::K_SLOT);
 #pragma unroll
         for (int k = 0; k < HD / UMMA_K; ++k) umma_f16(tmem_base, qdesc + 2u * k, kdesc + 2u * k, idesc_s, k != 0);
+        if constexpr (SPLIT) {  // + Q_lo K_hi^T + Q_hi K_lo^T
+          const uint64_t qldesc = make_smem_desc(sQ + Q_BYTES), kldesc = make_smem_desc(sK + st * C::K_SLOT + K_BYTES);
+#pragma unroll
+          for (int k = 0; k < HD / UMMA_K; ++k) umma_f16(tmem_base, qldesc + 2u * k, kdesc + 2u * k, idesc_s, 1u);
+#pragma unroll
+          for (int k = 0; k < HD / UMMA_K; ++k) umma_f16(tmem_base, qdesc + 2u * k, kldesc + 2u * k, idesc_s, 1u);
+        }
         umma_commit(bar(B_KEMPTY + st));  // K buffer free
         umma_commit(bar(B_SFULL));        // S complete
         return true;
@@ -169,8 +191,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
         for (int k = 0; k < BKV / UMMA_K; ++k) {
           // P: [128 rows][128 B] (64 keys), 16 keys = 32 bytes along a row.  V: 16 keys = 2048 bytes.
           const uint64_t pdesc = make_smem_desc(sP) + 2u * k;
-          const uint64_t vdesc = make_smem_desc_mn(sV + st * V_BYTES + k * (UMMA_K * 128));
+          const uint64_t vdesc = make_smem_desc_mn(sV + st * C::V_SLOT + k * (UMMA_K * 128));
           umma_f16(tmem_base + BKV, pdesc, vdesc, idesc_o, (j | k) != 0);
+        }
+        if constexpr (SPLIT) {  // + P_lo V_hi + P_hi V_lo
+#pragma unroll
+          for (int k = 0; k < BKV / UMMA_K; ++k) {
+            const uint64_t pldesc = make_smem_desc(sP + P_BYTES) + 2u * k;
+            const uint64_t vdesc = make_smem_desc_mn(sV + st * C::V_SLOT + k * (UMMA_K * 128));
+            umma_f16(tmem_base + BKV, pldesc, vdesc, idesc_o, 1u);
+          }
+#pragma unroll
+          for (int k = 0; k < BKV / UMMA_K; ++k) {
+            const uint64_t pdesc = make_smem_desc(sP) + 2u * k;
+            const uint64_t vldesc = make_smem_desc_mn(sV + st * C::V_SLOT + V_BYTES + k * (UMMA_K * 128));
+            umma_f16(tmem_base + BKV, pdesc, vldesc, idesc_o, 1u);
+          }
         }
         umma_commit(bar(B_VEMPTY + st));  // V buffer free
         umma_commit(bar(B_ODONE));        // products up to tile j complete (and P free)
@@ -183,7 +219,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
     const int qpos = q0 + r;                   // position in the sequence
     const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
     const uint32_t t_o = t_row + BKV;          // this row's slice of the output accumulator
-    uint8_t* sPg = smem + Q_BYTES + KV_RING;
+    uint8_t* sPg = smem + C::Q_ALL + KV_RING;
     // m_run is the reference maximum of the row (in raw score units); it trails the true running maximum by at
     // most kLazy / scale_log2e, so probabilities stay below 2^kLazy and the accumulator is rescaled only rarely
     constexpr float kLazy = 8.f;
@@ -233,7 +269,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
       float2 lsum = make_float2(0.f, 0.f);
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
-        uint32_t pk[4];
+        uint32_t pk[4], pl[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           float2 e = ffma2(make_float2(s[8 * q + 2 * i], s[8 * q + 2 * i + 1]), sc2, mb2);
@@ -242,8 +278,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
           lsum = fadd2(lsum, e);
           const __nv_bfloat162 pb = __floats2bfloat162_rn(e.x, e.y);
           pk[i] = *reinterpret_cast<const uint32_t*>(&pb);
+          if constexpr (SPLIT) {
+            const float2 hi = __bfloat1622float2(pb);
+            const __nv_bfloat162 pl2 = __floats2bfloat162_rn(e.x - hi.x, e.y - hi.y);
+            pl[i] = *reinterpret_cast<const uint32_t*>(&pl2);
+          }
         }
         *reinterpret_cast<uint4*>(sPg + swz128(r, q)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        if constexpr (SPLIT) *reinterpret_cast<uint4*>(sPg + P_BYTES + swz128(r, q)) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
       }
       l_run += lsum.x + lsum.y;
       fence_proxy_async_smem();
@@ -291,6 +333,28 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_co
         tma_store_3d(map_out, head * HD, q0 + quad * 32, slot, smem_u32(box));
         tma_store_commit();
         tma_store_wait_all();
+      }
+      if constexpr (SPLIT) {  // the low half of the output pair through the same box
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          uint32_t w[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float v0 = o[8 * k + 2 * i] * inv, v1 = o[8 * k + 2 * i + 1] * inv;
+            const float2 hi = __bfloat1622float2(__floats2bfloat162_rn(v0, v1));
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(v0 - hi.x, v1 - hi.y);
+            w[i] = *reinterpret_cast<const uint32_t*>(&lo);
+          }
+          *reinterpret_cast<uint4*>(box + swz128(lane, k)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && q0 + quad * 32 < L) {
+          tma_store_3d(map_out_lo, head * HD, q0 + quad * 32, slot, smem_u32(box));
+          tma_store_commit();
+          tma_store_wait_all();
+        }
       }
     }
   }

@@ -156,9 +156,10 @@ struct tf_model {
   void *xn = nullptr, *qkv = nullptr, *att = nullptr, *mlp = nullptr, *kcache = nullptr, *vcache = nullptr;
   void *xn_lo = nullptr, *qkv_lo = nullptr, *att_lo = nullptr, *mlp_lo = nullptr;  // second terms (bf16 engine)
   CUtensorMap map_xn, map_att, map_mlp, map_xn_lo, map_att_lo, map_mlp_lo;
-  enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_ATT3, SM_COUNT };
-  CUtensorMap map_qkv3, map_kv3;  // qkv as [slot][position][3d] for the tensor-core attention (query / key boxes)
+  enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_ATT3, SM_ATT3_LO, SM_COUNT };
+  CUtensorMap map_qkv3, map_kv3, map_qkv3_lo, map_kv3_lo;  // qkv as [slot][position][3d] for the tensor-core attention (query / key boxes)
   bool use_tc_attention = true;   // single-operand attention on tcgen05 (TARFLOW_ATTN_TC=0: the mma.sync kernel)
+  bool use_tc_attention_split = true;  // two-term attention on tcgen05 too (TARFLOW_ATTN_TC_SPLIT=0: mma.sync)
   CUtensorMap* store_maps = nullptr;  // device copy of the bulk-store maps of qkv, qkv_lo, mlp, mlp_lo, h
   CUtensorMap map_seq_a[3][3];  // sequential-step GEMM operands {xn, att, mlp} x row tile {16, 32, 64}
   bool use_pair_gemm = true;    // sweep GEMMs on 2-CTA tile pairs (false: one CTA per tile)
@@ -440,13 +441,18 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
     if constexpr (sizeof(T) == 2) {
       dim3 grid((L + attn::BQ - 1) / attn::BQ, m->cfg.n_heads, n_slots);
       const float sl2 = 1.4426950408889634f / sqrtf((float)m->hd);
-      if (hp)
+      const dim3 grid_tc((L + attn_tc::BQ - 1) / attn_tc::BQ, m->cfg.n_heads, n_slots);
+      if (hp && m->use_tc_attention && m->use_tc_attention_split)
+        LAUNCH_PDL(m, KC_ATTN, attn_tc::attention_tc_kernel<true>, grid_tc, attn_tc::NUM_THREADS_ATTN, attn_tc::Cfg<true>::SMEM_BYTES,
+                   m->map_qkv3, m->map_kv3, m->map_qkv3_lo, m->map_kv3_lo, m->store_maps + tf_model::SM_ATT3,
+                   m->store_maps + tf_model::SM_ATT3_LO, L, d, sl2, m->err);
+      else if (hp)
         LAUNCH(m, KC_ATTN, attn::attention_mma_kernel<true>, grid, 128, attn::smem_bytes<true>(), qkv, qkv_lo, att,
                att_lo, L, d, sl2);
       else if (m->use_tc_attention)
-        LAUNCH_PDL(m, KC_ATTN, attn_tc::attention_tc_kernel, dim3((L + attn_tc::BQ - 1) / attn_tc::BQ, m->cfg.n_heads, n_slots),
-               attn_tc::NUM_THREADS_ATTN, attn_tc::SMEM_BYTES, m->map_qkv3, m->map_kv3, m->store_maps + tf_model::SM_ATT3, L, d, sl2,
-               m->err);
+        LAUNCH_PDL(m, KC_ATTN, attn_tc::attention_tc_kernel<false>, grid_tc, attn_tc::NUM_THREADS_ATTN, attn_tc::Cfg<false>::SMEM_BYTES,
+                   m->map_qkv3, m->map_kv3, m->map_qkv3, m->map_kv3, m->store_maps + tf_model::SM_ATT3,
+                   m->store_maps + tf_model::SM_ATT3, L, d, sl2, m->err);
       else
         LAUNCH(m, KC_ATTN, attn::attention_mma_kernel<false>, grid, 128, attn::smem_bytes<false>(), qkv, qkv_lo, att,
                att_lo, L, d, sl2);
@@ -1048,7 +1054,14 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
       TF_TRY(make_map_3d(&sm[tf_model::SM_ATT3], m->att, B, L, d, 32));
       TF_TRY(make_map_3d(&m->map_qkv3, m->qkv, B, L, 3 * (uint64_t)d, attn_tc::BQ));
       TF_TRY(make_map_3d(&m->map_kv3, m->qkv, B, L, 3 * (uint64_t)d, attn_tc::BKV));
-      CU_OK(cudaFuncSetAttribute(attn_tc::attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_tc::SMEM_BYTES));
+      TF_TRY(make_map_3d(&sm[tf_model::SM_ATT3_LO], m->att_lo, B, L, d, 32));
+      TF_TRY(make_map_3d(&m->map_qkv3_lo, m->qkv_lo, B, L, 3 * (uint64_t)d, attn_tc::BQ));
+      TF_TRY(make_map_3d(&m->map_kv3_lo, m->qkv_lo, B, L, 3 * (uint64_t)d, attn_tc::BKV));
+      CU_OK(cudaFuncSetAttribute(attn_tc::attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 attn_tc::Cfg<false>::SMEM_BYTES));
+      CU_OK(cudaFuncSetAttribute(attn_tc::attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 attn_tc::Cfg<true>::SMEM_BYTES));
+      if (const char* e = getenv("TARFLOW_ATTN_TC_SPLIT")) m->use_tc_attention_split = atoi(e) != 0;
       if (const char* e = getenv("TARFLOW_ATTN_TC")) m->use_tc_attention = atoi(e) != 0;
       TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->store_maps), sizeof(sm)));
       CU_OK(cudaMemcpy(m->store_maps, sm, sizeof(sm), cudaMemcpyHostToDevice));

@@ -289,6 +289,27 @@ def test_bf16_optional_kernel_paths_agree(monkeypatch):
     assert rel_l2(outs["single_cta"], outs["default"]) <= 1e-4
 
 
+def test_bf16_two_term_attention_paths_agree(monkeypatch):
+    """tau mode escalates to two-term operands: the tcgen05 two-term attention (default) and the mma.sync one converge
+    to the same answer in the same number of sweeps (within one) and both match the oracle."""
+    cfg = synth.config("cfg2", n_blocks=2, n_layers=2)
+    z = synth.make_latents(cfg, 23, B=5)
+    outs = {}
+    for name, env in (("tcgen05", {}), ("mma_sync", {"TARFLOW_ATTN_TC_SPLIT": "0"})):
+        monkeypatch.delenv("TARFLOW_ATTN_TC_SPLIT", raising=False)
+        for k, v in env.items():
+            monkeypatch.setenv(k, v)
+        with Model(cfg, max_batch=5) as m:      # the switch is read when the model is loaded
+            x, _, its, rc = m.inverse(z, None, [1, 1], 1e-3, m.L + 1)
+            assert rc == 0 and np.isfinite(x).all()
+            outs[name] = (x, its)
+    xo, ito = O.model_inverse(synth.make_weights(cfg), z, None, cfg, [1, 1], 1e-3, synth.seq_len(cfg) + 1)
+    for name, (x, its) in outs.items():
+        assert rel_l2(x, xo) <= BF16_REL_L2, name
+        assert np.abs(its - ito).max() <= 1, name
+    assert rel_l2(outs["tcgen05"][0], outs["mma_sync"][0]) <= 5e-3
+
+
 @pytest.mark.gpu
 def test_bf16_optional_sequential_paths_agree(monkeypatch):
     """Sequential decoding: fused bias + GELU, the mma.sync step GEMM and the unfused step tail give the default path's result."""
