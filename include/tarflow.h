@@ -22,6 +22,12 @@
  *     passed the stopping test (x holds the last iterate; not an error); negative = error, with a
  *     message available from tf_last_error().  Nothing aborts, throws or traps.
  *   - A tf_model is not thread-safe: it owns one workspace; use it from one thread/stream at a time.
+ *   - Device-side waits (mbarrier waits inside the tensor-core kernels) are bounded by wall time (2 s).  A wait
+ *     that runs out records a code in the model's error word; kernels that see the word set return without
+ *     work.  The next synchronising call (tf_forward, tf_inverse_*) returns TF_ETIMEOUT ONCE and clears the
+ *     word: the outputs of that call are undefined, the model is usable again for the next call.
+ *   - Class labels are read from caller memory, so they are validated on the device before any kernel uses
+ *     them: an id outside [0, n_classes) makes the call return TF_EINVAL (no table is ever indexed with it).
  *   - Tuning aids read from the environment (bf16 engine, sequential decoding only; results are unchanged
  *     up to summation order): TARFLOW_SEQ_MMA=1 selects the mma.sync step GEMM instead of the tcgen05 one,
  *     TARFLOW_SEQ_KBN=1|2|4 the 64-wide k slabs per CTA of the tcgen05 step GEMM, TARFLOW_SEQ_NC=8|16|32|64
@@ -89,7 +95,8 @@ void tf_free(tf_model* m);
  * tf_forward -- data to latent, x -> z, and logdet = -sum(alpha) (paper Eq. 4 applied through
  * blocks K-1 .. 0, Eq. 1 for the log-determinant).  One causal pass per block, no iteration.
  *   x_dev [B,C,H,W] in, labels_dev [B] int32 class ids or NULL, z_dev [B,C,H,W] out,
- *   logdet_dev [B] fp32 out (may be NULL).  1 <= B <= max_batch.  Asynchronous on the stream.
+ *   logdet_dev [B] fp32 out (may be NULL).  1 <= B <= max_batch.  Synchronises the stream before returning
+ *   (that is where a device-side timeout is reported).
  */
 int tf_forward(tf_model* m, const float* x_dev, const int32_t* labels_dev, int32_t B, float* z_dev,
                float* logdet_dev, void* cuda_stream);
@@ -166,7 +173,8 @@ int tf_gemm_bf16(const void* a_dev, const void* w_dev, const float* bias_dev, fl
  *   How: the fp32 partial tiles of the K slices ((K/256) * M * N * 4 bytes) and one control word live in a
  *   static device array of TF_NOALLOC_SCRATCH_BYTES that every GPU which loads the library holds until
  *   the process exits.  A problem whose tiles do not fit is refused with TF_EINVAL and a message that
- *   names both sizes.  Requirements: M >= 1, N % 8 == 0, K % 256 == 0, pointers 16-byte aligned.
+ *   names both sizes.  Requirements: M >= 1, N % 8 == 0, K % 256 == 0, a_dev and w_dev 16-byte aligned, c_dev and
+ *   bias_dev 4-byte aligned (checked: TF_EINVAL, nothing is launched).
  *   First call on a device: looks up the array's device address (cudaGetSymbolAddress) and raises the
  *   kernel's shared-memory limit, with that device current; make this first call outside any stream capture.
  *   Sharing: all calls on a device use the one array, which keeps the contents of the previous call; the
@@ -178,8 +186,8 @@ int tf_gemm_bf16(const void* a_dev, const void* w_dev, const float* bias_dev, fl
 int tf_skinny_gemm_noalloc(const void* a_dev, const void* w_dev, const float* bias_dev, float* c_dev,
                            int32_t M, int32_t N, int32_t K, void* cuda_stream);
 
-/* tf_gemm_status -- synchronise `cuda_stream` and report whether any tf_gemm_bf16 launch so far
- * gave up on a bounded device-side wait (TF_ETIMEOUT) or all completed (TF_OK). */
+/* tf_gemm_status -- synchronise `cuda_stream` and report whether any tf_gemm_bf16 launch on the current device
+ * since the last report gave up on a bounded device-side wait (TF_ETIMEOUT, reported once) or all completed (TF_OK). */
 int tf_gemm_status(void* cuda_stream);
 
 /*
@@ -220,6 +228,14 @@ int tf_set_precision(tf_model* m, int32_t mode, float switch_threshold, float si
 int tf_trace_enable(tf_model* m, int32_t on);
 int tf_trace_read(tf_model* m, int32_t* block, int32_t* sweep, int32_t* active, float* maxdiff,
                   int32_t cap);
+
+/*
+ * tf_selftest_wait_timeout -- exercises the bounded-wait path without any fault: launches one CTA whose thread
+ * waits, for at most limit_us microseconds (1 .. 1 000 000), on an mbarrier that nothing arrives on.  The wait runs
+ * out, the kernel records its code in the model's error word and returns; the call then synchronises and returns
+ * what any synchronising call would: TF_ETIMEOUT, once, with the word cleared.  The model remains usable.
+ */
+int tf_selftest_wait_timeout(tf_model* m, int32_t limit_us, void* cuda_stream);
 
 /* tf_device_bytes -- device memory owned by the model (weights + workspace + KV cache), bytes. */
 int64_t tf_device_bytes(tf_model* m);

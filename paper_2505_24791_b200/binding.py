@@ -56,6 +56,7 @@ def lib():
         L.tf_set_precision.argtypes = [vp, i32, f32, f32]
         L.tf_trace_enable.argtypes = [vp, i32]
         L.tf_trace_read.argtypes = [vp, vp, vp, vp, vp, i32]
+        L.tf_selftest_wait_timeout.argtypes = [vp, i32, vp]
         L.tf_launch_count.argtypes = [vp]
         L.tf_launch_count.restype = C.c_int64
         L.tf_device_bytes.argtypes = [vp]
@@ -178,6 +179,10 @@ def tf_trace_read(m, cap=4096):
     md = (C.c_float * cap)()
     n = _check(lib().tf_trace_read(m, blk, swp, act, md, cap))
     return [(blk[i], swp[i], act[i], md[i]) for i in range(min(n, cap))]
+
+
+def tf_selftest_wait_timeout(m, limit_us, stream=None):
+    return _check(lib().tf_selftest_wait_timeout(m, int(limit_us), _stream(stream)))
 
 
 def tf_launch_count(m):

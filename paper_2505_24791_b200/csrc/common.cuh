@@ -14,6 +14,7 @@ enum : int {
   TFERR_WAIT_EMPTY = 2,       // TMA warp: stage never released
   TFERR_WAIT_TMEM_FULL = 3,   // epilogue: accumulator never committed
   TFERR_WAIT_TMEM_EMPTY = 4,  // MMA warp: accumulator never drained
+  TFERR_WAIT_SELFTEST = 9,    // the bounded-wait self-test (a wait nothing satisfies) ran out, as it must
 };
 
 __device__ __forceinline__ float to_f32(float x) { return x; }

@@ -56,20 +56,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false (after recording `code`) when the limit passes or another role
+// Bounded wait.  Returns false (after recording `code`) when `limit_ns` of wall time pass or another role
 // already reported a failure.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, int code) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, int* err, int code, unsigned long long limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   unsigned long long t0 = globaltimer_ns();
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((spin & 255u) == 0) {
       if (*reinterpret_cast<volatile int*>(err) != 0) return false;
-      if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+      if (globaltimer_ns() - t0 > limit_ns) {
         atomicCAS(err, 0, code);
         return false;
       }
     }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, int code) {
+  return mbar_wait_limit(bar, parity, err, code, WAIT_LIMIT_NS);
+}
+
+// Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever arrives on.  The wait runs out
+// after limit_ns, records TFERR_WAIT_SELFTEST in *err and the kernel returns normally (nothing faults or hangs).
+__global__ void wait_selftest_kernel(int* err, unsigned long long limit_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_wait_limit(smem_u32(&bar), 0u, err, TFERR_WAIT_SELFTEST, limit_ns);
   }
 }
 

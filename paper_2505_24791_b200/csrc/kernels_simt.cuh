@@ -617,6 +617,19 @@ __global__ void jacobi_begin_kernel(float* __restrict__ maxdiff, int* __restrict
   if (threadIdx.x == 0) { ctrl[0] = B; ctrl[1] = 0; ctrl[2] = 0; ctrl[3] = start_phase ? B : 0; }
 }
 
+// out[b] = labels[b] clamped to [0, n_classes); *flag is set when a label had to be clamped.
+__global__ void labels_check_kernel(const int* __restrict__ labels, int* __restrict__ out, int B, int n_classes,
+                                    int* __restrict__ flag) {
+  int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  int y = labels[b];
+  if (y < 0 || y >= n_classes) {
+    *flag = 1;
+    y = y < 0 ? 0 : n_classes - 1;
+  }
+  out[b] = y;
+}
+
 __global__ void fill_int_kernel(int* p, int n, int v) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) p[i] = v;

@@ -215,6 +215,9 @@ seq_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W, int B, i
 //   * the four warps read their 32 TMEM lanes (lane = output column n), transpose through shared memory
 //     and store part[ks][b][n] with 16-byte stores, 512 contiguous bytes per warp.
 //   grid = (ceil(N / 128), (K / 64) / kbn, ceil(B / RT)), 128 threads, RT in {16, 32, 64}.
+// The launch covers the B samples row_base .. row_base + B - 1 of the activation buffer the tensor map describes
+// (several such launches, each on its own group of samples, may run side by side); part and gelu_out are indexed
+// by the sample's position inside the group.
 // When the whole reduction fits the CTA's slab buffers (K <= 64 NS, one K slice) the kernel can finish the output
 // itself: bf16(GELU(sum + bias)) for the MLP hidden layer, so no partial tiles and no consumer kernel are needed.
 // Every wait is bounded (see gemm_tc.cuh); a wait that expires records a code in *err and the CTA
@@ -227,9 +230,9 @@ __host__ __device__ constexpr int gemm_tc_smem_bytes() { return NS * (128 * 64 *
 
 template <int RT, int NS = 4>
 __global__ void __launch_bounds__(128)
-seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a, int B, int N, int kbn,
-                   float* __restrict__ part, const int* __restrict__ step_base, int step_off, int n_steps, int check_steps,
-                   int* err, const float* __restrict__ gelu_bias, bf16* __restrict__ gelu_out) {
+seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a, int row_base, int B,
+                   int N, int kbn, float* __restrict__ part, const int* __restrict__ step_base, int step_off, int n_steps,
+                   int check_steps, int* err, const float* __restrict__ gelu_bias, bf16* __restrict__ gelu_out) {
   using namespace tc;
   pdl_launch_dependents();
   constexpr int W_BYTES = 128 * 64 * 2, A_BYTES = RT * 64 * 2, STAGE = W_BYTES + A_BYTES;
@@ -269,7 +272,7 @@ seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   bool ok = true;
   if (threadIdx.x == 0) {
     for (int kb = 0; kb < kbn; ++kb)
-      tma_load_2d(smem_base + kb * STAGE + W_BYTES, &map_a, k0 + kb * 64, row0, bar_base + 8u * kb);
+      tma_load_2d(smem_base + kb * STAGE + W_BYTES, &map_a, k0 + kb * 64, row_base + row0, bar_base + 8u * kb);
     constexpr uint32_t idesc = make_idesc(RT);
     for (int kb = 0; kb < kbn && ok; ++kb) {
       ok = mbar_wait(bar_base + 8u * kb, 0u, err, TFERR_WAIT_FULL);

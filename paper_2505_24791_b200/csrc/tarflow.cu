@@ -14,6 +14,7 @@
 #include <cstring>
 #include <map>
 #include <string>
+#include <tuple>
 #include <vector>
 
 #include "../../include/tarflow.h"
@@ -181,7 +182,13 @@ struct tf_model {
   int* labels_own = nullptr;
   cudaStream_t cap_stream = nullptr;
   struct SeqGraph { cudaGraphExec_t exec = nullptr; int unroll = 0; int nodes = 0; };
-  std::map<std::pair<int, int>, SeqGraph> seq_graphs;  // (block g, B)
+  std::map<std::tuple<int, int, int>, SeqGraph> seq_graphs;  // (block g, first sample, samples) of a chain
+  enum { MAX_CHAINS = 4 };
+  cudaStream_t seq_streams[MAX_CHAINS] = {nullptr};  // one stream per chain of a sequential block
+  cudaEvent_t seq_fork = nullptr, seq_join[MAX_CHAINS] = {nullptr};
+  int seq_chains_force = 0;  // TARFLOW_SEQ_CHAINS=1|2|4: chains per sequential block (0 = by the size of the weights)
+  int seq_kbn_force = 0;     // TARFLOW_SEQ_KBN
+  size_t seq_part_row_floats = 0;  // floats of partial tiles available per sample
   bool use_graphs = true;
   int seq_check_steps = 0;    // 1 when a replayed graph can run past the last step (kernels then test the counter)
   float* seq_part = nullptr;  // fp32 partial tiles [K slices][B][N] of the projection in flight
@@ -281,6 +288,14 @@ static int check_launch(const char* what) {
   return TF_OK;
 }
 
+// Per-device host state (kernel attributes set, error words, symbol addresses) is indexed by device ordinal.
+constexpr int kMaxDevices = 64;
+static int current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+
 template <class T>
 static int dev_alloc(tf_model* m, T** p, size_t count) {
   size_t bytes = ((count * sizeof(T)) + 255) & ~(size_t)255;
@@ -306,10 +321,12 @@ static int launch_gemm_tc(tf_model* m, int cls, cudaStream_t stream, const CUten
                           int64_t* launches) {
   using SL = tc::SmemLayout<BN, STAGES>;
   auto kern = tc::gemm_tc_kernel<BN, STAGES, Epi>;
-  static bool configured = false;  // per instantiation
-  if (!configured) {
+  static bool configured[kMaxDevices] = {false};  // per instantiation and device
+  const int dev = current_device();
+  if (dev < 0) return fail(TF_ECUDA, "no usable current device");
+  if (!configured[dev]) {
     CU_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::TOTAL));
-    configured = true;
+    configured[dev] = true;
   }
   int tiles = ((M + tc::BM - 1) / tc::BM) * ((N + BN - 1) / BN);
   int grid = tiles < num_sms ? tiles : num_sms;
@@ -325,10 +342,12 @@ template <class Epi>
 static int launch_gemm_tc2(tf_model* m, int cls, const CUtensorMap& ma, const CUtensorMap* ma_lo, const CUtensorMap& mw, int M,
                            int N, int K, const Epi& epi) {
   auto kern = tc2::gemm_tc2_kernel<Epi>;
-  static bool configured = false;  // per instantiation
-  if (!configured) {
+  static bool configured[kMaxDevices] = {false};  // per instantiation and device
+  const int dev = current_device();
+  if (dev < 0) return fail(TF_ECUDA, "no usable current device");
+  if (!configured[dev]) {
     CU_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::Smem2::TOTAL));
-    configured = true;
+    configured[dev] = true;
   }
   const int tiles = ((M + 2 * tc::BM - 1) / (2 * tc::BM)) * (N / tc2::BN2);
   int pairs = m->num_sms / 2;
@@ -551,44 +570,52 @@ static int launch_seq(tf_model* m, int cls, void (*kern)(KArgs...), dim3 grid, i
   return TF_OK;
 }
 
+// A chain decodes the samples b0 .. b0 + B - 1 of a sequential block on its own stream, with its own step counter
+// and its own region of the partial-tile buffer.  Samples are independent, so a block's batch may be split over a few
+// chains that run side by side: every kernel of a decoding step is bound by the latency of its dependent chain, not
+// by throughput, and the chains fill each other's idle time.  A sample's arithmetic does not depend on the split.
+struct SeqCtx {
+  int b0 = 0, B = 0;
+  int* step_ctr = nullptr;
+  float* part = nullptr;
+};
+
 // One skinny GEMM of a decoding step: part[ks][B, N] = A[B, K slice ks] W[N, K slice ks]^T.  Returns the number of
 // K slices in *nsplit; the kernel that consumes the tiles adds them up.  CTAs of 64 columns x 256 of K read as many
 // activation bytes as weight bytes and give a grid of (N / 64) * (K / 256) CTAs.
 // gelu_bias / gelu_out non-null: the caller wants bf16(GELU(product + bias)) in gelu_out.  When the whole reduction
 // fits one CTA (K <= 512) the GEMM writes that itself and *nsplit = 0; otherwise it writes partial tiles as usual
 // and the caller runs the bias + GELU kernel.
-static int seq_gemm(tf_model* m, int cls, int abuf, const Matrix& W, int B, int step_off, int* nsplit,
+static int seq_gemm(tf_model* m, const SeqCtx& cx, int cls, int abuf, const Matrix& W, int step_off, int* nsplit,
                     const float* gelu_bias = nullptr, bf16* gelu_out = nullptr) {
-  const int N = W.N, K = W.K, n_steps = m->L - 1;
-  const bf16* A = reinterpret_cast<const bf16*>(abuf == 0 ? m->xn : abuf == 1 ? m->att : m->mlp);
+  const int N = W.N, K = W.K, n_steps = m->L - 1, B = cx.B;
+  const bf16* A = reinterpret_cast<const bf16*>(abuf == 0 ? m->xn : abuf == 1 ? m->att : m->mlp) + (size_t)cx.b0 * K;
   const bf16* w = reinterpret_cast<const bf16*>(W.w);
+  const size_t part_cap = (size_t)B * m->seq_part_row_floats;
   if (m->seq_use_tc && gelu_out != nullptr && m->seq_fuse_gelu && K % 64 == 0 && K / 64 <= 8 && N % 4 == 0) {
     *nsplit = 0;
     dim3 grid((N + 127) / 128, 1, (B + 63) / 64);
     return launch_seq(m, cls, seq::seq_gemm_tc_kernel<64, 8>, grid, 128, seq::gemm_tc_smem_bytes<64, 8>(), W.map_seq,
-                      m->map_seq_a[abuf][2], B, N, K / 64, m->seq_part, m->step_ctr, step_off, n_steps, m->seq_check_steps,
-                      m->err, gelu_bias, gelu_out);
+                      m->map_seq_a[abuf][2], cx.b0, B, N, K / 64, cx.part, cx.step_ctr, step_off, n_steps, m->seq_check_steps,
+                      m->err, gelu_bias, gelu_out + (size_t)cx.b0 * N);
   }
   if (m->seq_use_tc) {  // tcgen05 kernel: CTAs of 128 columns x kbn slabs of 64 k
     const int slabs = K / 64;
     int kbn = slabs % 4 == 0 ? 4 : slabs % 2 == 0 ? 2 : 1;
     // two slabs per CTA (more CTAs) while the grid is below one wave and the partial tiles stay <= 16
     if (kbn == 4 && ((N + 127) / 128) * (slabs / 4) < m->num_sms && slabs / 2 <= 16) kbn = 2;
-    if (const char* e = getenv("TARFLOW_SEQ_KBN")) {
-      const int f = atoi(e);
-      if ((f == 1 || f == 2 || f == 4) && slabs % f == 0 && slabs / f <= 16) kbn = f;
-    }
+    if (m->seq_kbn_force > 0 && slabs % m->seq_kbn_force == 0 && slabs / m->seq_kbn_force <= 16) kbn = m->seq_kbn_force;
     const int ksplit = slabs / kbn;
     if (ksplit > 16) return fail(TF_EINVAL, "sequential decoding: reduction length %d not supported", K);
     *nsplit = ksplit;
-    if ((size_t)ksplit * B * N > m->seq_part_floats) return fail(TF_EINVAL, "sequential decoding: partial-tile buffer too small");
+    if ((size_t)ksplit * B * N > part_cap) return fail(TF_EINVAL, "sequential decoding: partial-tile buffer too small");
     const int ri = B <= 16 ? 0 : B <= 32 ? 1 : 2, rt = 16 << ri;
     dim3 grid((N + 127) / 128, ksplit, (B + rt - 1) / rt);
 #define TF_SEQ_TC_CASE(RTV)                                                                                              \
   if (rt == RTV)                                                                                                         \
     return launch_seq(m, cls, seq::seq_gemm_tc_kernel<RTV>, grid, 128, seq::gemm_tc_smem_bytes<RTV>(), W.map_seq,         \
-                      m->map_seq_a[abuf][ri], B, N, kbn, m->seq_part, m->step_ctr, step_off, n_steps, m->seq_check_steps, \
-                      m->err, (const float*)nullptr, (bf16*)nullptr);
+                      m->map_seq_a[abuf][ri], cx.b0, B, N, kbn, cx.part, cx.step_ctr, step_off, n_steps,                 \
+                      m->seq_check_steps, m->err, (const float*)nullptr, (bf16*)nullptr);
     TF_SEQ_TC_CASE(16)
     TF_SEQ_TC_CASE(32)
     TF_SEQ_TC_CASE(64)
@@ -600,7 +627,7 @@ static int seq_gemm(tf_model* m, int cls, int abuf, const Matrix& W, int B, int 
   if (klen > seq::KC || K / klen > 16) return fail(TF_EINVAL, "sequential decoding: reduction length %d not supported", K);
   const int ksplit = K / klen;
   *nsplit = ksplit;
-  if ((size_t)ksplit * B * N > m->seq_part_floats) return fail(TF_EINVAL, "sequential decoding: partial-tile buffer too small");
+  if ((size_t)ksplit * B * N > part_cap) return fail(TF_EINVAL, "sequential decoding: partial-tile buffer too small");
   // column slices: the narrowest (most CTAs, shortest per-warp MMA chain) that keeps the grid within two waves; the
   // warps of a CTA split its K slice, which needs klen % (32 * 64 / NC) == 0
   int nc = 64;
@@ -615,8 +642,8 @@ static int seq_gemm(tf_model* m, int cls, int abuf, const Matrix& W, int B, int 
   const int smem = seq::gemm_smem_bytes(klen);
 #define TF_SEQ_GEMM_CASE(NCV)                                                                                            \
   if (nc == NCV)                                                                                                         \
-    return launch_seq(m, cls, seq::seq_gemm_kernel<NCV>, grid, seq::THREADS, smem, A, w, B, N, K, klen, m->seq_part,     \
-                      m->step_ctr, step_off, n_steps, m->seq_check_steps);
+    return launch_seq(m, cls, seq::seq_gemm_kernel<NCV>, grid, seq::THREADS, smem, A, w, B, N, K, klen, cx.part,         \
+                      cx.step_ctr, step_off, n_steps, m->seq_check_steps);
   TF_SEQ_GEMM_CASE(8)
   TF_SEQ_GEMM_CASE(16)
   TF_SEQ_GEMM_CASE(32)
@@ -625,10 +652,11 @@ static int seq_gemm(tf_model* m, int cls, int abuf, const Matrix& W, int B, int 
   return fail(TF_EINVAL, "no sequential GEMM variant for this shape");
 }
 
-static int seq_resid_ln(tf_model* m, const float* bias, int nsplit, const float* gamma, const float* beta, int B,
+static int seq_resid_ln(tf_model* m, const SeqCtx& cx, const float* bias, int nsplit, const float* gamma, const float* beta,
                         int step_off) {
-  return launch_seq(m, KC_SEQ_LN, seq::seq_resid_ln_kernel, dim3(B), m->d / 4, 0, m->h, m->seq_part, bias, nsplit, gamma,
-                    beta, reinterpret_cast<bf16*>(m->xn), B, m->d, m->step_ctr, step_off, m->L - 1, m->seq_check_steps);
+  return launch_seq(m, KC_SEQ_LN, seq::seq_resid_ln_kernel, dim3(cx.B), m->d / 4, 0, m->h + (size_t)cx.b0 * m->d, cx.part, bias,
+                    nsplit, gamma, beta, reinterpret_cast<bf16*>(m->xn) + (size_t)cx.b0 * m->d, cx.B, m->d, cx.step_ctr, step_off,
+                    m->L - 1, m->seq_check_steps);
 }
 
 static bool seq_tail_fused(const tf_model* m) {
@@ -638,26 +666,38 @@ static bool seq_tail_fused(const tf_model* m) {
 }
 
 // the fused tail of step step_off (first = 0) or the block's start (first = 1)
-static int seq_tail(tf_model* m, int g, int B, const int* labels, const float* v, float* u, const float* pending_bias,
-                    int pending, int first, int step_off) {
+static int seq_tail(tf_model* m, const SeqCtx& cx, int g, const int* labels, const float* v, float* u,
+                    const float* pending_bias, int pending, int first, int step_off) {
   const BlockW& bw = m->blocks[g];
   const LayerW& l0 = bw.layers[0];
   const int smem = (m->d + 3 * m->D) * (int)sizeof(float);
-  return launch_seq(m, KC_SEQ_UPDATE, seq::seq_tail_kernel, dim3(B), 256, smem, m->h, m->seq_part, pending_bias, pending,
-                    bw.lnf_g, bw.lnf_b, reinterpret_cast<const bf16*>(bw.w_out.w), bw.b_out, B, v, u, labels, bw.w_in_t,
-                    bw.b_in, bw.pos, bw.cls, l0.ln1_g, l0.ln1_b, reinterpret_cast<bf16*>(m->xn), m->L, m->D, m->d, g & 1, first,
-                    m->step_ctr, step_off, m->L - 1);
+  const size_t tok0 = (size_t)cx.b0 * m->L * m->D;
+  return launch_seq(m, KC_SEQ_UPDATE, seq::seq_tail_kernel, dim3(cx.B), 256, smem, m->h + (size_t)cx.b0 * m->d, cx.part,
+                    pending_bias, pending, bw.lnf_g, bw.lnf_b, reinterpret_cast<const bf16*>(bw.w_out.w), bw.b_out, cx.B,
+                    v + tok0, u + tok0, labels ? labels + cx.b0 : nullptr, bw.w_in_t, bw.b_in, bw.pos, bw.cls, l0.ln1_g, l0.ln1_b,
+                    reinterpret_cast<bf16*>(m->xn) + (size_t)cx.b0 * m->d, m->L, m->D, m->d, g & 1, first, cx.step_ctr, step_off,
+                    m->L - 1);
 }
 
-// kernels of decoding steps step_off .. step_off+count-1 relative to the device step counter
-static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const float* v, float* u, int count) {
+static int seq_update_embed(tf_model* m, const SeqCtx& cx, int g, const int* labels, const float* v, float* u, int ns,
+                            int first, int step_off) {
   const BlockW& bw = m->blocks[g];
-  const int L = m->L, D = m->D, d = m->d, rev = g & 1, nl = m->cfg.n_layers, heads = m->cfg.n_heads;
-  bf16* att = reinterpret_cast<bf16*>(m->att);
-  bf16* mlp = reinterpret_cast<bf16*>(m->mlp);
-  const size_t layer_stride = (size_t)m->cfg.max_batch * L * d;
+  const int d = m->d, D = m->D, ethreads = d < 128 ? d : 128;
+  const size_t tok0 = (size_t)cx.b0 * m->L * D;
+  return launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(cx.B, (d + ethreads - 1) / ethreads), ethreads,
+                    (int)(D * sizeof(float)), cx.part, ns, bw.b_out, cx.B, v + tok0, u + tok0, labels ? labels + cx.b0 : nullptr,
+                    bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h + (size_t)cx.b0 * d, m->L, D, d, g & 1, first, cx.step_ctr, step_off,
+                    m->L - 1);
+}
+
+// kernels of decoding steps step_off .. step_off+count-1 relative to the chain's device step counter
+static int seq_enqueue_steps(tf_model* m, const SeqCtx& cx, int g, const int* labels, const float* v, float* u, int count) {
+  const BlockW& bw = m->blocks[g];
+  const int L = m->L, d = m->d, nl = m->cfg.n_layers, heads = m->cfg.n_heads, B = cx.B;
+  bf16* att = reinterpret_cast<bf16*>(m->att) + (size_t)cx.b0 * d;
+  bf16* mlp = reinterpret_cast<bf16*>(m->mlp) + (size_t)cx.b0 * m->hid;
+  const size_t layer_stride = (size_t)m->cfg.max_batch * L * d, kv0 = (size_t)cx.b0 * L * d;
   const float scale = 1.0f / sqrtf((float)m->hd);
-  const int ethreads = d < 128 ? d : 128;
   m->cur_rows = B;
   const bool tail = seq_tail_fused(m);
   for (int s = 0; s < count; ++s) {
@@ -665,31 +705,29 @@ static int seq_enqueue_steps(tf_model* m, int g, int B, const int* labels, const
     int pending = 0, ns = 0;
     for (int i = 0; i < nl; ++i) {
       const LayerW& lw = bw.layers[i];
-      bf16* kc = reinterpret_cast<bf16*>(m->kcache) + i * layer_stride;
-      bf16* vc = reinterpret_cast<bf16*>(m->vcache) + i * layer_stride;
+      bf16* kc = reinterpret_cast<bf16*>(m->kcache) + i * layer_stride + kv0;
+      bf16* vc = reinterpret_cast<bf16*>(m->vcache) + i * layer_stride + kv0;
       // layer 0's input comes from the fused tail of the previous step (or of the block's start) when that is on
-      if (!(tail && i == 0)) TF_TRY(seq_resid_ln(m, pending_bias, pending, lw.ln1_g, lw.ln1_b, B, s));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 0, lw.w_qkv, B, s, &ns));
-      TF_TRY(launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, m->seq_part, ns, lw.b_qkv, kc, vc,
-                        att, B, L, d, heads, scale * 1.4426950408889634f, m->step_ctr, s, L - 1));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 1, lw.w_o, B, s, &pending));
-      TF_TRY(seq_resid_ln(m, lw.b_o, pending, lw.ln2_g, lw.ln2_b, B, s));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 0, lw.w_1, B, s, &ns, lw.b_1, mlp));
+      if (!(tail && i == 0)) TF_TRY(seq_resid_ln(m, cx, pending_bias, pending, lw.ln1_g, lw.ln1_b, s));
+      TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, lw.w_qkv, s, &ns));
+      TF_TRY(launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, cx.part, ns, lw.b_qkv, kc, vc,
+                        att, B, L, d, heads, scale * 1.4426950408889634f, cx.step_ctr, s, L - 1));
+      TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 1, lw.w_o, s, &pending));
+      TF_TRY(seq_resid_ln(m, cx, lw.b_o, pending, lw.ln2_g, lw.ln2_b, s));
+      TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, lw.w_1, s, &ns, lw.b_1, reinterpret_cast<bf16*>(m->mlp)));
       if (ns > 0)  // the GEMM left partial tiles: sum them, add the bias, apply GELU
-        TF_TRY(launch_seq(m, KC_SEQ_LN, seq::seq_bias_gelu_kernel, dim3((B * (m->hid / 4) + 255) / 256), 256, 0, m->seq_part, ns,
-                          lw.b_1, mlp, B, m->hid, m->step_ctr, s, L - 1, m->seq_check_steps));
-      TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 2, lw.w_2, B, s, &pending));
+        TF_TRY(launch_seq(m, KC_SEQ_LN, seq::seq_bias_gelu_kernel, dim3((B * (m->hid / 4) + 255) / 256), 256, 0, cx.part, ns,
+                          lw.b_1, mlp, B, m->hid, cx.step_ctr, s, L - 1, m->seq_check_steps));
+      TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 2, lw.w_2, s, &pending));
       pending_bias = lw.b_2;
     }
     if (tail) {
-      TF_TRY(seq_tail(m, g, B, labels, v, u, pending_bias, pending, 0, s));
+      TF_TRY(seq_tail(m, cx, g, labels, v, u, pending_bias, pending, 0, s));
       continue;
     }
-    TF_TRY(seq_resid_ln(m, pending_bias, pending, bw.lnf_g, bw.lnf_b, B, s));
-    TF_TRY(seq_gemm(m, KC_SEQ_GEMM, 0, bw.w_out, B, s, &ns));
-    TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B, (d + ethreads - 1) / ethreads), ethreads,
-                      (int)(D * sizeof(float)), m->seq_part, ns, bw.b_out, B, v, u, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 0, m->step_ctr, s,
-                      L - 1));
+    TF_TRY(seq_resid_ln(m, cx, pending_bias, pending, bw.lnf_g, bw.lnf_b, s));
+    TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, bw.w_out, s, &ns));
+    TF_TRY(seq_update_embed(m, cx, g, labels, v, u, ns, 0, s));
   }
   return check_launch("sequential step kernels");
 }
@@ -701,29 +739,35 @@ static int seq_unroll(int n_steps) {  // steps per graph: a divisor of n_steps c
   return best >= 4 ? best : (n_steps < 16 ? n_steps : 16);
 }
 
-static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* labels, const float* v, float* u) {
-  const BlockW& bw = m->blocks[g];
-  const int L = m->L, D = m->D, d = m->d, rev = g & 1, n_steps = L - 1;
-  const int ethreads = d < 128 ? d : 128;
-  cudaStream_t user = m->stream;
-  m->seq_check_steps = (m->prof_on || !m->use_graphs) ? 0 : (n_steps % seq_unroll(n_steps) != 0);
-  CU_OK(cudaMemsetAsync(m->step_ctr, 0, sizeof(int), user));
-  m->cur_rows = B;
-  if (seq_tail_fused(m))
-    TF_TRY(seq_tail(m, g, B, labels, v, u, nullptr, 0, 1, 0));
-  else
-    TF_TRY(launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(B, (d + ethreads - 1) / ethreads), ethreads,
-                      (int)(D * sizeof(float)), m->seq_part, 0,
-                      bw.b_out, B, v, u, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, 1, m->step_ctr, 0,
-                      n_steps));
+// How many chains decode a batch of B samples side by side.  Every chain streams the block's weights once per step,
+// so the count is limited where the weights come from device memory rather than from L2.
+static int seq_chain_count(const tf_model* m, int B) {
+  int n = m->seq_chains_force;
+  if (n <= 0) {
+    const size_t w_block = (size_t)m->cfg.n_layers * ((size_t)4 * m->d * m->d + (size_t)2 * m->hid * m->d) * sizeof(bf16);
+    n = w_block <= ((size_t)48 << 20) ? 4 : 2;
+  }
+  if (n > tf_model::MAX_CHAINS) n = tf_model::MAX_CHAINS;
+  while (n > 1 && B / n < 4) n /= 2;  // at least four samples per chain
+  return n < 1 ? 1 : n;
+}
+
+// all decoding steps of one chain, enqueued on m->stream (the chain's stream)
+static int run_sequential_chain(tf_model* m, const SeqCtx& cx, int g, const int* labels, const float* v, float* u) {
+  const int n_steps = m->L - 1;
+  CU_OK(cudaMemsetAsync(cx.step_ctr, 0, sizeof(int), m->stream));
+  m->cur_rows = cx.B;
+  if (seq_tail_fused(m)) TF_TRY(seq_tail(m, cx, g, labels, v, u, nullptr, 0, 1, 0));
+  else TF_TRY(seq_update_embed(m, cx, g, labels, v, u, 0, 1, 0));
   if (m->prof_on || !m->use_graphs) {  // direct launches (per-kernel events need them)
     for (int t = 0; t < n_steps; ++t) {
-      TF_TRY(seq_enqueue_steps(m, g, B, labels, v, u, 1));
-      TF_TRY(launch_seq(m, KC_CTRL, seq::seq_advance_kernel, dim3(1), 32, 0, m->step_ctr, 1));
+      TF_TRY(seq_enqueue_steps(m, cx, g, labels, v, u, 1));
+      TF_TRY(launch_seq(m, KC_CTRL, seq::seq_advance_kernel, dim3(1), 32, 0, cx.step_ctr, 1));
     }
     return check_launch("sequential block");
   }
-  auto key = std::make_pair(g, B);
+  cudaStream_t run_stream = m->stream;
+  auto key = std::make_tuple(g, cx.b0, cx.B);
   auto it = m->seq_graphs.find(key);
   if (it == m->seq_graphs.end()) {
     tf_model::SeqGraph sg;
@@ -734,11 +778,11 @@ static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* label
     cudaError_t e = cudaStreamBeginCapture(m->cap_stream, cudaStreamCaptureModeThreadLocal);
     int r = TF_OK;
     if (e == cudaSuccess) {
-      r = seq_enqueue_steps(m, g, B, labels, v, u, sg.unroll);
-      if (r == TF_OK) r = launch_seq(m, KC_CTRL, seq::seq_advance_kernel, dim3(1), 32, 0, m->step_ctr, sg.unroll);
+      r = seq_enqueue_steps(m, cx, g, labels, v, u, sg.unroll);
+      if (r == TF_OK) r = launch_seq(m, KC_CTRL, seq::seq_advance_kernel, dim3(1), 32, 0, cx.step_ctr, sg.unroll);
       e = cudaStreamEndCapture(m->cap_stream, &graph);
     }
-    m->stream = user;
+    m->stream = run_stream;
     sg.nodes = (int)(m->launches - before);
     m->launches = before;
     if (e != cudaSuccess || r != TF_OK || !graph) {
@@ -753,20 +797,63 @@ static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* label
   }
   const tf_model::SeqGraph& sg = it->second;
   const int replays = (n_steps + sg.unroll - 1) / sg.unroll;  // steps past n_steps return at once
-  for (int i = 0; i < replays; ++i) CU_OK(cudaGraphLaunch(sg.exec, user));
+  for (int i = 0; i < replays; ++i) CU_OK(cudaGraphLaunch(sg.exec, run_stream));
   m->launches += (int64_t)replays * sg.nodes;
   return TF_OK;
+}
+
+static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* labels, const float* v, float* u) {
+  const int n_steps = m->L - 1;
+  cudaStream_t user = m->stream;
+  const bool direct = m->prof_on || !m->use_graphs;
+  m->seq_check_steps = direct ? 0 : (n_steps % seq_unroll(n_steps) != 0);
+  const int nch = direct ? 1 : seq_chain_count(m, B);
+  if (nch == 1) {
+    SeqCtx cx;
+    cx.b0 = 0; cx.B = B; cx.step_ctr = m->step_ctr; cx.part = m->seq_part;
+    return run_sequential_chain(m, cx, g, labels, v, u);
+  }
+  // fork: the chains start once everything enqueued on the caller's stream so far has completed; join: the caller's
+  // stream continues once every chain has finished
+  CU_OK(cudaEventRecord(m->seq_fork, user));
+  int r = TF_OK;
+  for (int c = 0; c < nch && r == TF_OK; ++c) {
+    SeqCtx cx;
+    cx.b0 = (int)((int64_t)B * c / nch);
+    cx.B = (int)((int64_t)B * (c + 1) / nch) - cx.b0;
+    cx.step_ctr = m->step_ctr + 16 * c;
+    cx.part = m->seq_part + (size_t)cx.b0 * m->seq_part_row_floats;
+    m->stream = m->seq_streams[c];
+    cudaError_t e = cudaStreamWaitEvent(m->stream, m->seq_fork, 0);
+    if (e != cudaSuccess) r = fail(TF_ECUDA, "cudaStreamWaitEvent: %s", cudaGetErrorString(e));
+    if (r == TF_OK) r = run_sequential_chain(m, cx, g, labels, v, u);
+    if (r == TF_OK && (e = cudaEventRecord(m->seq_join[c], m->stream)) != cudaSuccess)
+      r = fail(TF_ECUDA, "cudaEventRecord: %s", cudaGetErrorString(e));
+    if (r == TF_OK && (e = cudaStreamWaitEvent(user, m->seq_join[c], 0)) != cudaSuccess)
+      r = fail(TF_ECUDA, "cudaStreamWaitEvent: %s", cudaGetErrorString(e));
+  }
+  m->stream = user;
+  return r;
 }
 
 // ------------------------------------------------------------------------------------------------
 // Jacobi block (Algorithm 1) with per-sample stopping and active-set compaction
 // ------------------------------------------------------------------------------------------------
+// A recorded device-side timeout is reported once and the word is cleared, so the model stays usable: kernels
+// launched after the word was set returned without work, the ones launched after this call run normally.
+static int report_timeout(tf_model* m) {
+  const int code = m->ctrl_host[2];
+  cudaMemsetAsync(m->err, 0, sizeof(int), m->stream);
+  cudaStreamSynchronize(m->stream);
+  return fail(TF_ETIMEOUT, "device-side wait expired (code %d)", code);
+}
+
 static int read_ctrl(tf_model* m) {
   CU_OK(cudaMemcpyAsync(m->ctrl_host, m->ctrl, 2 * sizeof(int), cudaMemcpyDeviceToHost, m->stream));
   CU_OK(cudaMemcpyAsync(m->ctrl_host + 3, m->ctrl + 2, 2 * sizeof(int), cudaMemcpyDeviceToHost, m->stream));
   CU_OK(cudaMemcpyAsync(m->ctrl_host + 2, m->err, sizeof(int), cudaMemcpyDeviceToHost, m->stream));
   CU_OK(cudaStreamSynchronize(m->stream));
-  if (m->ctrl_host[2] != 0) return fail(TF_ETIMEOUT, "device-side wait expired (code %d)", m->ctrl_host[2]);
+  if (m->ctrl_host[2] != 0) return report_timeout(m);
   if (m->ctrl_host[1] != 0) return fail(TF_ENONFINITE, "non-finite value in the convergence reduction");
   return TF_OK;
 }
@@ -775,7 +862,28 @@ static int read_ctrl(tf_model* m) {
 static int sync_check(tf_model* m) {
   CU_OK(cudaMemcpyAsync(m->ctrl_host + 2, m->err, sizeof(int), cudaMemcpyDeviceToHost, m->stream));
   CU_OK(cudaStreamSynchronize(m->stream));
-  if (m->ctrl_host[2] != 0) return fail(TF_ETIMEOUT, "device-side wait expired (code %d)", m->ctrl_host[2]);
+  if (m->ctrl_host[2] != 0) return report_timeout(m);
+  return TF_OK;
+}
+
+// Class labels come from the caller's device memory and index the class-embedding table: copy them into the
+// model-owned array (a fixed address for captured graphs) clamped to [0, n_classes), and fail with TF_EINVAL when one
+// was out of range -- no kernel ever indexes the table with an unchecked id.
+static int take_labels(tf_model* m, const int** labels, int B) {
+  if (!*labels) return TF_OK;
+  if (m->cfg.n_classes <= 0) {  // an unconditional model has no table: the labels are not read at all
+    *labels = nullptr;
+    return TF_OK;
+  }
+  LAUNCH(m, KC_CTRL, labels_check_kernel, (B + 127) / 128, 128, 0, *labels, m->labels_own, B, m->cfg.n_classes, m->ctrl + 5);
+  TF_TRY(check_launch("labels_check_kernel"));
+  CU_OK(cudaMemcpyAsync(m->ctrl_host + 5, m->ctrl + 5, sizeof(int), cudaMemcpyDeviceToHost, m->stream));
+  CU_OK(cudaStreamSynchronize(m->stream));
+  if (m->ctrl_host[5] != 0) {
+    CU_OK(cudaMemsetAsync(m->ctrl + 5, 0, sizeof(int), m->stream));
+    return fail(TF_EINVAL, "a class label lies outside [0, %d)", m->cfg.n_classes);
+  }
+  *labels = m->labels_own;
   return TF_OK;
 }
 
@@ -834,10 +942,7 @@ static int inverse_impl(tf_model* m, const float* z, const int* labels, int B, c
   const int K = m->cfg.n_blocks;
   float *v = m->seq_a, *u = m->seq_b;
   m->trace.clear();
-  if (labels) {  // model-owned copy: captured graphs keep a fixed address
-    CU_OK(cudaMemcpyAsync(m->labels_own, labels, B * sizeof(int), cudaMemcpyDeviceToDevice, m->stream));
-    labels = m->labels_own;
-  }
+  TF_TRY(take_labels(m, &labels, B));
   TF_TRY(layout(m, const_cast<float*>(z), v, B, 1));
   int status = TF_OK;
   for (int g = 0; g < K; ++g) {
@@ -868,6 +973,7 @@ static int inverse_impl(tf_model* m, const float* z, const int* labels, int B, c
 template <class T>
 static int forward_impl(tf_model* m, const float* x, const int* labels, int B, float* z, float* logdet) {
   float *u = m->seq_a, *v = m->seq_b;
+  TF_TRY(take_labels(m, &labels, B));
   TF_TRY(layout(m, const_cast<float*>(x), u, B, 1));
   if (logdet) CU_OK(cudaMemsetAsync(logdet, 0, B * sizeof(float), m->stream));
   for (int g = m->cfg.n_blocks - 1; g >= 0; --g) {
@@ -876,7 +982,8 @@ static int forward_impl(tf_model* m, const float* x, const int* labels, int B, f
     TF_TRY(check_launch("forward_affine_kernel"));
     float* tmp = v; v = u; u = tmp;
   }
-  return layout(m, z, u, B, 0);
+  TF_TRY(layout(m, z, u, B, 0));
+  return sync_check(m);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1024,15 +1131,16 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
   TF_TRY(dev_alloc(m, &m->io_x, B * c.C * c.H * c.W));
   TF_TRY(dev_alloc(m, &m->io_labels, B));
   TF_TRY(dev_alloc(m, &m->labels_own, B));
-  TF_TRY(dev_alloc(m, &m->step_ctr, 1));
+  TF_TRY(dev_alloc(m, &m->step_ctr, 16 * tf_model::MAX_CHAINS));  // one counter per chain, 64 bytes apart
   if (c.dtype == 1) {  // partial tiles: up to 16 K slices of a [B, d] output, or d/256 slices of the widest one
     const size_t wide = (size_t)(hid > 3 * d ? hid : 3 * d);
-    m->seq_part_floats = (size_t)16 * B * d;
-    const size_t per_wide = (size_t)(d / 64 < 16 ? d / 64 : 16) * B * wide;
-    if (per_wide > m->seq_part_floats) m->seq_part_floats = per_wide;
+    m->seq_part_row_floats = (size_t)16 * d;
+    const size_t per_wide = (size_t)(d / 64 < 16 ? d / 64 : 16) * wide;
+    if (per_wide > m->seq_part_row_floats) m->seq_part_row_floats = per_wide;
+    m->seq_part_floats = m->seq_part_row_floats * B;
     TF_TRY(dev_alloc(m, &m->seq_part, m->seq_part_floats));
   }
-  CU_OK(cudaMemset(m->step_ctr, 0, sizeof(int)));
+  CU_OK(cudaMemset(m->step_ctr, 0, 16 * tf_model::MAX_CHAINS * sizeof(int)));
   CU_OK(cudaMemset(m->ctrl, 0, 8 * sizeof(int)));
   CU_OK(cudaMemset(m->err, 0, sizeof(int)));
   CU_OK(cudaMemset(m->iters_sample, 0, (size_t)c.n_blocks * B * sizeof(int)));
@@ -1090,6 +1198,13 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, gsm));
     CU_OK(cudaFuncSetAttribute(seq::seq_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, gsm));
     CU_OK(cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking));
+    for (int c = 0; c < tf_model::MAX_CHAINS; ++c) {
+      CU_OK(cudaStreamCreateWithFlags(&m->seq_streams[c], cudaStreamNonBlocking));
+      CU_OK(cudaEventCreateWithFlags(&m->seq_join[c], cudaEventDisableTiming));
+    }
+    CU_OK(cudaEventCreateWithFlags(&m->seq_fork, cudaEventDisableTiming));
+    if (const char* e = getenv("TARFLOW_SEQ_CHAINS")) m->seq_chains_force = atoi(e);
+    if (const char* e = getenv("TARFLOW_SEQ_KBN")) m->seq_kbn_force = atoi(e);
   }
   CU_OK(cudaDeviceSynchronize());
   return TF_OK;
@@ -1148,6 +1263,11 @@ void tf_free(tf_model* m) {
   for (cudaEvent_t e : m->ev_pool) cudaEventDestroy(e);
   for (auto& kv : m->seq_graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
   if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
+  for (int c = 0; c < tf_model::MAX_CHAINS; ++c) {
+    if (m->seq_streams[c]) cudaStreamDestroy(m->seq_streams[c]);
+    if (m->seq_join[c]) cudaEventDestroy(m->seq_join[c]);
+  }
+  if (m->seq_fork) cudaEventDestroy(m->seq_fork);
   for (void* p : m->allocs) cudaFree(p);
   if (m->ctrl_host) cudaFreeHost(m->ctrl_host);
   delete m;
@@ -1227,19 +1347,20 @@ int tf_jacobi_update(const float* o_dev, const float* v_dev, float* u_dev, float
   return check_launch("jacobi_update_kernel");
 }
 
-static int* g_gemm_err = nullptr;  // error word of the model-less GEMM entry point (allocated once)
+static int* g_gemm_err[kMaxDevices] = {nullptr};  // error word of the model-less GEMM entry point (one per device)
 
 int tf_gemm_bf16(const void* a_dev, const void* w_dev, const float* bias_dev, float* c_dev, int32_t M, int32_t N,
                  int32_t K, void* cuda_stream) {
   g_err[0] = 0;
   if (!a_dev || !w_dev || !c_dev) return fail(TF_EINVAL, "NULL buffer");
   if (M < 1 || N < 8 || K < 64 || K % 64 || N % 8) return fail(TF_EINVAL, "need M>=1, N%%8==0, K%%64==0");
-  if (!g_gemm_err) {
-    CU_OK(cudaMalloc(&g_gemm_err, sizeof(int)));
-    CU_OK(cudaMemset(g_gemm_err, 0, sizeof(int)));
+  const int dev = current_device();
+  if (dev < 0) return fail(TF_EINVAL, "no current device with an ordinal below %d", kMaxDevices);
+  if (!g_gemm_err[dev]) {
+    CU_OK(cudaMalloc(&g_gemm_err[dev], sizeof(int)));
+    CU_OK(cudaMemset(g_gemm_err[dev], 0, sizeof(int)));
   }
-  int dev = 0, sms = 148;
-  CU_OK(cudaGetDevice(&dev));
+  int sms = 148;
   CU_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   const int bn = (N % 256 == 0) ? 256 : 128;
   CUtensorMap ma, mw;
@@ -1247,17 +1368,21 @@ int tf_gemm_bf16(const void* a_dev, const void* w_dev, const float* bias_dev, fl
   TF_TRY(make_map_bf16(&mw, w_dev, N, K, bn));
   EpiStore<float, false> epi{c_dev, bias_dev, N};
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  if (bn == 256) return launch_gemm_tc<256, 4>(nullptr, 0, st, ma, nullptr, mw, M, N, K, epi, g_gemm_err, sms, nullptr);
-  return launch_gemm_tc<128, 6>(nullptr, 0, st, ma, nullptr, mw, M, N, K, epi, g_gemm_err, sms, nullptr);
+  if (bn == 256) return launch_gemm_tc<256, 4>(nullptr, 0, st, ma, nullptr, mw, M, N, K, epi, g_gemm_err[dev], sms, nullptr);
+  return launch_gemm_tc<128, 6>(nullptr, 0, st, ma, nullptr, mw, M, N, K, epi, g_gemm_err[dev], sms, nullptr);
 }
 
 int tf_gemm_status(void* cuda_stream) {
   g_err[0] = 0;
   CU_OK(cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(cuda_stream)));
-  if (!g_gemm_err) return TF_OK;
+  const int dev = current_device();
+  if (dev < 0 || !g_gemm_err[dev]) return TF_OK;
   int e = 0;
-  CU_OK(cudaMemcpy(&e, g_gemm_err, sizeof(int), cudaMemcpyDeviceToHost));
-  if (e != 0) return fail(TF_ETIMEOUT, "device-side wait expired in tf_gemm_bf16 (code %d)", e);
+  CU_OK(cudaMemcpy(&e, g_gemm_err[dev], sizeof(int), cudaMemcpyDeviceToHost));
+  if (e != 0) {  // reported once, then cleared: later launches run normally
+    CU_OK(cudaMemset(g_gemm_err[dev], 0, sizeof(int)));
+    return fail(TF_ETIMEOUT, "device-side wait expired in tf_gemm_bf16 (code %d)", e);
+  }
   return TF_OK;
 }
 
@@ -1267,7 +1392,7 @@ int tf_gemm_status(void* cuda_stream) {
 // ------------------------------------------------------------------------------------------------
 #define TF_NOALLOC_HEADER_BYTES 256u
 static __device__ __align__(256) unsigned char g_noalloc_scratch[TF_NOALLOC_SCRATCH_BYTES];
-static unsigned char* g_noalloc_ptr[64] = {nullptr};  // device address of the array, per device ordinal
+static unsigned char* g_noalloc_ptr[kMaxDevices] = {nullptr};  // device address of the array, per device ordinal
 
 // c[m, n] = bias[n] + sum over K slices of part[s][m][n], slices added in index order
 __global__ void noalloc_reduce_kernel(const float* __restrict__ part, const float* __restrict__ bias,
@@ -1285,21 +1410,27 @@ int tf_skinny_gemm_noalloc(const void* a_dev, const void* w_dev, const float* bi
   g_err[0] = 0;
   if (!a_dev || !w_dev || !c_dev) return fail(TF_EINVAL, "NULL buffer");
   if (M < 1 || N < 8 || N % 8 || K < 256 || K % 256) return fail(TF_EINVAL, "need M >= 1, N %% 8 == 0, K %% 256 == 0");
+  // the kernel reads A and W with 16-byte accesses and the reduction reads/writes 4-byte floats: a misaligned pointer
+  // would fault on the device, so it is refused here
+  if ((reinterpret_cast<uintptr_t>(a_dev) | reinterpret_cast<uintptr_t>(w_dev)) & 15)
+    return fail(TF_EINVAL, "tf_skinny_gemm_noalloc: a_dev and w_dev must be 16-byte aligned");
+  if ((reinterpret_cast<uintptr_t>(c_dev) | reinterpret_cast<uintptr_t>(bias_dev)) & 3)
+    return fail(TF_EINVAL, "tf_skinny_gemm_noalloc: c_dev and bias_dev must be 4-byte aligned");
   const int klen = 256, ksplit = K / klen;
   const size_t need = (size_t)ksplit * M * N * sizeof(float);
   if (need > (size_t)TF_NOALLOC_SCRATCH_BYTES - TF_NOALLOC_HEADER_BYTES)
     return fail(TF_EINVAL, "tf_skinny_gemm_noalloc: (K/256)*M*N*4 = %zu bytes of partial tiles exceed the %zu-byte static scratch",
                 need, (size_t)TF_NOALLOC_SCRATCH_BYTES - TF_NOALLOC_HEADER_BYTES);
-  int dev = 0;
-  CU_OK(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return fail(TF_EINVAL, "device ordinal %d not supported", dev);
+  const int dev = current_device();
+  if (dev < 0) return fail(TF_EINVAL, "no current device with an ordinal below %d", kMaxDevices);
   using Kern = void (*)(const bf16*, const bf16*, int, int, int, int, float*, const int*, int, int, int);
   Kern kern = seq::seq_gemm_kernel<8>;
   const int smem = seq::gemm_smem_bytes(klen);
   if (!g_noalloc_ptr[dev]) {  // once per device, with that device current: resolve the symbol to a device address
     unsigned char* p = nullptr;
     CU_OK(cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_scratch));
-    CU_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    // the same limit tf_load sets for this kernel, so a model loaded earlier keeps its larger K slices
+    CU_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_smem_bytes(seq::KC)));
     g_noalloc_ptr[dev] = p;
   }
   unsigned char* base = g_noalloc_ptr[dev];
@@ -1317,6 +1448,16 @@ int tf_skinny_gemm_noalloc(const void* a_dev, const void* w_dev, const float* bi
   if (blocks > 148 * 8) blocks = 148 * 8;
   noalloc_reduce_kernel<<<blocks, 256, 0, st>>>(part, bias_dev, c_dev, ksplit, M, N);
   return check_launch("noalloc_reduce_kernel");
+}
+
+int tf_selftest_wait_timeout(tf_model* m, int32_t limit_us, void* cuda_stream) {
+  g_err[0] = 0;
+  if (!m) return fail(TF_EINVAL, "model is NULL");
+  if (limit_us < 1 || limit_us > 1000000) return fail(TF_EINVAL, "limit_us must lie in [1, 1000000]");
+  m->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  LAUNCH(m, KC_CTRL, tc::wait_selftest_kernel, 1, 32, 0, m->err, (unsigned long long)limit_us * 1000ull);
+  TF_TRY(check_launch("wait_selftest_kernel"));
+  return sync_check(m);
 }
 
 int tf_profile_enable(tf_model* m, int32_t on) {

@@ -15,6 +15,12 @@ pytestmark = pytest.mark.gpu
 
 FP32_TOL = 1e-4
 BF16_REL_L2 = 2e-2
+BF16_MAX_ABS = 5e-2   # element-wise companion of the norm: no entry may be off by more than this
+
+
+def bf16_close(x, xo):
+    """Relative L2 within the contract's tolerance and no single entry far off."""
+    return bool(np.isfinite(x).all() and rel_l2(x, xo) <= BF16_REL_L2 and np.abs(x - xo).max() <= BF16_MAX_ABS)
 
 
 # ---------------------------------------------------------------- single kernels
@@ -202,7 +208,7 @@ def test_bf16_small_model_selective_parity():
     cfg = synth.config("cfg2")
     m, x, xo, its, ito, rc = _bf16_case(cfg, 4, 2024, [0, 1, 1, 1], cfg["tau"])
     assert rc == 0
-    assert rel_l2(x, xo) <= BF16_REL_L2
+    assert bf16_close(x, xo)
     assert np.abs(its - ito).max() <= 1
 
 
@@ -221,7 +227,7 @@ def test_bf16_cfg2_full_batch_sampled_against_oracle():
         assert (its[1:] >= 2).all() and (its[1:] <= m.L).all()  # Jacobi: at least two sweeps, at most L (Prop. 3.2)
         pick = [0, 37, B - 1]
         xo, ito = O.model_inverse(m.blocks, z[pick], None, cfg, policy, cfg["tau"], m.L + 1)
-        assert rel_l2(x[pick], xo) <= BF16_REL_L2
+        assert bf16_close(x[pick], xo)
         assert np.abs(its[:, pick] - ito).max() <= 1
         x2, _, its2, rc2 = m.inverse(z, None, policy, cfg["tau"], m.L + 1)  # run-twice determinism
         assert rc2 == 0 and np.array_equal(x, x2) and np.array_equal(its, its2)
@@ -241,7 +247,7 @@ def test_bf16_cfg3_full_batch_sampled_against_oracle():
         assert (its[0] == m.L - 1).all() and (its[1:] >= 2).all() and (its[1:] <= m.L).all()
         pick = [41]
         xo, ito = O.model_inverse(m.blocks, z[pick], lab[pick], cfg, policy, cfg["tau"], m.L + 1)
-        assert rel_l2(x[pick], xo) <= BF16_REL_L2
+        assert bf16_close(x[pick], xo)
         assert np.abs(its[:, pick] - ito).max() <= 1
 
 
@@ -251,14 +257,16 @@ def test_bf16_all_jacobi_and_all_sequential_agree_with_oracle():
         z = synth.make_latents(cfg, 99, B=3)
         xo = O.model_inverse_sequential(m.blocks, z, None, cfg)
         xs = m.inverse_sequential(z, None)
-        assert rel_l2(xs, xo) <= BF16_REL_L2
+        assert bf16_close(xs, xo)
         xj, ib, its, rc = m.inverse(z, None, [1, 1], 1e-3, m.L + 1)
         xjo, ito = O.model_inverse(m.blocks, z, None, cfg, [1, 1], 1e-3, m.L + 1)
-        assert rc == 0 and rel_l2(xj, xjo) <= BF16_REL_L2 and np.abs(its - ito).max() <= 1
+        assert rc == 0 and bf16_close(xj, xjo) and np.abs(its - ito).max() <= 1
         zg, ld = m.forward(xo, None)
         zo, ldo = O.model_forward(m.blocks, xo, None, cfg)
-        assert rel_l2(zg, zo) <= BF16_REL_L2
-        assert np.abs(ld - ldo).max() <= 2e-2 * np.abs(ldo).max() + 0.5
+        assert bf16_close(zg, zo)
+        # logdet = -sum of L*D alphas, each carrying activation-rounding error of a few 1e-3 with random sign:
+        # a bound relative to the root-sum-square scale of the sum, without absolute slack
+        assert np.abs(ld - ldo).max() <= 2e-2 * max(np.abs(ldo).max(), np.sqrt(m.L * synth.token_dim(cfg)) * 0.1)
 
 
 def test_bf16_ragged_sequence_length_and_classes():
@@ -266,7 +274,7 @@ def test_bf16_ragged_sequence_length_and_classes():
     cfg = synth.config("cfg3", H=36, W=36, n_blocks=2, n_layers=2, width=256, n_heads=4, n_classes=10)
     lab = synth.make_labels(cfg, B=3)
     m, x, xo, its, ito, rc = _bf16_case(cfg, 3, 5, [0, 1], 1e-3, labels=lab)
-    assert rc == 0 and rel_l2(x, xo) <= BF16_REL_L2 and np.abs(its - ito).max() <= 1
+    assert rc == 0 and bf16_close(x, xo) and np.abs(its - ito).max() <= 1
 
 
 def test_bf16_optional_kernel_paths_agree(monkeypatch):
@@ -284,7 +292,7 @@ def test_bf16_optional_kernel_paths_agree(monkeypatch):
             assert rc == 0 and np.isfinite(outs[name]).all()
     xo, _ = O.model_inverse(synth.make_weights(cfg), z, None, cfg, [1], -1.0, 3)
     for name, x in outs.items():
-        assert rel_l2(x, xo) <= BF16_REL_L2, name
+        assert bf16_close(x, xo), name
     assert rel_l2(outs["attn_mma"], outs["default"]) <= 5e-3
     assert rel_l2(outs["single_cta"], outs["default"]) <= 1e-4
 
@@ -305,7 +313,7 @@ def test_bf16_two_term_attention_paths_agree(monkeypatch):
             outs[name] = (x, its)
     xo, ito = O.model_inverse(synth.make_weights(cfg), z, None, cfg, [1, 1], 1e-3, synth.seq_len(cfg) + 1)
     for name, (x, its) in outs.items():
-        assert rel_l2(x, xo) <= BF16_REL_L2, name
+        assert bf16_close(x, xo), name
         assert np.abs(its - ito).max() <= 1, name
     assert rel_l2(outs["tcgen05"][0], outs["mma_sync"][0]) <= 5e-3
 
@@ -327,7 +335,7 @@ def test_bf16_optional_sequential_paths_agree(monkeypatch):
             assert rc == 0 and np.isfinite(outs[name]).all()
     xo, _ = O.model_inverse(synth.make_weights(cfg), z, None, cfg, [0], -1.0, 3)
     for name, x in outs.items():
-        assert rel_l2(x, xo) <= BF16_REL_L2, name
+        assert bf16_close(x, xo), name
     assert rel_l2(outs["gelu_fused"], outs["default"]) <= 5e-3
     assert rel_l2(outs["mma_sync"], outs["default"]) <= 5e-3
     assert rel_l2(outs["tail_kernels"], outs["default"]) <= 5e-3

@@ -237,13 +237,13 @@ def test_per_sample_stopping_is_independent_of_batch_mates():
     L = synth.seq_len(cfg)
     rng = np.random.default_rng(12)
     v = rng.standard_normal((4, L, synth.token_dim(cfg)))
-    v[1] *= 0.01                                  # an easy sample next to hard ones
+    v[1] *= 0.01                                  # samples of different scale side by side
     u, it, _ = O.block_inverse_jacobi(blocks[0], v, None, cfg, 1e-4, L + 1)
     for b in range(4):
         ub, itb, _ = O.block_inverse_jacobi(blocks[0], v[b:b + 1], None, cfg, 1e-4, L + 1)
         assert itb[0] == it[b]
         assert np.array_equal(ub[0], u[b])
-    assert len(set(it.tolist())) > 1 or True
+    assert len(set(it.tolist())) > 1              # the samples really stop at different sweeps
 
 
 def test_zero_head_makes_every_block_the_identity_and_jacobi_stops_at_sweep_two():
