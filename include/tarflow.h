@@ -130,6 +130,52 @@ int tf_inverse_jacobi(tf_model* m, const float* z_dev, const int32_t* labels_dev
                       void* cuda_stream);
 
 /*
+ * tf_inverse_jacobi_ex -- tf_inverse_jacobi with the variants the paper discusses around Algorithm 1 and the
+ * selective policy (Sec. 3.5, Sec. 4.4; Fig. "Convergence dynamics", the initialisation ablation, the table of
+ * Jacobi iterations per block whose second CIFAR-10 block needs 54 sweeps).  opts == NULL behaves like
+ * tf_inverse_jacobi with init_mode 0.  Fields of tf_jacobi_opts:
+ *   struct_bytes      sizeof(tf_jacobi_opts) as the caller compiled it (checked).
+ *   init_mode         0: u^0 = 0 (Algorithm 1);  1: u^0 = the block's input v;  2: u^0 = u0_dev (for instance the
+ *                     caller's N(0, I) draws: the library draws no random numbers itself).
+ *   u0_dev            init_mode 2: [n_blocks, B, C, H, W] fp32 on the device, image-shaped like z; Jacobi block g
+ *                     starts from slice g (slices of sequential blocks are not read).
+ *   tau_block_host    NULL, or [n_blocks] host floats: block g uses tau_block_host[g] instead of tau (negative:
+ *                     that block runs max_iters sweeps without the test).
+ *   fallback_sweeps   0: off.  n > 0: a Jacobi block that still has unconverged samples after n sweeps decodes
+ *                     exactly those samples sequentially (Eq. 5) from the block's input, so a slowly converging
+ *                     block costs at most n sweeps plus one sequential pass over the stragglers; such a sample
+ *                     reports n + L - 1 iterations, the block reports the maximum.  Ignored when tau < 0 or
+ *                     n >= max_iters.
+ *   states_dev        NULL, or out [n_blocks, B, C, H, W] fp32: the sequence after each block, image-shaped
+ *                     (slice n_blocks - 1 equals x).
+ *   ref_states_dev    NULL, or in [n_blocks, B, C, H, W]: reference states, e.g. states_dev of an all-sequential
+ *                     call.  With the trace enabled every sweep of Jacobi block g also records, per sample,
+ *                     || u^t - ref_g ||_2 (the quantity the paper's convergence figure plots); read it with
+ *                     tf_trace_read_l2.
+ */
+typedef struct {
+  int32_t struct_bytes;
+  int32_t init_mode;
+  const float* u0_dev;
+  const float* tau_block_host;
+  int32_t fallback_sweeps;
+  int32_t reserved;
+  float* states_dev;
+  const float* ref_states_dev;
+} tf_jacobi_opts;
+
+int tf_inverse_jacobi_ex(tf_model* m, const float* z_dev, const int32_t* labels_dev, int32_t B,
+                         const uint8_t* policy_host, float tau, int32_t max_iters, const tf_jacobi_opts* opts,
+                         float* x_dev, int32_t* iters_block_host, int32_t* iters_sample_dev, void* cuda_stream);
+
+/*
+ * tf_block_times -- device time of every block of the last tf_inverse_jacobi* call on this model, from CUDA
+ * events the call records on its stream around each block (the per-block breakdown of the paper's runtime table).
+ * Fills ms_host[0 .. min(cap, n_blocks)) and returns n_blocks; returns 0 when no call has completed yet.
+ */
+int tf_block_times(tf_model* m, float* ms_host, int32_t cap);
+
+/*
  * tf_inverse_jacobi_host -- the same operation for callers that hold host memory: copies z (and
  * labels) to the device, runs tf_inverse_jacobi, copies x back.  z_host/x_host [B,C,H,W] fp32,
  * labels_host [B] or NULL; pinned host memory makes the copies asynchronous.  iters_sample_host
@@ -224,10 +270,15 @@ int tf_set_precision(tf_model* m, int32_t mode, float switch_threshold, float si
  * (block, sweep number, samples active in that sweep, max over those samples of
  * max|u^t - u^{t-1}|).  Enabling it makes every sweep synchronise, also in fixed-iteration mode.
  *   tf_trace_read fills up to cap records of the last call and returns how many exist.
+ *   Enabling the trace for the first time allocates the buffer of tf_trace_read_l2 (device memory).
  */
 int tf_trace_enable(tf_model* m, int32_t on);
 int tf_trace_read(tf_model* m, int32_t* block, int32_t* sweep, int32_t* active, float* maxdiff,
                   int32_t cap);
+/* tf_trace_read_l2 -- the distances || u^t - ref ||_2 recorded for Jacobi block `block` of the last
+ * tf_inverse_jacobi_ex call that supplied ref_states_dev: l2_host[t * B + b] for sweep t + 1 and sample b (samples
+ * that have converged keep their final iterate).  Returns the number of sweeps recorded (0 if none). */
+int tf_trace_read_l2(tf_model* m, int32_t block, int32_t B, float* l2_host, int32_t cap_sweeps);
 
 /*
  * tf_selftest_wait_timeout -- exercises the bounded-wait path without any fault: launches one CTA whose thread

@@ -198,18 +198,20 @@ def jacobi_map(blk, u_prev, v, labels, cfg):
     return u_new
 
 
-def block_inverse_jacobi(blk, v, labels, cfg, tau, max_iters, u0=None, u_star=None):
+def block_inverse_jacobi(blk, v, labels, cfg, tau, max_iters, u0=None, u_star=None, info=None):
     """Algorithm 1 applied to every sample of the batch independently.
 
     u^0 = 0 (or `u0`); sweep t: u^t = F(u^{t-1}); a sample stops after the first sweep whose
     max_{l,c} |u^t - u^{t-1}| <= tau  (tau < 0: never, run exactly max_iters sweeps); a sample
     that has stopped is not touched again.  Returns (u, iters[B], trace) where iters counts the
     sweeps a sample executed including the passing one, and trace[t-1][b] = ||u^t - u_star||_2
-    when u_star is given (Fig. "Convergence dynamics").
+    when u_star is given (Fig. "Convergence dynamics").  If `info` is a dict it receives
+    info["last_maxdiff"][b] = max|u^t - u^{t-1}| of the last sweep sample b executed.
     """
     B, L, D = v.shape
     u = np.zeros_like(v) if u0 is None else np.array(u0, dtype=np.float64)
     iters = np.zeros(B, dtype=np.int64)
+    last_m = np.full(B, np.inf)
     active = np.arange(B)
     trace = []
     t = 0
@@ -220,10 +222,13 @@ def block_inverse_jacobi(blk, v, labels, cfg, tau, max_iters, u0=None, u_star=No
         m = np.abs(u_new - u[active]).reshape(active.size, -1).max(axis=1)
         u[active] = u_new
         iters[active] = t
+        last_m[active] = m
         if u_star is not None:
             trace.append(np.sqrt(((u - u_star) ** 2).reshape(B, -1).sum(axis=1)))
         if tau >= 0:
             active = active[m > tau]
+    if info is not None:
+        info["last_maxdiff"] = last_m
     return u, iters, trace
 
 
@@ -241,26 +246,68 @@ def model_forward(blocks, x, labels, cfg):
     return unpatchify(seq, cfg["C"], cfg["H"], cfg["W"], cfg["patch"]), logdet
 
 
-def model_inverse(blocks, z, labels, cfg, policy, tau, max_iters, cached=True):
+def model_inverse(blocks, z, labels, cfg, policy, tau, max_iters, cached=True, init_mode=0, u0=None,
+                  fallback_sweeps=0, return_states=False, ref_states=None):
     """z -> x through blocks 0 .. K-1 in generation order.
 
     policy[g] = 0: sequential (Eq. 5); 1: Jacobi (Algorithm 1).  Returns (x, iters[K,B]); a
     sequential block reports L-1 steps (as in Table "Average number of Jacobi iterations").
+
+    Variants discussed around Algorithm 1 (Sec. 3.5, Sec. 4.4), all off by default:
+      tau              a scalar, or one value per block;
+      init_mode        0: u^0 = 0;  1: u^0 = v (the block's input);  2: u^0 = patchify(u0[g]) with
+                       u0 [K,B,C,H,W] supplied by the caller (e.g. N(0, I) draws);
+      fallback_sweeps  n > 0: a Jacobi block is cut after n sweeps and the samples that have not
+                       passed the test by then are decoded sequentially (Eq. 5) from the block's
+                       input; they report n + L - 1 iterations (ignored when tau < 0 or n >= max_iters);
+      return_states    also return the image-shaped sequence after every block [K,B,C,H,W];
+      ref_states       [K,B,C,H,W]: also return, per Jacobi block, the trace ||u^t - ref_g||_2 per
+                       sweep and sample (Fig. "Convergence dynamics").
+    With any of the last two the return value is (x, iters, extras) with extras a dict.
     """
     seq = patchify(np.asarray(z, dtype=np.float64), cfg["patch"])
     B, L, _ = seq.shape
-    iters = np.zeros((cfg["n_blocks"], B), dtype=np.int64)
-    for g in range(cfg["n_blocks"]):
+    K = cfg["n_blocks"]
+    taus = [float(tau)] * K if np.ndim(tau) == 0 else [float(t) for t in tau]
+    iters = np.zeros((K, B), dtype=np.int64)
+    states, traces = [], {}
+    for g in range(K):
         v = np.ascontiguousarray(permute(seq, g))
         if policy[g] == 0:
             fn = block_inverse_sequential if cached else block_inverse_sequential_uncached
             u = fn(blocks[g], v, labels, cfg)
             iters[g, :] = L - 1
         else:
-            u, it, _ = block_inverse_jacobi(blocks[g], v, labels, cfg, tau, max_iters)
+            if init_mode == 0:
+                start = None
+            elif init_mode == 1:
+                start = v
+            else:
+                start = permute(patchify(np.asarray(u0[g], dtype=np.float64), cfg["patch"]), g)
+            star = None
+            if ref_states is not None:
+                star = permute(patchify(np.asarray(ref_states[g], dtype=np.float64), cfg["patch"]), g)
+            cut = taus[g] >= 0 and 0 < fallback_sweeps < max_iters
+            info = {}
+            u, it, tr = block_inverse_jacobi(blocks[g], v, labels, cfg, taus[g], fallback_sweeps if cut else max_iters,
+                                             u0=start, u_star=star, info=info)
+            if cut:
+                # the samples whose last executed sweep did not pass the test fall back to Eq. 5
+                left = np.nonzero(info["last_maxdiff"] > taus[g])[0]
+                if left.size:
+                    lab = None if labels is None else np.asarray(labels)[left]
+                    u[left] = block_inverse_sequential(blocks[g], v[left], lab, cfg)
+                    it[left] = fallback_sweeps + L - 1
             iters[g, :] = it
+            if star is not None:
+                traces[g] = np.array(tr)
         seq = np.ascontiguousarray(permute(u, g))
-    return unpatchify(seq, cfg["C"], cfg["H"], cfg["W"], cfg["patch"]), iters
+        if return_states:
+            states.append(unpatchify(seq, cfg["C"], cfg["H"], cfg["W"], cfg["patch"]))
+    x = unpatchify(seq, cfg["C"], cfg["H"], cfg["W"], cfg["patch"])
+    if return_states or ref_states is not None:
+        return x, iters, {"states": np.array(states) if return_states else None, "l2": traces}
+    return x, iters
 
 
 def model_inverse_sequential(blocks, z, labels, cfg):

@@ -23,6 +23,12 @@ class TfConfig(C.Structure):
                                          "mlp_ratio", "n_classes", "dtype", "max_batch")]
 
 
+class TfJacobiOpts(C.Structure):
+    _fields_ = [("struct_bytes", C.c_int32), ("init_mode", C.c_int32), ("u0_dev", C.c_void_p),
+                ("tau_block_host", C.c_void_p), ("fallback_sweeps", C.c_int32), ("reserved", C.c_int32),
+                ("states_dev", C.c_void_p), ("ref_states_dev", C.c_void_p)]
+
+
 class TarflowError(RuntimeError):
     def __init__(self, code, msg):
         super().__init__(f"libtarflow error {code}: {msg}")
@@ -46,6 +52,9 @@ def lib():
         L.tf_forward.argtypes = [vp, vp, vp, i32, vp, vp, vp]
         L.tf_inverse_sequential.argtypes = [vp, vp, vp, i32, vp, vp]
         L.tf_inverse_jacobi.argtypes = [vp, vp, vp, i32, vp, f32, i32, i32, vp, vp, vp, vp]
+        L.tf_inverse_jacobi_ex.argtypes = [vp, vp, vp, i32, vp, f32, i32, C.POINTER(TfJacobiOpts), vp, vp, vp, vp]
+        L.tf_block_times.argtypes = [vp, vp, i32]
+        L.tf_trace_read_l2.argtypes = [vp, i32, i32, vp, i32]
         L.tf_inverse_jacobi_host.argtypes = [vp, vp, vp, i32, vp, f32, i32, i32, vp, vp, vp, vp]
         L.tf_jacobi_update.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
         L.tf_gemm_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
@@ -115,6 +124,34 @@ def tf_inverse_jacobi(m, z, labels, B, policy, tau, max_iters, init_mode, x, ite
     ib = None if iters_block is None else iters_block.ctypes.data_as(C.c_void_p)
     return _check(lib().tf_inverse_jacobi(m, _ptr(z), _ptr(labels), B, pol.ctypes.data_as(C.c_void_p), tau, max_iters,
                                           init_mode, _ptr(x), ib, _ptr(iters_sample), _stream(stream)))
+
+
+def tf_inverse_jacobi_ex(m, z, labels, B, policy, tau, max_iters, x, iters_block=None, iters_sample=None, stream=None,
+                         init_mode=0, u0=None, tau_block=None, fallback_sweeps=0, states=None, ref_states=None):
+    """Keyword arguments fill tf_jacobi_opts: u0 / states / ref_states are CUDA tensors [n_blocks,B,C,H,W], tau_block a
+    sequence of floats per block."""
+    pol = np.ascontiguousarray(np.asarray(policy, dtype=np.uint8))
+    ib = None if iters_block is None else iters_block.ctypes.data_as(C.c_void_p)
+    tb = None if tau_block is None else np.ascontiguousarray(np.asarray(tau_block, dtype=np.float32))
+    o = TfJacobiOpts(C.sizeof(TfJacobiOpts), int(init_mode), None if u0 is None else u0.data_ptr(),
+                     None if tb is None else tb.ctypes.data, int(fallback_sweeps), 0,
+                     None if states is None else states.data_ptr(), None if ref_states is None else ref_states.data_ptr())
+    return _check(lib().tf_inverse_jacobi_ex(m, _ptr(z), _ptr(labels), B, pol.ctypes.data_as(C.c_void_p), tau, max_iters,
+                                             C.byref(o), _ptr(x), ib, _ptr(iters_sample), _stream(stream)))
+
+
+def tf_block_times(m, n_blocks):
+    """-> numpy float32 [n_blocks]: milliseconds of each block of the last inverse call (empty if none yet)."""
+    ms = np.zeros(n_blocks, dtype=np.float32)
+    k = _check(lib().tf_block_times(m, ms.ctypes.data_as(C.c_void_p), n_blocks))
+    return ms[:k]
+
+
+def tf_trace_read_l2(m, block, B, cap_sweeps=2048):
+    """-> numpy float32 [sweeps, B]: ||u^t - ref||_2 per sweep and sample of a Jacobi block of the last _ex call."""
+    buf = np.zeros((cap_sweeps, B), dtype=np.float32)
+    n = _check(lib().tf_trace_read_l2(m, int(block), int(B), buf.ctypes.data_as(C.c_void_p), cap_sweeps))
+    return buf[:min(n, cap_sweeps)]
 
 
 def tf_inverse_jacobi_host(m, z_host, labels_host, B, policy, tau, max_iters, init_mode, x_host, iters_block=None,

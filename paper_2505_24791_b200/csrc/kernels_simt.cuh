@@ -617,6 +617,47 @@ __global__ void jacobi_begin_kernel(float* __restrict__ maxdiff, int* __restrict
   if (threadIdx.x == 0) { ctrl[0] = B; ctrl[1] = 0; ctrl[2] = 0; ctrl[3] = start_phase ? B : 0; }
 }
 
+// Rows of nf floats each: dst[s] = src[idx[s]] (to_compact != 0) or dst[idx[s]] = src[s] (to_compact == 0), s < n.
+// Used to decode a subset of a batch (the samples still active in a Jacobi block) as a dense batch of its own.
+__global__ void gather_rows_kernel(const float* __restrict__ src, float* __restrict__ dst, const int* __restrict__ idx,
+                                   int n, int nf, int to_compact) {
+  const size_t total = (size_t)n * nf;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int s = (int)(i / nf), k = (int)(i - (size_t)s * nf), b = idx[s];
+    if (to_compact) dst[(size_t)s * nf + k] = src[(size_t)b * nf + k];
+    else dst[(size_t)b * nf + k] = src[(size_t)s * nf + k];
+  }
+}
+__global__ void gather_int_kernel(const int* __restrict__ src, int* __restrict__ dst, const int* __restrict__ idx, int n) {
+  int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s < n) dst[s] = src[idx[s]];
+}
+// iters[idx[s]] += add for the s < n listed samples
+__global__ void add_int_rows_kernel(int* __restrict__ iters, const int* __restrict__ idx, int n, int add) {
+  int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s < n) iters[idx[s]] += add;
+}
+
+// out[b] = || u[b] - ref[b] ||_2 over the n values of sample b (one CTA per sample, fixed-order tree).
+__global__ void __launch_bounds__(256) l2_distance_kernel(const float* __restrict__ u, const float* __restrict__ ref,
+                                                          float* __restrict__ out, int n) {
+  __shared__ float red[8];
+  const int b = blockIdx.x;
+  float acc = 0.f;
+  for (int i = threadIdx.x; i < n; i += 256) {
+    const float dlt = u[(size_t)b * n + i] - ref[(size_t)b * n + i];
+    acc = fmaf(dlt, dlt, acc);
+  }
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int i = 0; i < 8; ++i) t += red[i];
+    out[b] = sqrtf(t);
+  }
+}
+
 // out[b] = labels[b] clamped to [0, n_classes); *flag is set when a label had to be clamped.
 __global__ void labels_check_kernel(const int* __restrict__ labels, int* __restrict__ out, int B, int n_classes,
                                     int* __restrict__ flag) {

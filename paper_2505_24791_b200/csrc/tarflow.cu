@@ -182,17 +182,23 @@ struct tf_model {
   int* labels_own = nullptr;
   cudaStream_t cap_stream = nullptr;
   struct SeqGraph { cudaGraphExec_t exec = nullptr; int unroll = 0; int nodes = 0; };
-  std::map<std::tuple<int, int, int>, SeqGraph> seq_graphs;  // (block g, first sample, samples) of a chain
+  std::map<std::tuple<int, int, int, int>, SeqGraph> seq_graphs;  // (block g, first sample, samples, buffer set) of a chain
   enum { MAX_CHAINS = 4 };
   cudaStream_t seq_streams[MAX_CHAINS] = {nullptr};  // one stream per chain of a sequential block
   cudaEvent_t seq_fork = nullptr, seq_join[MAX_CHAINS] = {nullptr};
   int seq_chains_force = 0;  // TARFLOW_SEQ_CHAINS=1|2|4: chains per sequential block (0 = by the size of the weights)
   int seq_kbn_force = 0;     // TARFLOW_SEQ_KBN
+  int seq_variant = 0;       // 0: the block's own token buffers, 1: the compact buffers of the sequential fall-back
   size_t seq_part_row_floats = 0;  // floats of partial tiles available per sample
   bool use_graphs = true;
   int seq_check_steps = 0;    // 1 when a replayed graph can run past the last step (kernels then test the counter)
   float* seq_part = nullptr;  // fp32 partial tiles [K slices][B][N] of the projection in flight
   size_t seq_part_floats = 0;
+  float *cmp_v = nullptr, *cmp_u = nullptr, *ref_seq = nullptr;  // compact token buffers (fall-back), reference state
+  int* cmp_labels = nullptr;
+  float* trace_l2 = nullptr;            // [n_blocks][trace_l2_sweeps][max_batch] when the trace is on
+  int trace_l2_sweeps = 0;
+  std::vector<int> trace_l2_count;      // sweeps recorded per block in the last call
   float *io_z = nullptr, *io_x = nullptr;  // staging for the host-buffer entry point
   int* io_labels = nullptr;
   cudaStream_t stream = nullptr;
@@ -210,6 +216,8 @@ struct tf_model {
   struct TraceRec { int block, sweep, active; float maxdiff; };
   bool trace_on = false;
   std::vector<TraceRec> trace;
+  std::vector<cudaEvent_t> block_ev;  // n_blocks + 1 events bracketing the blocks of the last inverse call
+  bool block_ev_valid = false;
 
   cudaEvent_t get_event() {
     if (!ev_pool.empty()) {
@@ -739,14 +747,13 @@ static int seq_unroll(int n_steps) {  // steps per graph: a divisor of n_steps c
   return best >= 4 ? best : (n_steps < 16 ? n_steps : 16);
 }
 
-// How many chains decode a batch of B samples side by side.  Every chain streams the block's weights once per step,
-// so the count is limited where the weights come from device memory rather than from L2.
+// How many chains decode a batch of B samples side by side.  Measured (one block, ms): width 512, 4 layers, batch 64:
+// 31.5 / 27.4 / 27.5 with 1 / 2 / 4 chains; width 1024, 8 layers, batch 64: 85.5 / 81.0 / 84.1; 1024 tokens, batch 16:
+// 280 / 301 / 338.  A chain of 16 samples takes as long as one of 64: the block's time is the length of the dependent
+// kernel chain, and a split only hides the small throughput-bound part (attention over the cache, partial sums), while
+// every chain streams the weights again.  So: two chains from 32 samples up, otherwise one.
 static int seq_chain_count(const tf_model* m, int B) {
-  int n = m->seq_chains_force;
-  if (n <= 0) {
-    const size_t w_block = (size_t)m->cfg.n_layers * ((size_t)4 * m->d * m->d + (size_t)2 * m->hid * m->d) * sizeof(bf16);
-    n = w_block <= ((size_t)48 << 20) ? 4 : 2;
-  }
+  int n = m->seq_chains_force > 0 ? m->seq_chains_force : (B >= 32 ? 2 : 1);
   if (n > tf_model::MAX_CHAINS) n = tf_model::MAX_CHAINS;
   while (n > 1 && B / n < 4) n /= 2;  // at least four samples per chain
   return n < 1 ? 1 : n;
@@ -767,7 +774,7 @@ static int run_sequential_chain(tf_model* m, const SeqCtx& cx, int g, const int*
     return check_launch("sequential block");
   }
   cudaStream_t run_stream = m->stream;
-  auto key = std::make_tuple(g, cx.b0, cx.B);
+  auto key = std::make_tuple(g, cx.b0, cx.B, m->seq_variant);
   auto it = m->seq_graphs.find(key);
   if (it == m->seq_graphs.end()) {
     tf_model::SeqGraph sg;
@@ -887,12 +894,29 @@ static int take_labels(tf_model* m, const int** labels, int B) {
   return TF_OK;
 }
 
+// Options of one inverse call beyond the policy (all optional; see tf_jacobi_opts in tarflow.h).
+struct InvOpts {
+  int init_mode = 0;
+  const float* u0_img = nullptr;        // [n_blocks][B][C][H][W]
+  const float* tau_block = nullptr;     // host [n_blocks]
+  int fallback_sweeps = 0;
+  float* states_img = nullptr;          // out [n_blocks][B][C][H][W]
+  const float* ref_img = nullptr;       // in  [n_blocks][B][C][H][W]
+};
+
+static int layout(tf_model* m, float* img, float* seq, int B, int to_seq);
+template <class T>
+static int run_sequential_any(tf_model* m, int g, int B, const int* labels, const float* v, float* u);
+
 template <class T>
 static int run_jacobi_block(tf_model* m, int g, int B, const int* labels, const float* v, float* u, float tau,
-                            int max_iters, int init_mode, int* sweeps_out, int* iters_row) {
-  const size_t n = (size_t)B * m->L * m->D;
-  if (init_mode == 0) CU_OK(cudaMemsetAsync(u, 0, n * sizeof(float), m->stream));
-  else CU_OK(cudaMemcpyAsync(u, v, n * sizeof(float), cudaMemcpyDeviceToDevice, m->stream));
+                            int max_iters, const InvOpts& op, int* sweeps_out, int* iters_row) {
+  const size_t n = (size_t)B * m->L * m->D, img = (size_t)B * m->cfg.C * m->cfg.H * m->cfg.W;
+  if (op.init_mode == 0) CU_OK(cudaMemsetAsync(u, 0, n * sizeof(float), m->stream));
+  else if (op.init_mode == 1) CU_OK(cudaMemcpyAsync(u, v, n * sizeof(float), cudaMemcpyDeviceToDevice, m->stream));
+  else TF_TRY(layout(m, const_cast<float*>(op.u0_img) + (size_t)g * img, u, B, 1));
+  const bool l2 = m->trace_on && op.ref_img != nullptr && m->trace_l2 != nullptr;
+  if (l2) TF_TRY(layout(m, const_cast<float*>(op.ref_img) + (size_t)g * img, m->ref_seq, B, 1));
   // precision policy (bf16 engine): which sweeps of a sample use two-term operands
   int start_phase = 0;
   float sw = -1.f;  // never escalate
@@ -902,14 +926,20 @@ static int run_jacobi_block(tf_model* m, int g, int B, const int* labels, const 
   }
   LAUNCH(m, KC_CTRL, jacobi_begin_kernel, 1, 256, 0, m->maxdiff, m->idx, m->phase, m->ctrl, B, start_phase);
   int n_active = B, n_hp = start_phase ? B : 0, t = 0;
-  while (t < max_iters && n_active > 0) {
+  const int cap = (op.fallback_sweeps > 0 && op.fallback_sweeps < max_iters) ? op.fallback_sweeps : max_iters;
+  while (t < cap && n_active > 0) {
     ++t;
     const int n_lp = n_active - n_hp;
     if (n_lp > 0) TF_TRY(run_pass<T>(m, g, n_lp, u, m->idx, labels, PASS_JACOBI, v, u, false));
     if (n_hp > 0) TF_TRY(run_pass<T>(m, g, n_hp, u, m->idx + n_lp, labels, PASS_JACOBI, v, u, true));
     LAUNCH_PDL(m, KC_CTRL, jacobi_finalize_kernel, 1, 256, 0, m->maxdiff, m->idx, m->idx_tmp, m->phase, m->ctrl, iters_row,
            tau, sw, t);
-    if (tau >= 0.f || t == max_iters || m->trace_on) {
+    if (l2 && t <= m->trace_l2_sweeps) {
+      LAUNCH(m, KC_CTRL, l2_distance_kernel, B, 256, 0, u, m->ref_seq,
+             m->trace_l2 + ((size_t)g * m->trace_l2_sweeps + (t - 1)) * m->cfg.max_batch, m->L * m->D);
+      m->trace_l2_count[g] = t;
+    }
+    if (tau >= 0.f || t == cap || m->trace_on) {
       const int before = n_active;
       TF_TRY(read_ctrl(m));
       n_active = m->ctrl_host[0];
@@ -922,6 +952,29 @@ static int run_jacobi_block(tf_model* m, int g, int B, const int* labels, const 
     }
   }
   *sweeps_out = t;
+  if (tau >= 0.f && n_active > 0 && cap < max_iters) {
+    // Fall-back: the samples still in the active list are decoded sequentially from the block's input (Eq. 5), as a
+    // dense batch of their own; their count becomes sweeps + L - 1.
+    const int nf = m->L * m->D, nb = n_active;
+    int gb = (int)(((size_t)nb * nf + 255) / 256);
+    if (gb > 148 * 16) gb = 148 * 16;
+    LAUNCH(m, KC_LAYOUT, gather_rows_kernel, gb, 256, 0, v, m->cmp_v, m->idx, nb, nf, 1);
+    const int* lab_c = nullptr;
+    if (labels) {
+      LAUNCH(m, KC_LAYOUT, gather_int_kernel, (nb + 127) / 128, 128, 0, labels, m->cmp_labels, m->idx, nb);
+      lab_c = m->cmp_labels;
+    }
+    TF_TRY(check_launch("gather kernels"));
+    m->seq_variant = 1;
+    int r = run_sequential_any<T>(m, g, nb, lab_c, m->cmp_v, m->cmp_u);
+    m->seq_variant = 0;
+    TF_TRY(r);
+    LAUNCH(m, KC_LAYOUT, gather_rows_kernel, gb, 256, 0, m->cmp_u, u, m->idx, nb, nf, 0);
+    LAUNCH(m, KC_CTRL, add_int_rows_kernel, (nb + 127) / 128, 128, 0, iters_row, m->idx, nb, m->L - 1);
+    TF_TRY(check_launch("scatter kernels"));
+    *sweeps_out = t + m->L - 1;
+    return TF_OK;
+  }
   return (tau >= 0.f && n_active > 0) ? TF_MAXITER : TF_OK;
 }
 
@@ -937,29 +990,41 @@ static int layout(tf_model* m, float* img, float* seq, int B, int to_seq) {
 }
 
 template <class T>
+static int run_sequential_any(tf_model* m, int g, int B, const int* labels, const float* v, float* u) {
+  if constexpr (sizeof(T) == 2) return run_sequential_block_bf16(m, g, B, labels, v, u);
+  else return run_sequential_block<T>(m, g, B, labels, v, u);
+}
+
+template <class T>
 static int inverse_impl(tf_model* m, const float* z, const int* labels, int B, const uint8_t* policy, float tau,
-                        int max_iters, int init_mode, float* x, int* iters_block_host, int* iters_sample_dev) {
+                        int max_iters, const InvOpts& op, float* x, int* iters_block_host, int* iters_sample_dev) {
   const int K = m->cfg.n_blocks;
+  const size_t img = (size_t)B * m->cfg.C * m->cfg.H * m->cfg.W;
   float *v = m->seq_a, *u = m->seq_b;
   m->trace.clear();
+  m->trace_l2_count.assign(K, 0);
   TF_TRY(take_labels(m, &labels, B));
   TF_TRY(layout(m, const_cast<float*>(z), v, B, 1));
   int status = TF_OK;
   for (int g = 0; g < K; ++g) {
     int* iters_row = m->iters_sample + (size_t)g * m->cfg.max_batch;
     int sweeps = m->L - 1;
+    if (m->block_ev[g]) cudaEventRecord(m->block_ev[g], m->stream);
     if (policy[g] == 0) {
-      if constexpr (sizeof(T) == 2) TF_TRY(run_sequential_block_bf16(m, g, B, labels, v, u));
-      else TF_TRY(run_sequential_block<T>(m, g, B, labels, v, u));
+      TF_TRY(run_sequential_any<T>(m, g, B, labels, v, u));
       LAUNCH(m, KC_CTRL, fill_int_kernel, (B + 127) / 128, 128, 0, iters_row, B, m->L - 1);
     } else {
-      int r = run_jacobi_block<T>(m, g, B, labels, v, u, tau, max_iters, init_mode, &sweeps, iters_row);
+      const float tau_g = op.tau_block ? op.tau_block[g] : tau;
+      int r = run_jacobi_block<T>(m, g, B, labels, v, u, tau_g, max_iters, op, &sweeps, iters_row);
       if (r < 0) return r;
       if (r == TF_MAXITER) status = TF_MAXITER;
     }
     if (iters_block_host) iters_block_host[g] = sweeps;
+    if (op.states_img) TF_TRY(layout(m, op.states_img + (size_t)g * img, u, B, 0));
     float* tmp = v; v = u; u = tmp;
   }
+  if (m->block_ev[K]) cudaEventRecord(m->block_ev[K], m->stream);
+  m->block_ev_valid = true;
   TF_TRY(layout(m, x, v, B, 0));
   if (iters_sample_dev) {
     for (int g = 0; g < K; ++g)
@@ -1106,6 +1171,10 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
   const size_t B = c.max_batch, M = B * L, esz = c.dtype == 1 ? 2 : 4;
   TF_TRY(dev_alloc(m, &m->seq_a, M * D));
   TF_TRY(dev_alloc(m, &m->seq_b, M * D));
+  TF_TRY(dev_alloc(m, &m->cmp_v, M * D));
+  TF_TRY(dev_alloc(m, &m->cmp_u, M * D));
+  TF_TRY(dev_alloc(m, &m->ref_seq, M * D));
+  TF_TRY(dev_alloc(m, &m->cmp_labels, B));
   TF_TRY(dev_alloc(m, &m->h, M * d));
   TF_TRY(dev_alloc(m, &m->o, M * 2 * D));
   TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->xn), M * d * esz));
@@ -1145,6 +1214,8 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
   CU_OK(cudaMemset(m->err, 0, sizeof(int)));
   CU_OK(cudaMemset(m->iters_sample, 0, (size_t)c.n_blocks * B * sizeof(int)));
   CU_OK(cudaMallocHost(&m->ctrl_host, 8 * sizeof(int)));
+  m->block_ev.assign(c.n_blocks + 1, nullptr);
+  for (auto& e : m->block_ev) CU_OK(cudaEventCreate(&e));
   if (c.dtype == 1) {
     TF_TRY(make_map_bf16(&m->map_xn, m->xn, M, d, tc::BM));
     TF_TRY(make_map_bf16(&m->map_att, m->att, M, d, tc::BM));
@@ -1261,6 +1332,7 @@ void tf_free(tf_model* m) {
   cudaDeviceSynchronize();
   m->prof_collect();
   for (cudaEvent_t e : m->ev_pool) cudaEventDestroy(e);
+  for (cudaEvent_t e : m->block_ev) if (e) cudaEventDestroy(e);
   for (auto& kv : m->seq_graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
   if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
   for (int c = 0; c < tf_model::MAX_CHAINS; ++c) {
@@ -1284,23 +1356,67 @@ int tf_forward(tf_model* m, const float* x_dev, const int32_t* labels_dev, int32
                            : forward_impl<float>(m, x_dev, labels_dev, B, z_dev, logdet_dev);
 }
 
-int tf_inverse_jacobi(tf_model* m, const float* z_dev, const int32_t* labels_dev, int32_t B, const uint8_t* policy_host,
-                      float tau, int32_t max_iters, int32_t init_mode, float* x_dev, int32_t* iters_block_host,
-                      int32_t* iters_sample_dev, void* cuda_stream) {
-  g_err[0] = 0;
+static int inverse_checked(tf_model* m, const float* z_dev, const int32_t* labels_dev, int32_t B, const uint8_t* policy_host,
+                           float tau, int32_t max_iters, const InvOpts& op, float* x_dev, int32_t* iters_block_host,
+                           int32_t* iters_sample_dev, void* cuda_stream) {
   TF_TRY(check_call(m, B));
   if (!z_dev || !x_dev || !policy_host) return fail(TF_EINVAL, "NULL buffer");
   if (m->cfg.n_classes > 0 && !labels_dev) return fail(TF_EINVAL, "class-conditional model needs labels");
   if (max_iters < 1) return fail(TF_EINVAL, "max_iters must be >= 1");
-  if (init_mode != 0 && init_mode != 1) return fail(TF_EINVAL, "init_mode must be 0 or 1");
+  if (op.init_mode < 0 || op.init_mode > 2) return fail(TF_EINVAL, "init_mode must be 0, 1 or 2");
+  if (op.init_mode == 2 && !op.u0_img) return fail(TF_EINVAL, "init_mode 2 needs u0_dev");
+  if (op.fallback_sweeps < 0) return fail(TF_EINVAL, "fallback_sweeps must be >= 0");
   if (tau != tau) return fail(TF_EINVAL, "tau is NaN");
-  for (int g = 0; g < m->cfg.n_blocks; ++g)
+  for (int g = 0; g < m->cfg.n_blocks; ++g) {
     if (policy_host[g] > 1) return fail(TF_EINVAL, "policy[%d]=%d is neither 0 nor 1", g, (int)policy_host[g]);
+    if (op.tau_block && op.tau_block[g] != op.tau_block[g]) return fail(TF_EINVAL, "tau_block[%d] is NaN", g);
+  }
   m->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
-  return m->cfg.dtype == 1 ? inverse_impl<bf16>(m, z_dev, labels_dev, B, policy_host, tau, max_iters, init_mode, x_dev,
+  return m->cfg.dtype == 1 ? inverse_impl<bf16>(m, z_dev, labels_dev, B, policy_host, tau, max_iters, op, x_dev,
                                                 iters_block_host, iters_sample_dev)
-                           : inverse_impl<float>(m, z_dev, labels_dev, B, policy_host, tau, max_iters, init_mode, x_dev,
+                           : inverse_impl<float>(m, z_dev, labels_dev, B, policy_host, tau, max_iters, op, x_dev,
                                                  iters_block_host, iters_sample_dev);
+}
+
+int tf_inverse_jacobi(tf_model* m, const float* z_dev, const int32_t* labels_dev, int32_t B, const uint8_t* policy_host,
+                      float tau, int32_t max_iters, int32_t init_mode, float* x_dev, int32_t* iters_block_host,
+                      int32_t* iters_sample_dev, void* cuda_stream) {
+  g_err[0] = 0;
+  if (init_mode != 0 && init_mode != 1) return fail(TF_EINVAL, "init_mode must be 0 or 1");
+  InvOpts op;
+  op.init_mode = init_mode;
+  return inverse_checked(m, z_dev, labels_dev, B, policy_host, tau, max_iters, op, x_dev, iters_block_host, iters_sample_dev,
+                         cuda_stream);
+}
+
+int tf_inverse_jacobi_ex(tf_model* m, const float* z_dev, const int32_t* labels_dev, int32_t B, const uint8_t* policy_host,
+                         float tau, int32_t max_iters, const tf_jacobi_opts* opts, float* x_dev, int32_t* iters_block_host,
+                         int32_t* iters_sample_dev, void* cuda_stream) {
+  g_err[0] = 0;
+  InvOpts op;
+  if (opts) {
+    if (opts->struct_bytes != (int32_t)sizeof(tf_jacobi_opts)) return fail(TF_EINVAL, "tf_jacobi_opts.struct_bytes is %d, expected %d", opts->struct_bytes, (int)sizeof(tf_jacobi_opts));
+    op.init_mode = opts->init_mode;
+    op.u0_img = opts->u0_dev;
+    op.tau_block = opts->tau_block_host;
+    op.fallback_sweeps = opts->fallback_sweeps;
+    op.states_img = opts->states_dev;
+    op.ref_img = opts->ref_states_dev;
+  }
+  return inverse_checked(m, z_dev, labels_dev, B, policy_host, tau, max_iters, op, x_dev, iters_block_host, iters_sample_dev,
+                         cuda_stream);
+}
+
+int tf_block_times(tf_model* m, float* ms_host, int32_t cap) {
+  if (!m) return fail(TF_EINVAL, "model is NULL");
+  const int K = m->cfg.n_blocks;
+  if (!m->block_ev_valid) return 0;
+  for (int g = 0; g < K && g < cap; ++g) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, m->block_ev[g], m->block_ev[g + 1]) != cudaSuccess) { cudaGetLastError(); return 0; }
+    if (ms_host) ms_host[g] = ms;
+  }
+  return K;
 }
 
 int tf_inverse_sequential(tf_model* m, const float* z_dev, const int32_t* labels_dev, int32_t B, float* x_dev,
@@ -1494,7 +1610,23 @@ int tf_trace_enable(tf_model* m, int32_t on) {
   if (!m) return fail(TF_EINVAL, "model is NULL");
   m->trace_on = on != 0;
   m->trace.clear();
+  m->trace_l2_count.assign(m->cfg.n_blocks, 0);
+  if (m->trace_on && !m->trace_l2) {  // distance records: up to L + 2 sweeps per block
+    m->trace_l2_sweeps = m->L + 2;
+    TF_TRY(dev_alloc(m, &m->trace_l2, (size_t)m->cfg.n_blocks * m->trace_l2_sweeps * m->cfg.max_batch));
+  }
   return TF_OK;
+}
+
+int tf_trace_read_l2(tf_model* m, int32_t block, int32_t B, float* l2_host, int32_t cap_sweeps) {
+  if (!m) return fail(TF_EINVAL, "model is NULL");
+  if (block < 0 || block >= m->cfg.n_blocks || B < 1 || B > m->cfg.max_batch) return fail(TF_EINVAL, "bad block or batch");
+  if (!m->trace_l2 || m->trace_l2_count.empty()) return 0;
+  const int n = m->trace_l2_count[block];
+  for (int t = 0; t < n && t < cap_sweeps && l2_host; ++t)
+    CU_OK(cudaMemcpy(l2_host + (size_t)t * B, m->trace_l2 + ((size_t)block * m->trace_l2_sweeps + t) * m->cfg.max_batch,
+                     B * sizeof(float), cudaMemcpyDeviceToHost));
+  return n;
 }
 
 int tf_trace_read(tf_model* m, int32_t* block, int32_t* sweep, int32_t* active, float* maxdiff, int32_t cap) {

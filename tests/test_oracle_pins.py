@@ -323,3 +323,84 @@ def test_cfg1_selective_policy_close_to_sequential():
     assert np.abs(x - x_seq).max() < 1e-4
     z2, ld = O.model_forward(blocks, x_seq, None, cfg)
     assert np.abs(z2 - z).max() < 1e-9
+
+
+# ---------------------------------------------------------------- variants around Algorithm 1
+def test_any_initial_iterate_reaches_the_sequential_solution_in_L_sweeps():
+    """Prop. 3.2's induction never uses u^0: from zeros, from the block input and from random draws, L sweeps
+    give the sequential solution exactly and after t sweeps the first t tokens are already exact."""
+    cfg, blocks = _model(H=2, W=5, patch=1, C=2, n_blocks=2)
+    L = synth.seq_len(cfg)
+    rng = np.random.default_rng(21)
+    z = rng.standard_normal((3, cfg["C"], cfg["H"], cfg["W"]))
+    u0 = rng.standard_normal((2, 3, cfg["C"], cfg["H"], cfg["W"]))
+    x_seq = O.model_inverse_sequential(blocks, z, None, cfg)
+    for mode in (0, 1, 2):
+        x, it = O.model_inverse(blocks, z, None, cfg, [1, 1], -1.0, L, init_mode=mode, u0=u0)
+        assert np.abs(x - x_seq).max() < 1e-12 and np.all(it == L)
+    # the start really is used: after one sweep only token 1 is fixed (it copies v_1), the rest depends on u^0
+    v = O.patchify(z, 1)
+    outs = [O.block_inverse_jacobi(blocks[0], v, None, cfg, -1.0, 1, u0=s)[0]
+            for s in (None, v, O.patchify(u0[0], 1))]
+    assert np.array_equal(outs[0][:, :1], outs[1][:, :1]) and np.array_equal(outs[0][:, :1], outs[2][:, :1])
+    assert np.abs(outs[0][:, 1:] - outs[1][:, 1:]).max() > 1e-3 and np.abs(outs[0][:, 1:] - outs[2][:, 1:]).max() > 1e-3
+
+
+def test_per_block_tau_equals_uniform_tau_blockwise_and_states_chain():
+    cfg, blocks = _model(H=2, W=4, patch=1, C=2, n_blocks=3, head_scale=0.3)
+    L = synth.seq_len(cfg)
+    rng = np.random.default_rng(22)
+    z = rng.standard_normal((2, cfg["C"], cfg["H"], cfg["W"]))
+    taus = [1e-2, 1e-6, 1e-4]
+    x, it, ex = O.model_inverse(blocks, z, None, cfg, [1, 1, 1], taus, L + 1, return_states=True)
+    # chaining single blocks by hand with each block's own tau gives the same states and counts
+    seq = O.patchify(z, 1)
+    for g in range(3):
+        u, itg, _ = O.block_inverse_jacobi(blocks[g], np.ascontiguousarray(O.permute(seq, g)), None, cfg, taus[g], L + 1)
+        seq = np.ascontiguousarray(O.permute(u, g))
+        assert np.array_equal(O.unpatchify(seq, cfg["C"], cfg["H"], cfg["W"], 1), ex["states"][g])
+        assert np.array_equal(itg, it[g])
+    assert np.array_equal(ex["states"][-1], x)
+    assert it[1].min() > it[0].max()            # the tighter threshold costs sweeps
+    xu, itu = O.model_inverse(blocks, z, None, cfg, [1, 1, 1], 1e-6, L + 1)
+    xl, itl = O.model_inverse(blocks, z, None, cfg, [1, 1, 1], [1e-6] * 3, L + 1)
+    assert np.array_equal(xu, xl) and np.array_equal(itu, itl)
+
+
+def test_fallback_decodes_exactly_the_stragglers_sequentially():
+    cfg, blocks = _model(H=2, W=6, patch=1, C=2, n_blocks=1, head_scale=0.5)
+    L = synth.seq_len(cfg)
+    rng = np.random.default_rng(12)
+    z = rng.standard_normal((4, cfg["C"], cfg["H"], cfg["W"]))
+    x_plain, it_plain = O.model_inverse(blocks, z, None, cfg, [1], 1e-3, L + 1)
+    x_seq = O.model_inverse_sequential(blocks, z, None, cfg)
+    cut = int(it_plain[0].min()) + 1             # some samples are done by then, others are not
+    assert it_plain[0].min() <= cut < it_plain[0].max()
+    x_fb, it_fb = O.model_inverse(blocks, z, None, cfg, [1], 1e-3, L + 1, fallback_sweeps=cut)
+    done = it_plain[0] <= cut
+    assert done.any() and (~done).any()
+    assert np.array_equal(x_fb[done], x_plain[done]) and np.array_equal(it_fb[0][done], it_plain[0][done])
+    assert np.array_equal(x_fb[~done], x_seq[~done])            # bit-identical to Eq. 5 for the stragglers
+    assert np.all(it_fb[0][~done] == cut + L - 1)
+    # a cut that nobody reaches, a cut at or beyond max_iters, and fixed-iteration mode change nothing
+    for kw in (dict(fallback_sweeps=int(it_plain.max())), dict(fallback_sweeps=L + 1)):
+        x2, it2 = O.model_inverse(blocks, z, None, cfg, [1], 1e-3, L + 1, **kw)
+        assert np.array_equal(x2, x_plain) and np.array_equal(it2, it_plain)
+    x3, it3 = O.model_inverse(blocks, z, None, cfg, [1], -1.0, 5, fallback_sweeps=2)
+    assert np.all(it3 == 5)
+
+
+def test_distance_trace_matches_direct_norms_and_ends_at_zero():
+    cfg, blocks = _model(H=2, W=4, patch=1, C=2, n_blocks=2)
+    L = synth.seq_len(cfg)
+    rng = np.random.default_rng(23)
+    z = rng.standard_normal((2, cfg["C"], cfg["H"], cfg["W"]))
+    _, _, ref = O.model_inverse(blocks, z, None, cfg, [0, 0], 0.0, 1, return_states=True)
+    x, it, ex = O.model_inverse(blocks, z, None, cfg, [1, 1], -1.0, L, ref_states=ref["states"], return_states=True)
+    for g in range(2):
+        tr = ex["l2"][g]
+        assert tr.shape == (L, 2)
+        assert np.all(tr[-1] < 1e-12)                          # u^L = sequential solution (Prop. 3.2)
+        assert np.all(tr[0] > 1e-3)
+        d = np.sqrt(((ex["states"][g] - ref["states"][g]) ** 2).reshape(2, -1).sum(axis=1))
+        assert np.allclose(tr[-1], d, atol=1e-12)
