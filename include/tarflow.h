@@ -239,7 +239,9 @@ int tf_gemm_status(void* cuda_stream);
 /*
  * Profiling aid: when enabled, calls on this model bracket every kernel class with CUDA events on
  * the caller's stream and accumulate elapsed milliseconds and launch counts.
- *   tf_profile_enable(m, on): switch on/off and reset the counters.
+ *   tf_profile_enable(m, on): switch on (1), off (0) and reset the counters.  on == 2: the kernels of Jacobi sweeps
+ *     are bracketed one by one as with 1, while a sequentially decoded block runs exactly as it does unprofiled
+ *     (replayed graphs, sample chains) and is timed as ONE unit of the class "seq_block" (rows = B * (L - 1)).
  *   tf_profile_read(m, names, ms, launches, rows, cap): fills up to cap entries, returns how many
  *     classes exist; names[i] points to a static string; rows[i] is the number of activation
  *     rows (tokens of a sweep, samples of a sequential step) the class's launches processed.

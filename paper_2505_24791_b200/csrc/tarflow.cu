@@ -121,12 +121,12 @@ static int make_map_3d(CUtensorMap* map, const void* ptr, uint64_t slots, uint64
 // ------------------------------------------------------------------------------------------------
 enum KernelClass {
   KC_LAYOUT, KC_EMBED, KC_LN, KC_GEMM_QKV, KC_ATTN, KC_GEMM_O, KC_GEMM_MLP1, KC_GEMM_MLP2, KC_GEMM_HEAD_UPDATE,
-  KC_GEMM_HEAD, KC_AFFINE, KC_CTRL, KC_SEQ_EMBED, KC_SEQ_LN, KC_SEQ_GEMM, KC_SEQ_ATTN, KC_SEQ_UPDATE, KC_COUNT
+  KC_GEMM_HEAD, KC_AFFINE, KC_CTRL, KC_SEQ_EMBED, KC_SEQ_LN, KC_SEQ_GEMM, KC_SEQ_ATTN, KC_SEQ_UPDATE, KC_SEQ_BLOCK, KC_COUNT
 };
 static const char* kKernelClassNames[KC_COUNT] = {
     "layout", "embed", "layernorm", "gemm_qkv", "attention", "gemm_out", "gemm_mlp_up", "gemm_mlp_down",
     "gemm_head_update", "gemm_head", "forward_affine", "sweep_control", "seq_embed", "seq_layernorm", "seq_gemm",
-    "seq_attention", "seq_update"};
+    "seq_attention", "seq_update", "seq_block"};
 
 struct Matrix {       // a linear layer's weight [N, K]
   void* w = nullptr;  // float* or bf16*
@@ -205,6 +205,8 @@ struct tf_model {
   int64_t launches = 0;
   // profiling
   bool prof_on = false;
+  int prof_mode = 0;       // 1: every launch; 2: sweep kernels per launch, a sequential block as one timed unit (from its graph)
+  bool prof_suspend = false;
   std::vector<cudaEvent_t> ev_pool;
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> ev_pending[KC_COUNT];
   double prof_ms[KC_COUNT] = {0};
@@ -230,14 +232,14 @@ struct tf_model {
     return e;
   }
   void pre(int) {
-    if (prof_on) {
+    if (prof_on && !prof_suspend) {
       cur_start = get_event();
       cudaEventRecord(cur_start, stream);
     }
   }
   void post(int cls) {
     ++launches;
-    if (prof_on) {
+    if (prof_on && !prof_suspend) {
       cudaEvent_t e = get_event();
       cudaEventRecord(e, stream);
       ev_pending[cls].push_back({cur_start, e});
@@ -766,7 +768,7 @@ static int run_sequential_chain(tf_model* m, const SeqCtx& cx, int g, const int*
   m->cur_rows = cx.B;
   if (seq_tail_fused(m)) TF_TRY(seq_tail(m, cx, g, labels, v, u, nullptr, 0, 1, 0));
   else TF_TRY(seq_update_embed(m, cx, g, labels, v, u, 0, 1, 0));
-  if (m->prof_on || !m->use_graphs) {  // direct launches (per-kernel events need them)
+  if ((m->prof_on && m->prof_mode == 1) || !m->use_graphs) {  // direct launches (per-kernel events need them)
     for (int t = 0; t < n_steps; ++t) {
       TF_TRY(seq_enqueue_steps(m, cx, g, labels, v, u, 1));
       TF_TRY(launch_seq(m, KC_CTRL, seq::seq_advance_kernel, dim3(1), 32, 0, cx.step_ctr, 1));
@@ -812,7 +814,7 @@ static int run_sequential_chain(tf_model* m, const SeqCtx& cx, int g, const int*
 static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* labels, const float* v, float* u) {
   const int n_steps = m->L - 1;
   cudaStream_t user = m->stream;
-  const bool direct = m->prof_on || !m->use_graphs;
+  const bool direct = (m->prof_on && m->prof_mode == 1) || !m->use_graphs;
   m->seq_check_steps = direct ? 0 : (n_steps % seq_unroll(n_steps) != 0);
   const int nch = direct ? 1 : seq_chain_count(m, B);
   if (nch == 1) {
@@ -991,8 +993,23 @@ static int layout(tf_model* m, float* img, float* seq, int B, int to_seq) {
 
 template <class T>
 static int run_sequential_any(tf_model* m, int g, int B, const int* labels, const float* v, float* u) {
-  if constexpr (sizeof(T) == 2) return run_sequential_block_bf16(m, g, B, labels, v, u);
-  else return run_sequential_block<T>(m, g, B, labels, v, u);
+  const bool unit = m->prof_on && m->prof_mode == 2;  // time the whole block as one unit of class seq_block
+  if (unit) {
+    m->cur_rows = (int64_t)B * (m->L - 1);
+    m->pre(KC_SEQ_BLOCK);
+    m->prof_suspend = true;
+  }
+  int r;
+  if constexpr (sizeof(T) == 2) r = run_sequential_block_bf16(m, g, B, labels, v, u);
+  else r = run_sequential_block<T>(m, g, B, labels, v, u);
+  if (unit) {
+    m->prof_suspend = false;
+    m->cur_rows = (int64_t)B * (m->L - 1);
+    const int64_t keep = m->launches;
+    m->post(KC_SEQ_BLOCK);
+    m->launches = keep;
+  }
+  return r;
 }
 
 template <class T>
@@ -1582,6 +1599,7 @@ int tf_profile_enable(tf_model* m, int32_t on) {
   m->prof_collect();
   for (int c = 0; c < KC_COUNT; ++c) { m->prof_ms[c] = 0; m->prof_n[c] = 0; m->prof_rows[c] = 0; }
   m->prof_on = on != 0;
+  m->prof_mode = on == 2 ? 2 : (on != 0 ? 1 : 0);
   return TF_OK;
 }
 
