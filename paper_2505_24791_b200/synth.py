@@ -189,3 +189,79 @@ def shard_batch(B: int, rank: int, world: int):
     base, rem = divmod(B, world)
     start = rank * base + min(rank, rem)
     return start, start + base + (1 if rank < rem else 0)
+
+
+# ------------------------------------------------------------------------------------------------
+# second workload: masked autoregressive flow (MLP-based, Jacobi decoding on every layer)
+# ------------------------------------------------------------------------------------------------
+MAF_MAGIC = 0x3146414D  # "MAF1" little endian
+
+# The paper's two MAF experiments are an 8-layer flow on a 2-D Ising lattice (100 000 samples) and an 8-layer flow
+# on binary MNIST (100 images); lattice size and hidden width are not stated, so these stand-ins fix them.
+MAF_CONFIGS = {
+    "maf_tiny": dict(D=12, hidden=32, n_blocks=3, dtype=0, B=5, tau=1e-6, z_scale=1.0),
+    "maf_ising": dict(D=256, hidden=1024, n_blocks=8, dtype=1, B=16384, tau=1e-3, z_scale=1.0),
+    "maf_mnist": dict(D=784, hidden=1024, n_blocks=8, dtype=1, B=100, tau=1e-3, z_scale=1.0),
+}
+
+
+def maf_config(name: str, **overrides) -> dict:
+    cfg = dict(MAF_CONFIGS[name])
+    cfg.update(overrides)
+    return cfg
+
+
+def maf_tensor_specs(cfg):
+    D, H = cfg["D"], cfg["hidden"]
+    return [("w1", (H, D)), ("b1", (H,)), ("w2", (H, H)), ("b2", (H,)), ("w3", (2 * D, H)), ("b3", (2 * D,))]
+
+
+def make_maf_weights(cfg, seed: int = WEIGHT_SEED, out_scale: float = 0.1, zero_out: bool = False):
+    """Seeded dense weights of every layer (no masks applied: masking is the method's, done by each side itself).
+
+    Hidden matrices: normal with std sqrt(2 / fan_in) scaled by sqrt(2) (about half of a row is masked away);
+    output matrix std = out_scale / sqrt(hidden / 2) so that mu and alpha have standard deviation of the order of
+    out_scale; biases std 0.02.  For dtype == 1 the matrices are rounded to bf16-representable values.
+    """
+    blocks = []
+    for g in range(cfg["n_blocks"]):
+        blk = {}
+        for ti, (name, shape) in enumerate(maf_tensor_specs(cfg)):
+            n = _rng(seed, 0x3AF, g, ti).standard_normal(shape, dtype=np.float32)
+            if name in ("w1", "w2"):
+                t = n * np.float32(2.0 / np.sqrt(shape[1]))
+            elif name == "w3":
+                t = n * np.float32(0.0 if zero_out else out_scale / np.sqrt(shape[1] / 2.0))
+            elif name == "b3":
+                t = n * np.float32(0.0 if zero_out else 0.02)
+            else:
+                t = n * np.float32(0.02)
+            if cfg["dtype"] == 1 and name.startswith("w"):
+                t = round_to_bf16(t)
+            blk[name] = np.ascontiguousarray(t, dtype=np.float32)
+        blocks.append(blk)
+    return blocks
+
+
+def pack_maf_blob(cfg, blocks, seed: int = WEIGHT_SEED) -> np.ndarray:
+    """16 int32 header {magic, version, D, hidden, n_blocks, dtype, seed, 0...} then the fp32 tensors of every layer."""
+    hdr = np.zeros(HEADER_INTS, dtype=np.int32)
+    hdr[:7] = [MAF_MAGIC, VERSION, cfg["D"], cfg["hidden"], cfg["n_blocks"], cfg["dtype"], seed]
+    parts = [hdr.view(np.uint8)]
+    for blk in blocks:
+        for name, shape in maf_tensor_specs(cfg):
+            a = blk[name]
+            assert a.shape == tuple(shape) and a.dtype == np.float32, name
+            parts.append(a.reshape(-1).view(np.uint8))
+    return np.concatenate(parts)
+
+
+def make_maf_latents(cfg, seed: int, B: int | None = None) -> np.ndarray:
+    """z ~ N(0,1) * z_scale, [B, D] fp32; row b depends only on (seed, b)."""
+    B = cfg["B"] if B is None else B
+    z = np.empty((B, cfg["D"]), dtype=np.float32)
+    blk = 4096
+    for b0 in range(0, B, blk):   # a generator per group of rows keeps large batches quick to draw
+        n = min(blk, B - b0)
+        z[b0:b0 + n] = _rng(seed, 0x3A11CE, b0).standard_normal((n, cfg["D"]), dtype=np.float32)
+    return z * np.float32(cfg["z_scale"])
