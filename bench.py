@@ -16,6 +16,7 @@ synthetic latents.  The line printed by rank 0 carries:
   blocks    device time per block (events recorded in the timed pass itself), sweeps and active samples per sweep,
   gpu_sequential / gpu_all_jacobi   the same batch decoded with the other policies,
   other_workloads   short legs on the other bf16 configurations (selective / sequential / all-Jacobi),
+  second_workload_maf   Jacobi against sequential decoding of an MLP-based autoregressive flow (paper App. E.3),
   cpu_baseline   the fp64 CPU oracle timed on this machine's host cores on a bounded sub-batch.
 `--impl reference` times only the CPU oracle (there is no other implementation of the paper).
 With N > 1 every rank decodes its own batch (weak scaling, no data-path collective); `--gpus N` without a
@@ -337,6 +338,8 @@ def main():
     ap.add_argument("--no-policies", action="store_true", help="skip the all-sequential / all-Jacobi legs")
     ap.add_argument("--no-legs", action="store_true", help="skip the short legs on the other bf16 configurations")
     ap.add_argument("--kernels", action="store_true", help="add the per-kernel-class table to the JSON line")
+    ap.add_argument("--maf", default=None, choices=["maf_ising", "maf_mnist"],
+                    help="only the second workload (MLP-based flow, Jacobi on every layer): one JSON line, not the bench line")
     ap.add_argument("--sweep", default=None, choices=["cfg5"],
                     help="policy x batch x tau table on the class-conditional architecture (one JSON line, not the bench line)")
     ap.add_argument("--probe", default=None, choices=["sweep", "seq"],
@@ -353,7 +356,7 @@ def main():
         args.warmup = 3
 
     # `--gpus N` outside a torchrun environment: start the N ranks (one process per GPU) and relay their output
-    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.probe or args.sweep or args.launch_list):
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.probe or args.sweep or args.maf or args.launch_list):
         port = 29500 + (os.getpid() % 2000)
         cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
                "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
@@ -419,6 +422,9 @@ def main():
         return
     if args.sweep:
         run_cfg5_sweep(args, binding, synth, torch, timed)
+        return
+    if args.maf:
+        print(json.dumps({"second_workload_maf": run_maf_leg(args.maf, binding, synth, torch, timed, peaks()[0])}), flush=True)
         return
 
     n_in = args.warmup + args.steps
@@ -555,11 +561,51 @@ def main():
             R2.close()
             del R2
         out["other_workloads"] = legs
+        out["second_workload_maf"] = run_maf_leg("maf_ising", binding, synth, torch, timed, pk)
 
     if rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_maf_leg(name, binding, synth, torch, timed, pk, steps=3):
+    """Second workload (paper App. E.3): Jacobi decoding on every layer of an MLP-based autoregressive flow against
+    sequential decoding (D whole passes per layer, no cache exists).  -> dict for the JSON line."""
+    cfg = synth.maf_config(name)
+    B, D, H, K = cfg["B"], cfg["D"], cfg["hidden"], cfg["n_blocks"]
+    blocks = synth.make_maf_weights(cfg)
+    model = binding.tf_maf_load(cfg, synth.pack_maf_blob(cfg, blocks), B)
+    stream = torch.cuda.current_stream()
+    zs = [torch.from_numpy(synth.make_maf_latents(cfg, 9000 + i, B=B)).cuda() for i in range(steps + 1)]
+    x = torch.empty_like(zs[0])
+    iters = np.zeros(K, dtype=np.int32)
+    its = torch.zeros((K, B), dtype=torch.int32, device="cuda")
+
+    def jac(i):
+        return binding.tf_maf_inverse_jacobi(model, zs[i], B, cfg["tau"], D + 1, 0, x, iters, its, stream)
+
+    jac(0)
+    ms, _, _ = timed(jac, list(range(1, steps + 1)))
+    ms /= steps
+    itn = its.cpu().numpy()
+    flops_row = 2.0 * (D * H + H * H + 2 * D * H)                     # one pass of one sample through one layer
+    rows = float(itn.sum())                                            # sample-sweeps of the last step
+    out = {"config": f"{name}: {D} dimensions, {K} layers, hidden {H}, batch {B}, tau {cfg['tau']}",
+           "jacobi": {"value": B / (ms * 1e-3), "unit": UNIT, "ms_per_step": round(ms, 3), "steps": steps,
+                      "sweeps_max": [int(v) for v in itn.max(axis=1)], "sweeps_mean": [round(float(v), 2) for v in itn.mean(axis=1)],
+                      "ms_per_block": [round(float(v), 3) for v in binding.tf_block_times(model, K)],
+                      "tensor_frac": round(rows * flops_row / (ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"], 4)}}
+    Bs = min(B, 4096)                                                  # sequential decoding: a bounded sub-batch
+    binding.tf_maf_inverse_sequential(model, zs[0][:Bs].contiguous(), Bs, x[:Bs], stream)
+    zsub = [z[:Bs].contiguous() for z in zs]
+    ms_s, _, _ = timed(lambda i: binding.tf_maf_inverse_sequential(model, zsub[i], Bs, x[:Bs], stream), [1])
+    out["sequential"] = {"value": Bs / (ms_s * 1e-3), "unit": UNIT, "ms_per_step": round(ms_s, 3), "steps": 1, "batch": Bs,
+                         "passes_per_layer": D,
+                         "tensor_frac": round(Bs * K * D * flops_row / (ms_s * 1e-3) / 1e12 / pk["bf16_tflops_sustained"], 4)}
+    out["jacobi_over_sequential"] = round(out["jacobi"]["value"] / out["sequential"]["value"], 2)
+    binding.tf_free(model)
+    return out
 
 
 def run_probe(args, B, binding, synth, torch):

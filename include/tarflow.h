@@ -187,6 +187,34 @@ int tf_inverse_jacobi_host(tf_model* m, const float* z_host, const int32_t* labe
                            int32_t* iters_sample_host, void* cuda_stream);
 
 /*
+ * Second workload: Jacobi decoding of an MLP-based masked autoregressive flow (paper App. E.3: Algorithm 1 on every
+ * layer of a flow whose networks have no key/value cache).  Each layer is the affine autoregressive block of Eq. 4 /
+ * Eq. 5 over the D scalar dimensions of a sample, x_i = z_i * exp(alpha_i(x_<i)) + mu_i(x_<i), with (mu, alpha) from a
+ * MADE network (two hidden layers of `hidden` ReLU units; input i and output i have degree i, hidden unit j degree
+ * 1 + (j mod (D - 1)); a hidden unit sees degrees <= its own, an output degrees < its own), and the order of the
+ * dimensions is reversed between layers.  Samples are fp32 [B, D].
+ *   tf_maf_load: blob = 16 int32 header {magic 0x3146414D, version 1, D, hidden, n_blocks, dtype, seed, 0...} then per
+ *     layer the dense fp32 tensors w1 [hidden, D], b1 [hidden], w2 [hidden, hidden], b2 [hidden], w3 [2D, hidden]
+ *     (rows mu | alpha), b3 [2D]; the masks are applied by the library.  bf16 engine: D % 8 == 0, hidden % 64 == 0.
+ *     The model is released with tf_free; tf_set_precision, tf_trace_*, tf_profile_*, tf_block_times,
+ *     tf_launch_count and tf_device_bytes apply to it, the TarFlow calls refuse it (TF_EINVAL) and vice versa.
+ *   tf_maf_forward: x -> z and logdet = -sum(alpha) (Eq. 4 through layers K-1 .. 0).  Synchronises.
+ *   tf_maf_inverse_sequential: Eq. 5, D whole passes of the network per layer (dimension i is final after pass i).
+ *   tf_maf_inverse_jacobi: Algorithm 1 on every layer with the per-sample stopping test (tau, max_iters, init_mode
+ *     0 | 1, outputs as for tf_inverse_jacobi; D sweeps reproduce sequential decoding, Prop. 3.2).  Synchronises.
+ */
+typedef struct {
+  int32_t D, hidden, n_blocks;
+  int32_t dtype;      /* 0 = fp32 SIMT engine, 1 = bf16 tensor-core engine */
+  int32_t max_batch;
+} tf_maf_config;
+int tf_maf_load(const tf_maf_config* cfg, const void* weights_host, size_t nbytes, tf_model** out);
+int tf_maf_forward(tf_model* m, const float* x_dev, int32_t B, float* z_dev, float* logdet_dev, void* cuda_stream);
+int tf_maf_inverse_sequential(tf_model* m, const float* z_dev, int32_t B, float* x_dev, void* cuda_stream);
+int tf_maf_inverse_jacobi(tf_model* m, const float* z_dev, int32_t B, float tau, int32_t max_iters, int32_t init_mode,
+                          float* x_dev, int32_t* iters_block_host, int32_t* iters_sample_dev, void* cuda_stream);
+
+/*
  * tf_jacobi_update -- the fused step of Algorithm 1 on its own: given the un-shifted head output
  * o_dev [B, L, 2D] = (mu~ | alpha~) of one causal pass, the block input v_dev [B,L,D] and the
  * previous iterate u_dev [B,L,D] (updated in place), set u_1 = v_1, u_l = v_l * exp(alpha~_{l-1})

@@ -23,6 +23,10 @@ class TfConfig(C.Structure):
                                          "mlp_ratio", "n_classes", "dtype", "max_batch")]
 
 
+class TfMafConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("D", "hidden", "n_blocks", "dtype", "max_batch")]
+
+
 class TfJacobiOpts(C.Structure):
     _fields_ = [("struct_bytes", C.c_int32), ("init_mode", C.c_int32), ("u0_dev", C.c_void_p),
                 ("tau_block_host", C.c_void_p), ("fallback_sweeps", C.c_int32), ("reserved", C.c_int32),
@@ -55,6 +59,10 @@ def lib():
         L.tf_inverse_jacobi_ex.argtypes = [vp, vp, vp, i32, vp, f32, i32, C.POINTER(TfJacobiOpts), vp, vp, vp, vp]
         L.tf_block_times.argtypes = [vp, vp, i32]
         L.tf_trace_read_l2.argtypes = [vp, i32, i32, vp, i32]
+        L.tf_maf_load.argtypes = [C.POINTER(TfMafConfig), vp, C.c_size_t, C.POINTER(vp)]
+        L.tf_maf_forward.argtypes = [vp, vp, i32, vp, vp, vp]
+        L.tf_maf_inverse_sequential.argtypes = [vp, vp, i32, vp, vp]
+        L.tf_maf_inverse_jacobi.argtypes = [vp, vp, i32, f32, i32, i32, vp, vp, vp, vp]
         L.tf_inverse_jacobi_host.argtypes = [vp, vp, vp, i32, vp, f32, i32, i32, vp, vp, vp, vp]
         L.tf_jacobi_update.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
         L.tf_gemm_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
@@ -168,6 +176,28 @@ def tf_inverse_jacobi_host(m, z_host, labels_host, B, policy, tau, max_iters, in
     return _check(lib().tf_inverse_jacobi_host(m, hp(z_host), hp(labels_host), B, pol.ctypes.data_as(C.c_void_p), tau,
                                                max_iters, init_mode, hp(x_host), ib, hp(iters_sample_host),
                                                _stream(stream)))
+
+
+def tf_maf_load(cfg: dict, blob: np.ndarray, max_batch: int):
+    blob = np.ascontiguousarray(blob)
+    out = C.c_void_p()
+    c = TfMafConfig(cfg["D"], cfg["hidden"], cfg["n_blocks"], cfg["dtype"], max_batch)
+    _check(lib().tf_maf_load(C.byref(c), blob.ctypes.data_as(C.c_void_p), blob.nbytes, C.byref(out)))
+    return out
+
+
+def tf_maf_forward(m, x, B, z, logdet, stream=None):
+    return _check(lib().tf_maf_forward(m, _ptr(x), B, _ptr(z), _ptr(logdet), _stream(stream)))
+
+
+def tf_maf_inverse_sequential(m, z, B, x, stream=None):
+    return _check(lib().tf_maf_inverse_sequential(m, _ptr(z), B, _ptr(x), _stream(stream)))
+
+
+def tf_maf_inverse_jacobi(m, z, B, tau, max_iters, init_mode, x, iters_block=None, iters_sample=None, stream=None):
+    ib = None if iters_block is None else iters_block.ctypes.data_as(C.c_void_p)
+    return _check(lib().tf_maf_inverse_jacobi(m, _ptr(z), B, tau, max_iters, init_mode, _ptr(x), ib, _ptr(iters_sample),
+                                              _stream(stream)))
 
 
 def tf_jacobi_update(o, v, u, maxdiff, B, L, D, reversed_, stream=None):

@@ -23,10 +23,13 @@ __device__ __forceinline__ void fence_proxy_async_smem();
 __device__ __forceinline__ uint32_t swz128(int r, int k);
 }  // namespace tc
 
+// Activation selector of the store epilogues: 0 = none, 1 = erf-GELU, 2 = ReLU (false / true select none / GELU).
+constexpr int ACT_NONE = 0, ACT_GELU = 1, ACT_RELU = 2;
+
 // out[row, col] = act(acc + bias[col]).  With `out_lo` set (bf16 only) the value is stored as an
 // error-compensated pair: out = bf16(x), out_lo = bf16(x - out), so that out + out_lo carries about
 // 16 significant bits; the next GEMM/attention consumes both terms.
-template <class OutT, bool GELU>
+template <class OutT, int ACT>
 struct EpiStore {
   OutT* out;
   const float* bias;  // may be null
@@ -41,9 +44,13 @@ struct EpiStore {
       const float4 b = *reinterpret_cast<const float4*>(sbias + j);
       v[j] += b.x; v[j + 1] += b.y; v[j + 2] += b.z; v[j + 3] += b.w;
     }
-    if (GELU) {
+    if (ACT == ACT_GELU) {
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] = gelu_erf_fast(v[j]);
+    }
+    if (ACT == ACT_RELU) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
     }
     store_bf16<32>(out + (size_t)row * ldc + col0, v, nv);
     if (out_lo != nullptr) {
@@ -59,7 +66,7 @@ struct EpiStore {
 #pragma unroll
     for (int j = 0; j < NC; ++j) {
       float x = v[j] + ((bias != nullptr && j < nv) ? bias[col0 + j] : 0.f);
-      r[j] = GELU ? gelu_erf(x) : x;
+      r[j] = ACT == ACT_GELU ? gelu_erf(x) : (ACT == ACT_RELU ? fmaxf(x, 0.f) : x);
     }
     if constexpr (sizeof(OutT) == 4) {
       if (nv == NC && (ldc % 4) == 0) {
@@ -85,7 +92,8 @@ struct EpiStore {
   }
   __device__ __forceinline__ void store(int row, int col, float acc, float cc, bool col_ok, int) const {
     float x = acc + cc;
-    if (GELU) x = (sizeof(OutT) == 2) ? gelu_erf_fast(x) : gelu_erf(x);
+    if (ACT == ACT_GELU) x = (sizeof(OutT) == 2) ? gelu_erf_fast(x) : gelu_erf(x);
+    if (ACT == ACT_RELU) x = fmaxf(x, 0.f);
     if (!col_ok) return;
     const size_t e = (size_t)row * ldc + col;
     if constexpr (sizeof(OutT) == 4) {
@@ -336,12 +344,105 @@ struct EpiHeadUpdate {
   }
 };
 
+// The fused step of Algorithm 1 for the MLP-based flow (App. E.3): one output row holds (mu_i, alpha_i), i < D, of
+// one sample (columns interleaved, already in the sample's own dimension order), so row s updates sample b = idx[s]:
+//     u[b, i] <- v[b, i] * exp(alpha_i) + mu_i,   maxdiff[b] = max_i |u_new - u_old|.
+// With only_col >= 0 only dimension only_col is updated (one step of sequential decoding, Eq. 5).
+struct EpiMafUpdate {
+  const float* v;      // [B, D]
+  float* u;            // [B, D], updated in place
+  float* maxdiff;      // [B]
+  const int* idx;      // [n_slots] slot -> sample (null = identity)
+  const float* bias;   // [2D] interleaved
+  int D, only_col;
+  static constexpr bool kRowwise = false;
+  static constexpr int kTmaCols = 0;
+  __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
+  __device__ __forceinline__ void store(int row, int col, float acc, float cc, bool col_ok, int lane) const {
+    const float mine = acc + cc;
+    const float al = __shfl_down_sync(0xffffffffu, mine, 1);
+    const int b = idx ? idx[row] : row;
+    float df = 0.f;
+    const int c = col >> 1;
+    if (col_ok && (lane & 1) == 0 && (only_col < 0 || c == only_col)) {
+      const size_t e = (size_t)b * D + c;
+      const float old = u[e];
+      const float nw = fmaf(v[e], expf(al), mine);
+      u[e] = nw;
+      df = fabsf(nw - old);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {  // NaN-propagating max over the warp, then one atomic per row segment
+      const float other = __shfl_xor_sync(0xffffffffu, df, o);
+      df = (other > df || other != other) ? other : df;
+    }
+    if (lane == 0) atomic_max_nonneg(maxdiff + b, df);
+  }
+  template <int R>
+  __device__ __forceinline__ void store_rows(int row0, int col, const float (&acc)[R], float cc, bool col_ok, int lane) const {
+    const int c = col >> 1;
+    const bool active = col_ok && (lane & 1) == 0 && (only_col < 0 || c == only_col);
+    float mine[R], al[R], old[R], vv[R];
+    int bs[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      mine[r] = acc[r] + cc;
+      al[r] = __shfl_down_sync(0xffffffffu, mine[r], 1);
+      bs[r] = idx ? idx[row0 + r] : row0 + r;
+      old[r] = 0.f;
+      vv[r] = 0.f;
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+      if (active) {
+        old[r] = u[(size_t)bs[r] * D + c];
+        vv[r] = v[(size_t)bs[r] * D + c];
+      }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      float df = 0.f;
+      if (active) {
+        const float nw = fmaf(vv[r], expf(al[r]), mine[r]);
+        u[(size_t)bs[r] * D + c] = nw;
+        df = fabsf(nw - old[r]);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float other = __shfl_xor_sync(0xffffffffu, df, o);
+        df = (other > df || other != other) ? other : df;
+      }
+      if (lane == 0) atomic_max_nonneg(maxdiff + bs[r], df);
+    }
+  }
+  template <int NC>
+  __device__ __forceinline__ void apply(int row, int col0, const float (&acc)[NC], int nv) const {
+    const int b = idx ? idx[row] : row;
+    float m = 0.f;
+#pragma unroll
+    for (int j = 0; j < NC; j += 2) {
+      if (j < nv) {
+        const int c = (col0 + j) >> 1;
+        if (only_col < 0 || c == only_col) {
+          const float mu = acc[j] + bias[col0 + j], al = acc[j + 1] + bias[col0 + j + 1];
+          const size_t e = (size_t)b * D + c;
+          const float old = u[e];
+          const float nw = fmaf(v[e], expf(al), mu);
+          u[e] = nw;
+          const float df = fabsf(nw - old);
+          m = (df > m || df != df) ? df : m;
+        }
+      }
+    }
+    atomic_max_nonneg(maxdiff + b, m);
+  }
+};
+
 // ---- bulk-store forms for the tcgen05 GEMM (kTmaCols > 0): tma_box<CPG>(first chunk, last chunk, biases of the box's
 // columns in shared memory, first column, first row, staging box, its shared address, lane).  The lane owns row
 // `row0 + lane`; it writes its 128 bytes of the box as eight 16-byte pieces in the swizzled order of the tensor map.
 
 // bf16 activations: out[row, col..col+63] = bf16(act(acc + bias)), optionally with the second (error) term.
-template <bool GELU>
+template <int ACT>
 struct EpiStoreTma {
   const float* bias;  // may be null
   const CUtensorMap* tmap;
@@ -360,9 +461,13 @@ struct EpiStoreTma {
       float2 a1 = fadd2(make_float2(v0[j + 2], v0[j + 3]), make_float2(b0.z, b0.w));
       float2 c0 = fadd2(make_float2(v1[j], v1[j + 1]), make_float2(b1.x, b1.y));
       float2 c1 = fadd2(make_float2(v1[j + 2], v1[j + 3]), make_float2(b1.z, b1.w));
-      if (GELU) {
+      if (ACT == ACT_GELU) {
         a0 = gelu_erf_fast2(a0); a1 = gelu_erf_fast2(a1);
         c0 = gelu_erf_fast2(c0); c1 = gelu_erf_fast2(c1);
+      }
+      if (ACT == ACT_RELU) {
+        a0.x = fmaxf(a0.x, 0.f); a0.y = fmaxf(a0.y, 0.f); a1.x = fmaxf(a1.x, 0.f); a1.y = fmaxf(a1.y, 0.f);
+        c0.x = fmaxf(c0.x, 0.f); c0.y = fmaxf(c0.y, 0.f); c1.x = fmaxf(c1.x, 0.f); c1.y = fmaxf(c1.y, 0.f);
       }
       v0[j] = a0.x; v0[j + 1] = a0.y; v0[j + 2] = a1.x; v0[j + 3] = a1.y;
       v1[j] = c0.x; v1[j + 1] = c0.y; v1[j + 2] = c1.x; v1[j + 3] = c1.y;

@@ -658,6 +658,42 @@ __global__ void __launch_bounds__(256) l2_distance_kernel(const float* __restric
   }
 }
 
+// MLP-based flow: input of the first layer, a[s, :] = T(u[idx[s], :]) (+ the second bf16 term when a_lo != null).
+template <class T>
+__global__ void maf_cast_rows_kernel(const float* __restrict__ u, const int* __restrict__ idx, T* __restrict__ a,
+                                     T* __restrict__ a_lo, int n_slots, int D) {
+  const size_t total = (size_t)n_slots * D;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int s = (int)(i / D), c = (int)(i - (size_t)s * D);
+    const float x = u[(size_t)(idx ? idx[s] : s) * D + c];
+    const T hi = from_f32<T>(x);
+    a[i] = hi;
+    if (a_lo != nullptr) a_lo[i] = from_f32<T>(x - to_f32(hi));
+  }
+}
+
+// MLP-based flow, forward direction (Eq. 4): v = (u - mu) exp(-alpha), logdet[b] -= sum alpha.  One CTA per sample
+// (fixed-order tree: deterministic).  o: [B, 2D] interleaved (mu_i, alpha_i).
+__global__ void __launch_bounds__(256) maf_forward_affine_kernel(const float* __restrict__ o, const float* __restrict__ u,
+                                                                 float* __restrict__ v, float* __restrict__ logdet, int D) {
+  __shared__ float red[8];
+  const int b = blockIdx.x;
+  float part = 0.f;
+  for (int i = threadIdx.x; i < D; i += 256) {
+    const float mu = o[(size_t)b * 2 * D + 2 * i], al = o[(size_t)b * 2 * D + 2 * i + 1];
+    v[(size_t)b * D + i] = (u[(size_t)b * D + i] - mu) * expf(-al);
+    part += al;
+  }
+  part = warp_sum(part);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = part;
+  __syncthreads();
+  if (threadIdx.x == 0 && logdet != nullptr) {
+    float sum = 0.f;
+    for (int i = 0; i < 8; ++i) sum += red[i];
+    logdet[b] -= sum;
+  }
+}
+
 // out[b] = labels[b] clamped to [0, n_classes); *flag is set when a label had to be clamped.
 __global__ void labels_check_kernel(const int* __restrict__ labels, int* __restrict__ out, int B, int n_classes,
                                     int* __restrict__ flag) {

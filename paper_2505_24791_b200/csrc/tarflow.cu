@@ -199,6 +199,15 @@ struct tf_model {
   float* trace_l2 = nullptr;            // [n_blocks][trace_l2_sweeps][max_batch] when the trace is on
   int trace_l2_sweeps = 0;
   std::vector<int> trace_l2_count;      // sweeps recorded per block in the last call
+  // second workload: MLP-based autoregressive flow (MADE networks, App. E.3).  Such a model reuses the token buffers
+  // (L = D values of token dimension 1), the sweep control and the GEMM machinery; the TarFlow calls refuse it.
+  bool is_maf = false;
+  struct MafBlock { Matrix w1, w2, w3; float *b1 = nullptr, *b2 = nullptr, *b3 = nullptr; };
+  std::vector<MafBlock> maf_blocks;
+  int maf_H = 0;
+  void *maf_a0 = nullptr, *maf_a0_lo = nullptr, *maf_h1 = nullptr, *maf_h1_lo = nullptr, *maf_h2 = nullptr, *maf_h2_lo = nullptr;
+  CUtensorMap maf_map[3][2];               // A-operand maps of {a0, h1, h2} x {hi, lo}
+  CUtensorMap* maf_store_maps = nullptr;   // device copy: bulk-store maps of h1, h1_lo, h2, h2_lo
   float *io_z = nullptr, *io_x = nullptr;  // staging for the host-buffer entry point
   int* io_labels = nullptr;
   cudaStream_t stream = nullptr;
@@ -909,6 +918,17 @@ struct InvOpts {
 static int layout(tf_model* m, float* img, float* seq, int B, int to_seq);
 template <class T>
 static int run_sequential_any(tf_model* m, int g, int B, const int* labels, const float* v, float* u);
+template <class T>
+static int maf_pass(tf_model* m, int g, int n_slots, const float* u_src, const int* idx, int mode, const float* v, float* u_upd,
+                    bool hp, int only_col);
+
+// one causal pass of a Jacobi sweep over the listed slots, whichever flow the model is
+template <class T>
+static int sweep_pass(tf_model* m, int g, int n_slots, const float* u_src, const int* idx, const int* labels, const float* v,
+                      float* u_upd, bool hp) {
+  if (m->is_maf) return maf_pass<T>(m, g, n_slots, u_src, idx, 0, v, u_upd, hp, -1);
+  return run_pass<T>(m, g, n_slots, u_src, idx, labels, PASS_JACOBI, v, u_upd, hp);
+}
 
 template <class T>
 static int run_jacobi_block(tf_model* m, int g, int B, const int* labels, const float* v, float* u, float tau,
@@ -932,8 +952,8 @@ static int run_jacobi_block(tf_model* m, int g, int B, const int* labels, const 
   while (t < cap && n_active > 0) {
     ++t;
     const int n_lp = n_active - n_hp;
-    if (n_lp > 0) TF_TRY(run_pass<T>(m, g, n_lp, u, m->idx, labels, PASS_JACOBI, v, u, false));
-    if (n_hp > 0) TF_TRY(run_pass<T>(m, g, n_hp, u, m->idx + n_lp, labels, PASS_JACOBI, v, u, true));
+    if (n_lp > 0) TF_TRY(sweep_pass<T>(m, g, n_lp, u, m->idx, labels, v, u, false));
+    if (n_hp > 0) TF_TRY(sweep_pass<T>(m, g, n_hp, u, m->idx + n_lp, labels, v, u, true));
     LAUNCH_PDL(m, KC_CTRL, jacobi_finalize_kernel, 1, 256, 0, m->maxdiff, m->idx, m->idx_tmp, m->phase, m->ctrl, iters_row,
            tau, sw, t);
     if (l2 && t <= m->trace_l2_sweeps) {
@@ -1065,6 +1085,107 @@ static int forward_impl(tf_model* m, const float* x, const int* labels, int B, f
     float* tmp = v; v = u; u = tmp;
   }
   TF_TRY(layout(m, z, u, B, 0));
+  return sync_check(m);
+}
+
+// ------------------------------------------------------------------------------------------------
+// second workload: MLP-based autoregressive flow (App. E.3).  One pass = cast -> three masked linear layers.
+//   mode 0: Jacobi update in the last layer's epilogue (only_col >= 0: one step of sequential decoding)
+//   mode 1: forward direction, the raw (mu, alpha) go to m->o
+// The layer permutation (reversal on odd layers) and the MADE masks are folded into the weights when they are
+// loaded, so every buffer here is in the sample's own dimension order.
+// ------------------------------------------------------------------------------------------------
+template <class T>
+static int maf_pass(tf_model* m, int g, int n_slots, const float* u_src, const int* idx, int mode, const float* v, float* u_upd,
+                    bool hp, int only_col) {
+  const tf_model::MafBlock& bw = m->maf_blocks[g];
+  const int D = m->L, H = m->maf_H, M = n_slots;
+  T* a0 = reinterpret_cast<T*>(m->maf_a0);
+  T* h1 = reinterpret_cast<T*>(m->maf_h1);
+  T* h2 = reinterpret_cast<T*>(m->maf_h2);
+  T* a0_lo = hp ? reinterpret_cast<T*>(m->maf_a0_lo) : nullptr;
+  T* h1_lo = hp ? reinterpret_cast<T*>(m->maf_h1_lo) : nullptr;
+  T* h2_lo = hp ? reinterpret_cast<T*>(m->maf_h2_lo) : nullptr;
+  m->cur_rows = M;
+  int cb = (int)(((size_t)M * D + 255) / 256);
+  if (cb > 148 * 16) cb = 148 * 16;
+  LAUNCH(m, KC_EMBED, (maf_cast_rows_kernel<T>), cb, 256, 0, u_src, idx, a0, a0_lo, M, D);
+  TF_TRY(check_launch("maf_cast_rows_kernel"));
+  if constexpr (sizeof(T) == 2) {
+    const CUtensorMap* sm = m->maf_store_maps;
+    TF_TRY(gemm<T>(m, KC_GEMM_MLP1, a0, &m->maf_map[0][0], hp ? &m->maf_map[0][1] : nullptr, bw.w1, M,
+                   EpiStoreTma<ACT_RELU>{bw.b1, sm + 0, hp ? sm + 1 : nullptr}));
+    TF_TRY(gemm<T>(m, KC_GEMM_MLP2, h1, &m->maf_map[1][0], hp ? &m->maf_map[1][1] : nullptr, bw.w2, M,
+                   EpiStoreTma<ACT_RELU>{bw.b2, sm + 2, hp ? sm + 3 : nullptr}));
+  } else {
+    TF_TRY(gemm<T>(m, KC_GEMM_MLP1, a0, nullptr, nullptr, bw.w1, M, EpiStore<T, ACT_RELU>{h1, bw.b1, H, h1_lo}));
+    TF_TRY(gemm<T>(m, KC_GEMM_MLP2, h1, nullptr, nullptr, bw.w2, M, EpiStore<T, ACT_RELU>{h2, bw.b2, H, h2_lo}));
+  }
+  const CUtensorMap* map2 = sizeof(T) == 2 ? &m->maf_map[2][0] : nullptr;
+  const CUtensorMap* map2_lo = (sizeof(T) == 2 && hp) ? &m->maf_map[2][1] : nullptr;
+  if (mode == 0) {
+    EpiMafUpdate epi{v, u_upd, m->maxdiff, idx, bw.b3, D, only_col};
+    return gemm<T>(m, KC_GEMM_HEAD_UPDATE, h2, map2, map2_lo, bw.w3, M, epi);
+  }
+  return gemm<T>(m, KC_GEMM_HEAD, h2, map2, map2_lo, bw.w3, M, EpiStore<float, ACT_NONE>{m->o, bw.b3, 2 * D});
+}
+
+template <class T>
+static int maf_inverse_impl(tf_model* m, const float* z, int B, bool jacobi, float tau, int max_iters, int init_mode, float* x,
+                            int* iters_block_host, int* iters_sample_dev) {
+  const int K = m->cfg.n_blocks, D = m->L;
+  const size_t n = (size_t)B * D;
+  float *v = m->seq_a, *u = m->seq_b;
+  m->trace.clear();
+  m->trace_l2_count.assign(K, 0);
+  CU_OK(cudaMemcpyAsync(v, z, n * sizeof(float), cudaMemcpyDeviceToDevice, m->stream));
+  int status = TF_OK;
+  InvOpts op;
+  op.init_mode = init_mode;
+  for (int g = 0; g < K; ++g) {
+    int* iters_row = m->iters_sample + (size_t)g * m->cfg.max_batch;
+    int sweeps = D;
+    if (m->block_ev[g]) cudaEventRecord(m->block_ev[g], m->stream);
+    if (!jacobi) {
+      // Eq. 5: dimension i (in the layer's own order) is final after pass i; there is no cache, every pass is a whole one
+      CU_OK(cudaMemsetAsync(u, 0, n * sizeof(float), m->stream));
+      for (int i = 0; i < D; ++i)
+        TF_TRY(maf_pass<T>(m, g, B, u, nullptr, 0, v, u, m->precision_mode == 2, (g & 1) ? D - 1 - i : i));
+      LAUNCH(m, KC_CTRL, fill_int_kernel, (B + 127) / 128, 128, 0, iters_row, B, D);
+      CU_OK(cudaMemsetAsync(m->maxdiff, 0, B * sizeof(float), m->stream));
+    } else {
+      int r = run_jacobi_block<T>(m, g, B, nullptr, v, u, tau, max_iters, op, &sweeps, iters_row);
+      if (r < 0) return r;
+      if (r == TF_MAXITER) status = TF_MAXITER;
+    }
+    if (iters_block_host) iters_block_host[g] = sweeps;
+    float* tmp = v; v = u; u = tmp;
+  }
+  if (m->block_ev[K]) cudaEventRecord(m->block_ev[K], m->stream);
+  m->block_ev_valid = true;
+  CU_OK(cudaMemcpyAsync(x, v, n * sizeof(float), cudaMemcpyDeviceToDevice, m->stream));
+  if (iters_sample_dev)
+    for (int g = 0; g < K; ++g)
+      CU_OK(cudaMemcpyAsync(iters_sample_dev + (size_t)g * B, m->iters_sample + (size_t)g * m->cfg.max_batch, B * sizeof(int),
+                            cudaMemcpyDeviceToDevice, m->stream));
+  TF_TRY(sync_check(m));
+  return status;
+}
+
+template <class T>
+static int maf_forward_impl(tf_model* m, const float* x, int B, float* z, float* logdet) {
+  const int D = m->L;
+  const size_t n = (size_t)B * D;
+  float *u = m->seq_a, *v = m->seq_b;
+  CU_OK(cudaMemcpyAsync(u, x, n * sizeof(float), cudaMemcpyDeviceToDevice, m->stream));
+  if (logdet) CU_OK(cudaMemsetAsync(logdet, 0, B * sizeof(float), m->stream));
+  for (int g = m->cfg.n_blocks - 1; g >= 0; --g) {
+    TF_TRY(maf_pass<T>(m, g, B, u, nullptr, 1, nullptr, nullptr, false, -1));
+    LAUNCH(m, KC_AFFINE, maf_forward_affine_kernel, B, 256, 0, m->o, u, v, logdet, D);
+    TF_TRY(check_launch("maf_forward_affine_kernel"));
+    float* tmp = v; v = u; u = tmp;
+  }
+  CU_OK(cudaMemcpyAsync(z, u, n * sizeof(float), cudaMemcpyDeviceToDevice, m->stream));
   return sync_check(m);
 }
 
@@ -1298,8 +1419,114 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
   return TF_OK;
 }
 
-static int check_call(tf_model* m, int B) {
+// ---- loading an MLP-based flow: masks and the layer permutation are applied to the weights here ----------------
+// Degrees (MADE): input i has degree i + 1, hidden unit j of either hidden layer 1 + (j mod (D - 1)), output i degree
+// i + 1.  A hidden unit keeps the weights from inputs / hidden units of degree <= its own, an output those from
+// hidden units of degree < its own.  Odd layers act on the reversed dimension order: their first matrix gets its
+// columns reversed and their output matrix / bias their rows, so the kernels work in the sample's own order.
+static int maf_load_impl(tf_model* m, const void* blob, size_t nbytes, int D, int H) {
+  const tf_config& c = m->cfg;
+  const size_t per_block = (size_t)H * D + H + (size_t)H * H + H + (size_t)2 * D * H + 2 * D;
+  const size_t want = 64 + 4 * per_block * c.n_blocks;
+  if (nbytes != want) return fail(TF_ESIZE, "weight blob is %zu bytes, configuration needs %zu", nbytes, want);
+  const int32_t* hdr = reinterpret_cast<const int32_t*>(blob);
+  const int32_t expect[6] = {0x3146414D, 1, D, H, c.n_blocks, c.dtype};
+  for (int i = 0; i < 6; ++i)
+    if (hdr[i] != expect[i]) return fail(TF_ESIZE, "weight blob header field %d is %d, expected %d", i, hdr[i], expect[i]);
+  int dev = 0;
+  CU_OK(cudaGetDevice(&dev));
+  CU_OK(cudaDeviceGetAttribute(&m->num_sms, cudaDevAttrMultiProcessorCount, dev));
+  float* staging = nullptr;
+  size_t max_mat = (size_t)H * H;
+  if ((size_t)2 * D * H > max_mat) max_mat = (size_t)2 * D * H;
+  if (c.dtype == 1) CU_OK(cudaMalloc(&staging, max_mat * sizeof(float)));
+  struct Guard { float* p; ~Guard() { if (p) cudaFree(p); } } guard{staging};
+
+  auto deg_hidden = [&](int j) { return 1 + j % (D > 1 ? D - 1 : 1); };
+  BlobReader rd{reinterpret_cast<const float*>(reinterpret_cast<const char*>(blob) + 64), nullptr};
+  m->maf_blocks.resize(c.n_blocks);
+  std::vector<float> tmp, btmp(2 * D);
+  for (int g = 0; g < c.n_blocks; ++g) {
+    tf_model::MafBlock& bw = m->maf_blocks[g];
+    const bool rev = (g & 1) != 0;
+    const float* w1 = rd.take((size_t)H * D);
+    tmp.assign((size_t)H * D, 0.f);
+    for (int j = 0; j < H; ++j)
+      for (int i = 0; i < D; ++i)
+        if (deg_hidden(j) >= i + 1) tmp[(size_t)j * D + (rev ? D - 1 - i : i)] = w1[(size_t)j * D + i];
+    TF_TRY(upload_matrix(m, &bw.w1, tmp.data(), H, D, staging));
+    TF_TRY(upload_f32(m, &bw.b1, rd.take(H), H));
+    const float* w2 = rd.take((size_t)H * H);
+    tmp.assign((size_t)H * H, 0.f);
+    for (int j = 0; j < H; ++j)
+      for (int i = 0; i < H; ++i)
+        if (deg_hidden(j) >= deg_hidden(i)) tmp[(size_t)j * H + i] = w2[(size_t)j * H + i];
+    TF_TRY(upload_matrix(m, &bw.w2, tmp.data(), H, H, staging));
+    TF_TRY(upload_f32(m, &bw.b2, rd.take(H), H));
+    // output layer [mu | alpha] -> interleaved rows (2 i, 2 i + 1) = (mu_i, alpha_i) in the sample's own order
+    const float* w3 = rd.take((size_t)2 * D * H);
+    const float* b3 = rd.take((size_t)2 * D);
+    tmp.assign((size_t)2 * D * H, 0.f);
+    for (int i = 0; i < D; ++i) {
+      const int r = rev ? D - 1 - i : i;  // position of the layer's dimension i in the sample's order
+      for (int j = 0; j < H; ++j)
+        if (i + 1 > deg_hidden(j)) {
+          tmp[(size_t)(2 * r) * H + j] = w3[(size_t)i * H + j];
+          tmp[(size_t)(2 * r + 1) * H + j] = w3[(size_t)(D + i) * H + j];
+        }
+      btmp[2 * r] = b3[i];
+      btmp[2 * r + 1] = b3[D + i];
+    }
+    TF_TRY(upload_matrix(m, &bw.w3, tmp.data(), 2 * D, H, staging));
+    TF_TRY(upload_f32(m, &bw.b3, btmp.data(), btmp.size()));
+  }
+
+  const size_t B = c.max_batch, esz = c.dtype == 1 ? 2 : 4;
+  TF_TRY(dev_alloc(m, &m->seq_a, B * D));
+  TF_TRY(dev_alloc(m, &m->seq_b, B * D));
+  TF_TRY(dev_alloc(m, &m->o, B * 2 * D));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->maf_a0), B * D * esz));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->maf_a0_lo), B * D * esz));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->maf_h1), B * H * esz));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->maf_h1_lo), B * H * esz));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->maf_h2), B * H * esz));
+  TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->maf_h2_lo), B * H * esz));
+  TF_TRY(dev_alloc(m, &m->maxdiff, B));
+  TF_TRY(dev_alloc(m, &m->idx, B));
+  TF_TRY(dev_alloc(m, &m->idx_tmp, B));
+  TF_TRY(dev_alloc(m, &m->phase, B));
+  TF_TRY(dev_alloc(m, &m->ctrl, 8));
+  TF_TRY(dev_alloc(m, &m->err, 1));
+  TF_TRY(dev_alloc(m, &m->iters_sample, (size_t)c.n_blocks * B));
+  CU_OK(cudaMemset(m->ctrl, 0, 8 * sizeof(int)));
+  CU_OK(cudaMemset(m->err, 0, sizeof(int)));
+  CU_OK(cudaMemset(m->maxdiff, 0, B * sizeof(float)));
+  CU_OK(cudaMemset(m->iters_sample, 0, (size_t)c.n_blocks * B * sizeof(int)));
+  CU_OK(cudaMallocHost(&m->ctrl_host, 8 * sizeof(int)));
+  m->block_ev.assign(c.n_blocks + 1, nullptr);
+  for (auto& e : m->block_ev) CU_OK(cudaEventCreate(&e));
+  if (c.dtype == 1) {
+    void* bufs[3][2] = {{m->maf_a0, m->maf_a0_lo}, {m->maf_h1, m->maf_h1_lo}, {m->maf_h2, m->maf_h2_lo}};
+    const int cols[3] = {D, H, H};
+    for (int i = 0; i < 3; ++i)
+      for (int t = 0; t < 2; ++t) TF_TRY(make_map_bf16(&m->maf_map[i][t], bufs[i][t], B, cols[i], tc::BM));
+    CUtensorMap sm[4];
+    TF_TRY(make_map_store(&sm[0], m->maf_h1, B, H, 2));
+    TF_TRY(make_map_store(&sm[1], m->maf_h1_lo, B, H, 2));
+    TF_TRY(make_map_store(&sm[2], m->maf_h2, B, H, 2));
+    TF_TRY(make_map_store(&sm[3], m->maf_h2_lo, B, H, 2));
+    TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->maf_store_maps), sizeof(sm)));
+    CU_OK(cudaMemcpy(m->maf_store_maps, sm, sizeof(sm), cudaMemcpyHostToDevice));
+    if (const char* e = getenv("TARFLOW_PAIR_GEMM")) m->use_pair_gemm = atoi(e) != 0;
+  }
+  CU_OK(cudaDeviceSynchronize());
+  return TF_OK;
+}
+
+static int check_call(tf_model* m, int B, bool want_maf = false) {
   if (!m) return fail(TF_EINVAL, "model is NULL");
+  if (m->is_maf != want_maf)
+    return fail(TF_EINVAL, want_maf ? "this call needs a model loaded with tf_maf_load" : "this call needs a model loaded with tf_load");
   if (B < 1 || B > m->cfg.max_batch) return fail(TF_EINVAL, "B=%d outside [1, max_batch=%d]", B, m->cfg.max_batch);
   return TF_OK;
 }
@@ -1464,6 +1691,62 @@ int tf_inverse_jacobi_host(tf_model* m, const float* z_host, const int32_t* labe
                             B * sizeof(int), cudaMemcpyDeviceToHost, st));
   CU_OK(cudaStreamSynchronize(st));
   return r;
+}
+
+int tf_maf_load(const tf_maf_config* cfg, const void* weights_host, size_t nbytes, tf_model** out) {
+  g_err[0] = 0;
+  if (!cfg || !weights_host || !out) return fail(TF_EINVAL, "NULL argument");
+  *out = nullptr;
+  if (cfg->D < 2 || cfg->hidden < 1 || cfg->n_blocks < 1 || cfg->max_batch < 1) return fail(TF_EINVAL, "bad model dimensions");
+  if (cfg->dtype != 0 && cfg->dtype != 1) return fail(TF_EINVAL, "dtype must be 0 (fp32) or 1 (bf16)");
+  if (cfg->dtype == 1 && (cfg->D % 8 || cfg->hidden % 64))
+    return fail(TF_EINVAL, "bf16 engine needs D %% 8 == 0 and hidden %% 64 == 0");
+  tf_model* m = new (std::nothrow) tf_model();
+  if (!m) return fail(TF_ENOMEM, "host allocation failed");
+  m->is_maf = true;
+  m->cfg = tf_config{1, cfg->D, 1, 1, cfg->n_blocks, 2, cfg->hidden, 1, 1, 0, cfg->dtype, cfg->max_batch};
+  m->L = cfg->D;  // D values per sample, token dimension 1
+  m->D = 1;
+  m->d = m->hid = m->maf_H = cfg->hidden;
+  m->hd = cfg->hidden;
+  int r = maf_load_impl(m, weights_host, nbytes, cfg->D, cfg->hidden);
+  if (r != TF_OK) {
+    tf_free(m);
+    return r;
+  }
+  *out = m;
+  return TF_OK;
+}
+
+int tf_maf_forward(tf_model* m, const float* x_dev, int32_t B, float* z_dev, float* logdet_dev, void* cuda_stream) {
+  g_err[0] = 0;
+  TF_TRY(check_call(m, B, true));
+  if (!x_dev || !z_dev) return fail(TF_EINVAL, "NULL buffer");
+  m->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  return m->cfg.dtype == 1 ? maf_forward_impl<bf16>(m, x_dev, B, z_dev, logdet_dev) : maf_forward_impl<float>(m, x_dev, B, z_dev, logdet_dev);
+}
+
+int tf_maf_inverse_sequential(tf_model* m, const float* z_dev, int32_t B, float* x_dev, void* cuda_stream) {
+  g_err[0] = 0;
+  TF_TRY(check_call(m, B, true));
+  if (!z_dev || !x_dev) return fail(TF_EINVAL, "NULL buffer");
+  m->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  return m->cfg.dtype == 1 ? maf_inverse_impl<bf16>(m, z_dev, B, false, 0.f, 1, 0, x_dev, nullptr, nullptr)
+                           : maf_inverse_impl<float>(m, z_dev, B, false, 0.f, 1, 0, x_dev, nullptr, nullptr);
+}
+
+int tf_maf_inverse_jacobi(tf_model* m, const float* z_dev, int32_t B, float tau, int32_t max_iters, int32_t init_mode,
+                          float* x_dev, int32_t* iters_block_host, int32_t* iters_sample_dev, void* cuda_stream) {
+  g_err[0] = 0;
+  TF_TRY(check_call(m, B, true));
+  if (!z_dev || !x_dev) return fail(TF_EINVAL, "NULL buffer");
+  if (max_iters < 1) return fail(TF_EINVAL, "max_iters must be >= 1");
+  if (init_mode != 0 && init_mode != 1) return fail(TF_EINVAL, "init_mode must be 0 or 1");
+  if (tau != tau) return fail(TF_EINVAL, "tau is NaN");
+  m->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  return m->cfg.dtype == 1
+             ? maf_inverse_impl<bf16>(m, z_dev, B, true, tau, max_iters, init_mode, x_dev, iters_block_host, iters_sample_dev)
+             : maf_inverse_impl<float>(m, z_dev, B, true, tau, max_iters, init_mode, x_dev, iters_block_host, iters_sample_dev);
 }
 
 int tf_jacobi_update(const float* o_dev, const float* v_dev, float* u_dev, float* maxdiff_dev, int32_t B, int32_t L,
