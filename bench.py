@@ -596,7 +596,7 @@ def run_maf_leg(name, binding, synth, torch, timed, pk, steps=3):
                       "sweeps_max": [int(v) for v in itn.max(axis=1)], "sweeps_mean": [round(float(v), 2) for v in itn.mean(axis=1)],
                       "ms_per_block": [round(float(v), 3) for v in binding.tf_block_times(model, K)],
                       "tensor_frac": round(rows * flops_row / (ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"], 4)}}
-    Bs = min(B, 4096)                                                  # sequential decoding: a bounded sub-batch
+    Bs = min(B, 16384)                                                 # sequential decoding: a bounded sub-batch
     binding.tf_maf_inverse_sequential(model, zs[0][:Bs].contiguous(), Bs, x[:Bs], stream)
     zsub = [z[:Bs].contiguous() for z in zs]
     ms_s, _, _ = timed(lambda i: binding.tf_maf_inverse_sequential(model, zsub[i], Bs, x[:Bs], stream), [1])

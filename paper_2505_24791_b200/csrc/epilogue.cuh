@@ -36,6 +36,8 @@ struct EpiStore {
   int ldc;
   OutT* out_lo = nullptr;
   static constexpr bool kRowwise = sizeof(OutT) == 2;
+  static constexpr bool kRowReduce = false;
+  static constexpr int kRowsBatch = 8;
   static constexpr int kTmaCols = 0;
   // sbias: the 32 biases of columns col0.. (zeros without a bias), warp-private shared memory
   __device__ __forceinline__ void rowwise(int row, int col0, float (&v)[32], int nv, const float* sbias) const {
@@ -141,6 +143,8 @@ struct EpiResid {  // h[row, col] += acc + bias[col]   (fp32 residual stream, in
   const float* bias;
   int ldc;
   static constexpr bool kRowwise = false;
+  static constexpr bool kRowReduce = false;
+  static constexpr int kRowsBatch = 8;
   static constexpr int kTmaCols = 0;
   __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
   __device__ __forceinline__ void store(int row, int col, float acc, float cc, bool col_ok, int) const {
@@ -218,6 +222,8 @@ struct EpiHeadUpdate {
   const float* bias;   // [2D] interleaved
   int L, D, reversed;
   static constexpr bool kRowwise = false;
+  static constexpr bool kRowReduce = false;
+  static constexpr int kRowsBatch = 8;
   static constexpr int kTmaCols = 0;
   __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
   // lane-per-column form: even lanes hold mu~_c, the next lane alpha~_c
@@ -356,62 +362,51 @@ struct EpiMafUpdate {
   const float* bias;   // [2D] interleaved
   int D, only_col;
   static constexpr bool kRowwise = false;
+  static constexpr bool kRowReduce = false;
   static constexpr int kTmaCols = 0;
+  // lane = column: a warp's accesses to u and v are contiguous row segments.  All 32 rows of a chunk are handled in
+  // one batch, so the warp pays one memory round trip per chunk for the old iterate and the layer input.
+  static constexpr int kRowsBatch = 32;
   __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
   __device__ __forceinline__ void store(int row, int col, float acc, float cc, bool col_ok, int lane) const {
-    const float mine = acc + cc;
-    const float al = __shfl_down_sync(0xffffffffu, mine, 1);
-    const int b = idx ? idx[row] : row;
-    float df = 0.f;
-    const int c = col >> 1;
-    if (col_ok && (lane & 1) == 0 && (only_col < 0 || c == only_col)) {
-      const size_t e = (size_t)b * D + c;
-      const float old = u[e];
-      const float nw = fmaf(v[e], expf(al), mine);
-      u[e] = nw;
-      df = fabsf(nw - old);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {  // NaN-propagating max over the warp, then one atomic per row segment
-      const float other = __shfl_xor_sync(0xffffffffu, df, o);
-      df = (other > df || other != other) ? other : df;
-    }
-    if (lane == 0) atomic_max_nonneg(maxdiff + b, df);
+    const float a1[1] = {acc};
+    store_rows<1>(row, col, a1, cc, col_ok, lane);
   }
   template <int R>
   __device__ __forceinline__ void store_rows(int row0, int col, const float (&acc)[R], float cc, bool col_ok, int lane) const {
     const int c = col >> 1;
+    if (only_col >= 0 && __all_sync(0xffffffffu, c != only_col)) return;  // this chunk does not hold the one dimension
     const bool active = col_ok && (lane & 1) == 0 && (only_col < 0 || c == only_col);
-    float mine[R], al[R], old[R], vv[R];
+    float al[R], old[R], vv[R];
     int bs[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      mine[r] = acc[r] + cc;
-      al[r] = __shfl_down_sync(0xffffffffu, mine[r], 1);
+      al[r] = __shfl_down_sync(0xffffffffu, acc[r] + cc, 1);
       bs[r] = idx ? idx[row0 + r] : row0 + r;
-      old[r] = 0.f;
-      vv[r] = 0.f;
     }
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+    for (int r = 0; r < R; ++r) {
+      old[r] = 0.f;
+      vv[r] = 0.f;
       if (active) {
         old[r] = u[(size_t)bs[r] * D + c];
         vv[r] = v[(size_t)bs[r] * D + c];
       }
+    }
 #pragma unroll
     for (int r = 0; r < R; ++r) {
       float df = 0.f;
       if (active) {
-        const float nw = fmaf(vv[r], expf(al[r]), mine[r]);
+        const float nw = fmaf(vv[r], expf(al[r]), acc[r] + cc);
         u[(size_t)bs[r] * D + c] = nw;
         df = fabsf(nw - old[r]);
       }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
+      for (int o = 16; o > 0; o >>= 1) {  // NaN-propagating max over the row segment
         const float other = __shfl_xor_sync(0xffffffffu, df, o);
         df = (other > df || other != other) ? other : df;
       }
-      if (lane == 0) atomic_max_nonneg(maxdiff + bs[r], df);
+      if (lane == 0 && df != 0.f) atomic_max_nonneg(maxdiff + bs[r], df);  // maxdiff starts at 0: a zero adds nothing
     }
   }
   template <int NC>
@@ -433,7 +428,7 @@ struct EpiMafUpdate {
         }
       }
     }
-    atomic_max_nonneg(maxdiff + b, m);
+    if (m != 0.f) atomic_max_nonneg(maxdiff + b, m);
   }
 };
 
@@ -448,6 +443,7 @@ struct EpiStoreTma {
   const CUtensorMap* tmap;
   const CUtensorMap* tmap_lo;  // null = single term
   static constexpr bool kRowwise = false;
+  static constexpr bool kRowReduce = false;
   static constexpr int kTmaCols = 64;
   __device__ __forceinline__ float col_const(int col, bool col_ok) const { return (bias != nullptr && col_ok) ? bias[col] : 0.f; }
   template <int CPG>
@@ -512,6 +508,7 @@ struct EpiResidTma {
   const float* bias;
   const CUtensorMap* tmap;  // fp32 [rows, d], box 32 columns x 32 rows, 128-byte swizzle
   static constexpr bool kRowwise = false;
+  static constexpr bool kRowReduce = false;
   static constexpr int kTmaCols = 32;
   __device__ __forceinline__ float col_const(int col, bool col_ok) const { return col_ok ? bias[col] : 0.f; }
   template <int CPG>
@@ -531,5 +528,33 @@ struct EpiResidTma {
     tc::fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) { tc::tma_reduce_add_2d(tmap, col0, row0, box_addr); tc::tma_store_commit(); }
+  }
+};
+
+// fp32 output through the TMA engine: out[row, col..col+31] = acc + bias (box 32 columns x 32 rows, 128-byte swizzle).
+struct EpiStoreF32Tma {
+  const float* bias;
+  const CUtensorMap* tmap;
+  static constexpr bool kRowwise = false;
+  static constexpr bool kRowReduce = false;
+  static constexpr int kTmaCols = 32;
+  __device__ __forceinline__ float col_const(int col, bool col_ok) const { return (bias != nullptr && col_ok) ? bias[col] : 0.f; }
+  template <int CPG>
+  __device__ __forceinline__ void tma_box(float (&v)[32], float (&)[32], const float* sbias, int col0, int row0, uint8_t* box,
+                                          uint32_t box_addr, int lane) const {
+    static_assert(CPG == 1, "an fp32 box is one 32-column chunk");
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float4 b = *reinterpret_cast<const float4*>(sbias + 4 * k);
+      v[4 * k] += b.x; v[4 * k + 1] += b.y; v[4 * k + 2] += b.z; v[4 * k + 3] += b.w;
+    }
+    if (lane == 0) tc::tma_store_wait_read();  // the engine has read the warp's previous box
+    __syncwarp();
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      *reinterpret_cast<float4*>(box + tc::swz128(lane, k)) = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+    tc::fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) { tc::tma_store_2d(tmap, col0, row0, box_addr); tc::tma_store_commit(); }
   }
 };

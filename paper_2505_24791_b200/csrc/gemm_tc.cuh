@@ -366,6 +366,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       tcgen05_fence_after();
       const int row0 = m0 + quad * 32;
       const int nrows = (M - row0) < 32 ? (M - row0) : 32;  // rows of this warp inside the matrix (may be <= 0)
+      float row_acc = 0.f;  // kRowReduce functors: a per-row value carried over the warp's chunks of this tile
 #pragma unroll 1
       for (int c = cgroup; c < BN / 32; c += NUM_EPI_WARPS / 4) {
         const int col0 = n0 + c * 32;
@@ -380,7 +381,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           stage_out[lane] = cc;
           __syncwarp();
           const int nv = (N - col0) < 32 ? (N - col0) : 32;
-          if (lane < nrows) epi.rowwise(row0 + lane, col0, v, nv, stage_out);
+          if constexpr (Epi::kRowReduce) {
+            if (lane < nrows) row_acc = epi.rowwise_reduce(row0 + lane, col0, v, nv, stage_out, row_acc);
+          } else {
+            if (lane < nrows) epi.rowwise(row0 + lane, col0, v, nv, stage_out);
+          }
           __syncwarp();
         } else {
           // transpose through shared memory: lane = row on the way in, lane = column on the way out
@@ -388,18 +393,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           for (int j = 0; j < 32; ++j) stage_out[lane * 33 + j] = v[j];
           __syncwarp();
           if (nrows == 32) {
+            constexpr int RB = Epi::kRowsBatch;  // rows a functor handles per call (its loads are issued together)
 #pragma unroll
-            for (int r0 = 0; r0 < 32; r0 += 8) {
-              float a[8];
+            for (int r0 = 0; r0 < 32; r0 += RB) {
+              float a[RB];
 #pragma unroll
-              for (int r = 0; r < 8; ++r) a[r] = stage_out[(r0 + r) * 33 + lane];
-              epi.template store_rows<8>(row0 + r0, col, a, cc, col_ok, lane);
+              for (int r = 0; r < RB; ++r) a[r] = stage_out[(r0 + r) * 33 + lane];
+              epi.template store_rows<RB>(row0 + r0, col, a, cc, col_ok, lane);
             }
           } else {
             for (int r = 0; r < nrows; ++r) epi.store(row0 + r, col, stage_out[r * 33 + lane], cc, col_ok, lane);
           }
           __syncwarp();
         }
+      }
+      if constexpr (Epi::kRowReduce) {
+        if (lane < nrows) epi.row_done(row0 + lane, row_acc);
       }
       tcgen05_fence_before();
       __syncwarp();

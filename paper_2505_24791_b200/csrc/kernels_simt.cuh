@@ -607,14 +607,134 @@ jacobi_finalize_kernel(float* __restrict__ maxdiff, int* __restrict__ idx, int* 
   }
 }
 
+// The same sweep control for large batches (thousands of samples, the MLP-based flow): three launches instead of one
+// CTA walking the list.  Stable order, identical results.
+//   count:   CTA j looks at slots [1024 j, 1024 j + 1024): per-slot decision into code[] (0 = leaves, 1 = stays with
+//            single-term operands, 2 = stays with two-term operands), per-CTA survivor counts, maximum and flags;
+//   scan:    one CTA turns the counts into exclusive offsets and writes ctrl[];
+//   scatter: CTA j writes its survivors to idx_out at offset + rank (single-term samples first, then two-term).
+constexpr int FIN_CHUNK = 1024;
+
+__global__ void __launch_bounds__(FIN_CHUNK)
+jacobi_finalize_count_kernel(float* __restrict__ maxdiff, const int* __restrict__ idx, int* __restrict__ phase,
+                             const int* __restrict__ ctrl, int* __restrict__ iters_sample, unsigned char* __restrict__ code,
+                             int* __restrict__ blk_cnt /*[2][nblk]*/, float* __restrict__ blk_top, int* __restrict__ blk_flag,
+                             int nblk, float tau, float switch_thresh, int t) {
+  const int n = ctrl[0];
+  const int s = blockIdx.x * FIN_CHUNK + threadIdx.x;
+  bool f0 = false, f1 = false;
+  float top = 0.f;
+  int bad = 0, nan = 0;
+  if (s < n) {
+    const int b = idx[s];
+    const float m = maxdiff[b];
+    maxdiff[b] = 0.f;
+    if (m != m) nan = 1; else top = m;
+    if (iters_sample) iters_sample[b] = t;
+    if (!(m <= 3.0e38f)) bad = 1;
+    if (tau < 0.f || !(m <= tau)) {
+      int ph = phase[b];
+      if (m <= switch_thresh) { phase[b] = 1; ph = 1; }
+      f0 = ph == 0;
+      f1 = !f0;
+    }
+    code[s] = f0 ? 1 : (f1 ? 2 : 0);
+  }
+  const int c0 = __syncthreads_count(f0), c1 = __syncthreads_count(f1);
+  const int anybad = __syncthreads_or(bad), anynan = __syncthreads_or(nan);
+  __shared__ float s_top[32];
+  top = warp_max(top);
+  if ((threadIdx.x & 31) == 0) s_top[threadIdx.x >> 5] = top;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tt = 0.f;
+    for (int w = 0; w < FIN_CHUNK / 32; ++w) tt = fmaxf(tt, s_top[w]);
+    blk_cnt[blockIdx.x] = c0;
+    blk_cnt[nblk + blockIdx.x] = c1;
+    blk_top[blockIdx.x] = tt;
+    blk_flag[blockIdx.x] = (anybad ? 1 : 0) | (anynan ? 2 : 0);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+jacobi_finalize_scan_kernel(int* __restrict__ blk_cnt, const float* __restrict__ blk_top, const int* __restrict__ blk_flag,
+                            int* __restrict__ ctrl, int nblk) {
+  __shared__ int s_w[2][8];
+  __shared__ float s_top[8];
+  __shared__ int s_flag[8];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int base0 = 0, base1 = 0, flags = 0;
+  float top = 0.f;
+  for (int c0 = 0; c0 < nblk; c0 += 256) {
+    const int j = c0 + threadIdx.x;
+    const int a = j < nblk ? blk_cnt[j] : 0, b = j < nblk ? blk_cnt[nblk + j] : 0;
+    if (j < nblk) { top = fmaxf(top, blk_top[j]); flags |= blk_flag[j]; }
+    int xa = a, xb = b;  // inclusive scan inside the warp
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int ya = __shfl_up_sync(0xffffffffu, xa, o), yb = __shfl_up_sync(0xffffffffu, xb, o);
+      if (lane >= o) { xa += ya; xb += yb; }
+    }
+    if (lane == 31) { s_w[0][warp] = xa; s_w[1][warp] = xb; }
+    __syncthreads();
+    int wa = 0, wb = 0, ta = 0, tb = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      if (w < warp) { wa += s_w[0][w]; wb += s_w[1][w]; }
+      ta += s_w[0][w];
+      tb += s_w[1][w];
+    }
+    if (j < nblk) {
+      blk_cnt[j] = base0 + wa + xa - a;         // exclusive offsets
+      blk_cnt[nblk + j] = base1 + wb + xb - b;
+    }
+    base0 += ta;
+    base1 += tb;
+    __syncthreads();
+  }
+  top = warp_max(top);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) flags |= __shfl_xor_sync(0xffffffffu, flags, o);
+  if (lane == 0) { s_top[warp] = top; s_flag[warp] = flags; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 0; w < 8; ++w) { top = fmaxf(top, s_top[w]); flags |= s_flag[w]; }
+    ctrl[6] = ctrl[0];                 // slots of the sweep just finished (the scatter kernel's bound)
+    ctrl[0] = base0 + base1;
+    ctrl[1] = ctrl[1] | (flags & 1);
+    ctrl[2] = (flags & 2) ? 0x7fc00000 : __float_as_int(top);
+    ctrl[3] = base1;
+    ctrl[7] = base0;                   // two-term survivors start here
+  }
+}
+
+__global__ void __launch_bounds__(FIN_CHUNK)
+jacobi_finalize_scatter_kernel(const int* __restrict__ idx, int* __restrict__ idx_out, const unsigned char* __restrict__ code,
+                               const int* __restrict__ blk_off, const int* __restrict__ ctrl, int nblk) {
+  __shared__ int s_w[2][FIN_CHUNK / 32];
+  const int n = ctrl[6], base1 = ctrl[7];
+  const int s = blockIdx.x * FIN_CHUNK + threadIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned below = (1u << lane) - 1u;
+  int b = 0, cd = 0;
+  if (s < n) { b = idx[s]; cd = code[s]; }
+  const unsigned b0 = __ballot_sync(0xffffffffu, cd == 1), b1 = __ballot_sync(0xffffffffu, cd == 2);
+  if (lane == 0) { s_w[0][warp] = __popc(b0); s_w[1][warp] = __popc(b1); }
+  __syncthreads();
+  int o0 = blk_off[blockIdx.x], o1 = base1 + blk_off[nblk + blockIdx.x];
+  for (int w = 0; w < warp; ++w) { o0 += s_w[0][w]; o1 += s_w[1][w]; }
+  if (cd == 1) idx_out[o0 + __popc(b0 & below)] = b;
+  if (cd == 2) idx_out[o1 + __popc(b1 & below)] = b;
+}
+
 __global__ void jacobi_begin_kernel(float* __restrict__ maxdiff, int* __restrict__ idx, int* __restrict__ phase,
                                     int* __restrict__ ctrl, int B, int start_phase) {
-  for (int b = threadIdx.x; b < B; b += blockDim.x) {
+  for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < B; b += gridDim.x * blockDim.x) {
     maxdiff[b] = 0.f;
     idx[b] = b;
     phase[b] = start_phase;
   }
-  if (threadIdx.x == 0) { ctrl[0] = B; ctrl[1] = 0; ctrl[2] = 0; ctrl[3] = start_phase ? B : 0; }
+  if (blockIdx.x == 0 && threadIdx.x == 0) { ctrl[0] = B; ctrl[1] = 0; ctrl[2] = 0; ctrl[3] = start_phase ? B : 0; }
 }
 
 // Rows of nf floats each: dst[s] = src[idx[s]] (to_compact != 0) or dst[idx[s]] = src[s] (to_compact == 0), s < n.
@@ -670,6 +790,57 @@ __global__ void maf_cast_rows_kernel(const float* __restrict__ u, const int* __r
     a[i] = hi;
     if (a_lo != nullptr) a_lo[i] = from_f32<T>(x - to_f32(hi));
   }
+}
+
+// MLP-based flow, the update of Algorithm 1 from a stored output o [n_slots, 2D] (interleaved mu_i, alpha_i): one warp
+// per slot, u[b, i] <- v[b, i] exp(alpha_i) + mu_i for sample b = idx[slot], maxdiff[b] = max_i |u_new - u_old| (the warp
+// owns the row: plain store).  only_col >= 0: only that dimension changes (one step of sequential decoding, Eq. 5).
+__global__ void __launch_bounds__(256) maf_update_kernel(const float* __restrict__ o, const float* __restrict__ v,
+                                                         float* __restrict__ u, float* __restrict__ maxdiff,
+                                                         const int* __restrict__ idx, int n_slots, int D, int only_col) {
+  const int lane = threadIdx.x & 31;
+  const int s = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (s >= n_slots) return;
+  const int b = idx ? idx[s] : s;
+  const float2* orow = reinterpret_cast<const float2*>(o + (size_t)s * 2 * D);
+  const float* vrow = v + (size_t)b * D;
+  float* urow = u + (size_t)b * D;
+  float m = 0.f;
+  if (only_col >= 0) {
+    if (lane == 0) {
+      const float2 p = orow[only_col];
+      const float old = urow[only_col], nw = fmaf(vrow[only_col], expf(p.y), p.x);
+      urow[only_col] = nw;
+      m = fabsf(nw - old);
+      maxdiff[b] = m;
+    }
+    return;
+  }
+  for (int i0 = 0; i0 < D; i0 += 128) {  // four dimensions in flight per lane
+    float2 p[4];
+    float vv[4], old[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int i = i0 + k * 32 + lane;
+      if (i < D) { p[k] = orow[i]; vv[k] = vrow[i]; old[k] = urow[i]; }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int i = i0 + k * 32 + lane;
+      if (i < D) {
+        const float nw = fmaf(vv[k], expf(p[k].y), p[k].x);
+        urow[i] = nw;
+        const float df = fabsf(nw - old[k]);
+        m = (df > m || df != df) ? df : m;
+      }
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {  // NaN-propagating max
+    const float other = __shfl_xor_sync(0xffffffffu, m, off);
+    m = (other > m || other != other) ? other : m;
+  }
+  if (lane == 0) maxdiff[b] = m;
 }
 
 // MLP-based flow, forward direction (Eq. 4): v = (u - mu) exp(-alpha), logdet[b] -= sum alpha.  One CTA per sample

@@ -170,6 +170,10 @@ struct tf_model {
   bool seq_fuse_gelu = false;   // MLP-up step GEMM with K <= 512 applies bias + GELU itself (no K split): one kernel
                                 // less per layer, but 16 CTAs instead of 64 stream the weights; measured slower
   int *idx = nullptr, *idx_tmp = nullptr, *phase = nullptr, *ctrl = nullptr, *iters_sample = nullptr, *err = nullptr;
+  // sweep control of large batches (more than FIN_CHUNK samples): per-slot decisions and per-CTA counts
+  unsigned char* fin_code = nullptr;
+  int *fin_cnt = nullptr, *fin_flag = nullptr;
+  float* fin_top = nullptr;
   // precision policy of Jacobi blocks on the bf16 engine: 0 = escalate per sample, 1 = single bf16
   // operands only, 2 = two-term operands for every sweep
   int precision_mode = 0;
@@ -207,7 +211,7 @@ struct tf_model {
   int maf_H = 0;
   void *maf_a0 = nullptr, *maf_a0_lo = nullptr, *maf_h1 = nullptr, *maf_h1_lo = nullptr, *maf_h2 = nullptr, *maf_h2_lo = nullptr;
   CUtensorMap maf_map[3][2];               // A-operand maps of {a0, h1, h2} x {hi, lo}
-  CUtensorMap* maf_store_maps = nullptr;   // device copy: bulk-store maps of h1, h1_lo, h2, h2_lo
+  CUtensorMap* maf_store_maps = nullptr;   // device copy: bulk-store maps of h1, h1_lo, h2, h2_lo, o (fp32)
   float *io_z = nullptr, *io_x = nullptr;  // staging for the host-buffer entry point
   int* io_labels = nullptr;
   cudaStream_t stream = nullptr;
@@ -946,7 +950,8 @@ static int run_jacobi_block(tf_model* m, int g, int B, const int* labels, const 
     if (m->precision_mode == 2) start_phase = 1;
     else if (m->precision_mode == 0 && tau >= 0.f && tau < m->single_ok_tau) sw = m->switch_threshold;
   }
-  LAUNCH(m, KC_CTRL, jacobi_begin_kernel, 1, 256, 0, m->maxdiff, m->idx, m->phase, m->ctrl, B, start_phase);
+  LAUNCH(m, KC_CTRL, jacobi_begin_kernel, (B + 1023) / 1024 < 64 ? (B + 1023) / 1024 : 64, 256, 0, m->maxdiff, m->idx, m->phase,
+         m->ctrl, B, start_phase);
   int n_active = B, n_hp = start_phase ? B : 0, t = 0;
   const int cap = (op.fallback_sweeps > 0 && op.fallback_sweeps < max_iters) ? op.fallback_sweeps : max_iters;
   while (t < cap && n_active > 0) {
@@ -954,8 +959,19 @@ static int run_jacobi_block(tf_model* m, int g, int B, const int* labels, const 
     const int n_lp = n_active - n_hp;
     if (n_lp > 0) TF_TRY(sweep_pass<T>(m, g, n_lp, u, m->idx, labels, v, u, false));
     if (n_hp > 0) TF_TRY(sweep_pass<T>(m, g, n_hp, u, m->idx + n_lp, labels, v, u, true));
-    LAUNCH_PDL(m, KC_CTRL, jacobi_finalize_kernel, 1, 256, 0, m->maxdiff, m->idx, m->idx_tmp, m->phase, m->ctrl, iters_row,
-           tau, sw, t);
+    if (n_active <= FIN_CHUNK || m->fin_code == nullptr) {
+      LAUNCH_PDL(m, KC_CTRL, jacobi_finalize_kernel, 1, 256, 0, m->maxdiff, m->idx, m->idx_tmp, m->phase, m->ctrl, iters_row,
+                 tau, sw, t);
+    } else {  // large batches: count / scan / scatter over all SMs; the new slot list is written to the other buffer
+      const int nblk = (n_active + FIN_CHUNK - 1) / FIN_CHUNK;
+      LAUNCH(m, KC_CTRL, jacobi_finalize_count_kernel, nblk, FIN_CHUNK, 0, m->maxdiff, m->idx, m->phase, m->ctrl, iters_row,
+             m->fin_code, m->fin_cnt, m->fin_top, m->fin_flag, nblk, tau, sw, t);
+      LAUNCH(m, KC_CTRL, jacobi_finalize_scan_kernel, 1, 256, 0, m->fin_cnt, m->fin_top, m->fin_flag, m->ctrl, nblk);
+      LAUNCH(m, KC_CTRL, jacobi_finalize_scatter_kernel, nblk, FIN_CHUNK, 0, m->idx, m->idx_tmp, m->fin_code, m->fin_cnt, m->ctrl,
+             nblk);
+      TF_TRY(check_launch("sweep control kernels"));
+      int* sw_idx = m->idx; m->idx = m->idx_tmp; m->idx_tmp = sw_idx;
+    }
     if (l2 && t <= m->trace_l2_sweeps) {
       LAUNCH(m, KC_CTRL, l2_distance_kernel, B, 256, 0, u, m->ref_seq,
              m->trace_l2 + ((size_t)g * m->trace_l2_sweeps + (t - 1)) * m->cfg.max_batch, m->L * m->D);
@@ -1124,8 +1140,16 @@ static int maf_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
   const CUtensorMap* map2 = sizeof(T) == 2 ? &m->maf_map[2][0] : nullptr;
   const CUtensorMap* map2_lo = (sizeof(T) == 2 && hp) ? &m->maf_map[2][1] : nullptr;
   if (mode == 0) {
-    EpiMafUpdate epi{v, u_upd, m->maxdiff, idx, bw.b3, D, only_col};
-    return gemm<T>(m, KC_GEMM_HEAD_UPDATE, h2, map2, map2_lo, bw.w3, M, epi);
+    if constexpr (sizeof(T) == 2) {
+      // tensor-core engine: the raw (mu, alpha) leave through bulk stores, a row-per-warp kernel applies the update
+      // (measured: 381 us for the fused lane-per-column epilogue against 85 + 60 us for the pair on 69 k rows)
+      TF_TRY(gemm<T>(m, KC_GEMM_HEAD_UPDATE, h2, map2, map2_lo, bw.w3, M, EpiStoreF32Tma{bw.b3, m->maf_store_maps + 4}));
+      LAUNCH(m, KC_AFFINE, maf_update_kernel, (M + 7) / 8, 256, 0, m->o, v, u_upd, m->maxdiff, idx, M, D, only_col);
+      return check_launch("maf_update_kernel");
+    } else {
+      EpiMafUpdate epi{v, u_upd, m->maxdiff, idx, bw.b3, D, only_col};
+      return gemm<T>(m, KC_GEMM_HEAD_UPDATE, h2, map2, map2_lo, bw.w3, M, epi);
+    }
   }
   return gemm<T>(m, KC_GEMM_HEAD, h2, map2, map2_lo, bw.w3, M, EpiStore<float, ACT_NONE>{m->o, bw.b3, 2 * D});
 }
@@ -1331,6 +1355,13 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
   TF_TRY(dev_alloc(m, &m->idx, B));
   TF_TRY(dev_alloc(m, &m->idx_tmp, B));
   TF_TRY(dev_alloc(m, &m->phase, B));
+  if (B > (size_t)FIN_CHUNK) {
+    const size_t nblk = (B + FIN_CHUNK - 1) / FIN_CHUNK;
+    TF_TRY(dev_alloc(m, &m->fin_code, B));
+    TF_TRY(dev_alloc(m, &m->fin_cnt, 2 * nblk));
+    TF_TRY(dev_alloc(m, &m->fin_top, nblk));
+    TF_TRY(dev_alloc(m, &m->fin_flag, nblk));
+  }
   TF_TRY(dev_alloc(m, &m->ctrl, 8));
   TF_TRY(dev_alloc(m, &m->err, 1));
   TF_TRY(dev_alloc(m, &m->iters_sample, (size_t)c.n_blocks * B));
@@ -1495,6 +1526,13 @@ static int maf_load_impl(tf_model* m, const void* blob, size_t nbytes, int D, in
   TF_TRY(dev_alloc(m, &m->idx, B));
   TF_TRY(dev_alloc(m, &m->idx_tmp, B));
   TF_TRY(dev_alloc(m, &m->phase, B));
+  if (B > (size_t)FIN_CHUNK) {
+    const size_t nblk = (B + FIN_CHUNK - 1) / FIN_CHUNK;
+    TF_TRY(dev_alloc(m, &m->fin_code, B));
+    TF_TRY(dev_alloc(m, &m->fin_cnt, 2 * nblk));
+    TF_TRY(dev_alloc(m, &m->fin_top, nblk));
+    TF_TRY(dev_alloc(m, &m->fin_flag, nblk));
+  }
   TF_TRY(dev_alloc(m, &m->ctrl, 8));
   TF_TRY(dev_alloc(m, &m->err, 1));
   TF_TRY(dev_alloc(m, &m->iters_sample, (size_t)c.n_blocks * B));
@@ -1510,7 +1548,8 @@ static int maf_load_impl(tf_model* m, const void* blob, size_t nbytes, int D, in
     const int cols[3] = {D, H, H};
     for (int i = 0; i < 3; ++i)
       for (int t = 0; t < 2; ++t) TF_TRY(make_map_bf16(&m->maf_map[i][t], bufs[i][t], B, cols[i], tc::BM));
-    CUtensorMap sm[4];
+    CUtensorMap sm[5];
+    TF_TRY(make_map_store(&sm[4], m->o, B, 2 * (uint64_t)D, 4));
     TF_TRY(make_map_store(&sm[0], m->maf_h1, B, H, 2));
     TF_TRY(make_map_store(&sm[1], m->maf_h1_lo, B, H, 2));
     TF_TRY(make_map_store(&sm[2], m->maf_h2, B, H, 2));

@@ -200,7 +200,7 @@ MAF_MAGIC = 0x3146414D  # "MAF1" little endian
 # on binary MNIST (100 images); lattice size and hidden width are not stated, so these stand-ins fix them.
 MAF_CONFIGS = {
     "maf_tiny": dict(D=12, hidden=32, n_blocks=3, dtype=0, B=5, tau=1e-6, z_scale=1.0),
-    "maf_ising": dict(D=256, hidden=1024, n_blocks=8, dtype=1, B=16384, tau=1e-3, z_scale=1.0),
+    "maf_ising": dict(D=256, hidden=1024, n_blocks=8, dtype=1, B=100000, tau=1e-3, z_scale=1.0),
     "maf_mnist": dict(D=784, hidden=1024, n_blocks=8, dtype=1, B=100, tau=1e-3, z_scale=1.0),
 }
 

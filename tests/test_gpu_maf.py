@@ -129,13 +129,17 @@ def test_bf16_ising_shape_sampled_against_oracle():
         assert np.abs(its[:, pick] - ito).max() <= 1
         x2, _, its2, rc2 = m.jacobi(z, cfg["tau"], m.D + 1)
         assert rc2 == 0 and np.array_equal(x, x2) and np.array_equal(its, its2)
+        # the first 900 samples alone (one-CTA sweep control instead of the count / scan / scatter kernels, other row
+        # tiles): a sample's result and schedule do not depend on its batch mates
+        x3, _, its3, rc3 = m.jacobi(z[:900], cfg["tau"], m.D + 1)
+        assert rc3 == 0 and np.array_equal(x3, x[:900]) and np.array_equal(its3, its[:, :900])
 
 
 def test_bf16_ragged_dimension_sequential_forward_and_thresholds():
     """D = 72 (one full and one partial 64-wide k slab in the first layer, 144 output columns), hidden 192, 3 layers."""
     cfg = synth.maf_config("maf_ising", D=72, hidden=192, n_blocks=3)
     B = 37
-    with Maf(cfg, B, out_scale=0.3) as m:
+    with Maf(cfg, B) as m:
         z = synth.make_maf_latents(cfg, 22, B=B)
         xso, _ = MO.model_inverse(m.blocks, z, 0.0, 0, jacobi=False)
         xs = m.sequential(z)
@@ -148,4 +152,4 @@ def test_bf16_ragged_dimension_sequential_forward_and_thresholds():
         zg, ld = m.forward(xso)
         zo, ldo = MO.model_forward(m.blocks, xso)
         assert rel_l2(zg, zo) <= 2e-2 and np.abs(zg - zo).max() <= 5e-2
-        assert np.abs(ld - ldo).max() <= 2e-2 * max(np.abs(ldo).max(), np.sqrt(m.D * m.K) * 0.3)
+        assert np.abs(ld - ldo).max() <= 2e-2 * max(np.abs(ldo).max(), np.sqrt(m.D * m.K) * 0.1)
