@@ -647,7 +647,7 @@ def run_cfg5_sweep(args, binding, synth, torch, timed):
     frow = sweep_flops_per_row(cfg, L, D)
     _, w_blk = seq_block_bytes(cfg, L, D, 1)
     cells = []
-    for B in (1, 8, 64, 256):
+    for B in ((args.batch,) if args.batch else (1, 8, 64, 256)):
         zs = [torch.from_numpy(synth.make_latents(cfg, 7000 + i, B=B)).cuda() for i in range(3)]
         lab = torch.from_numpy(synth.make_labels(cfg, B=B)).cuda()
         x = torch.empty_like(zs[0])

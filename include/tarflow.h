@@ -35,7 +35,10 @@
  *     apply bias + GELU itself when its reduction fits one CTA (K <= 512), TARFLOW_SEQ_FUSE_TAIL=0|1 switches the one-kernel
  *     step tail (final LayerNorm, head, update, embedding, next LayerNorm) off or on whatever the head's size.  Sweeps: TARFLOW_PAIR_GEMM=0 runs the projections with
  *     one CTA per 128x256 tile instead of 2-CTA pairs; TARFLOW_ATTN_TC=0 runs attention on the mma.sync kernel
- *     instead of the tcgen05 one, TARFLOW_ATTN_TC_SPLIT=0 does so for two-term operands only.
+ *     instead of the tcgen05 one, TARFLOW_ATTN_TC_SPLIT=0 does so for two-term operands only.  TARFLOW_SEQ_CHAINS=1|2|4
+ *     sets how many sample chains decode a sequential block side by side (default: 2 from 32 samples up);
+ *     TARFLOW_SWEEP_GRAPH_ROWS=n replays Jacobi sweeps of at most n rows (slots x tokens, default 4096) from CUDA
+ *     graphs, 0 launches every kernel directly.
  */
 #ifndef TARFLOW_H_
 #define TARFLOW_H_

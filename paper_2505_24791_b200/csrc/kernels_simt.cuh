@@ -536,13 +536,14 @@ __global__ void __launch_bounds__(256) forward_affine_kernel(const float* __rest
 // [single-precision samples..., hp samples...] with a stable partition, so the slot order never
 // depends on timing and a sample's schedule depends on that sample alone.
 // ctrl[0] = n_active, ctrl[1] = non-finite flag, ctrl[2] = bits of max over active samples of
-// maxdiff, ctrl[3] = number of active samples in the hp phase (the tail of idx).
+// maxdiff, ctrl[3] = number of active samples in the hp phase (the tail of idx); ctrl[CTRL_SWEEP] = sweeps finished in
+// this block, ctrl[CTRL_TAU] / ctrl[CTRL_SWITCH] = bits of tau and of the escalation threshold.
 // ------------------------------------------------------------------------------------------------
+constexpr int CTRL_WORDS = 16, CTRL_LABEL_FLAG = 5, CTRL_SWEEP = 8, CTRL_TAU = 9, CTRL_SWITCH = 10;
 // One CTA of 256 threads; the order of the surviving samples is kept (stable compaction), single-term samples first.
 __global__ void __launch_bounds__(256)
 jacobi_finalize_kernel(float* __restrict__ maxdiff, int* __restrict__ idx, int* __restrict__ idx_tmp,
-                       int* __restrict__ phase, int* __restrict__ ctrl, int* __restrict__ iters_sample,
-                       float tau, float switch_thresh, int t) {
+                       int* __restrict__ phase, int* __restrict__ ctrl, int* __restrict__ iters_sample) {
   __shared__ int s_cnt[2][8];
   __shared__ float s_top[8];
   __shared__ int s_flag[2][8];
@@ -552,6 +553,10 @@ jacobi_finalize_kernel(float* __restrict__ maxdiff, int* __restrict__ idx, int* 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const unsigned below = (1u << lane) - 1u;
   const int n = ctrl[0];
+  // the sweep number and the two thresholds live in device memory (set by jacobi_begin_kernel), so one captured
+  // launch sequence serves every sweep of a block
+  const int t = ctrl[CTRL_SWEEP] + 1;
+  const float tau = __int_as_float(ctrl[CTRL_TAU]), switch_thresh = __int_as_float(ctrl[CTRL_SWITCH]);
   int base0 = 0, base1 = 0;  // survivors so far: single-term phase, two-term phase
   float top = 0.f;
   int bad = 0, nan = 0;
@@ -604,6 +609,7 @@ jacobi_finalize_kernel(float* __restrict__ maxdiff, int* __restrict__ idx, int* 
     ctrl[1] = anybad;
     ctrl[2] = anynan ? 0x7fc00000 : __float_as_int(top);
     ctrl[3] = base1;
+    ctrl[CTRL_SWEEP] = t;
   }
 }
 
@@ -619,8 +625,10 @@ __global__ void __launch_bounds__(FIN_CHUNK)
 jacobi_finalize_count_kernel(float* __restrict__ maxdiff, const int* __restrict__ idx, int* __restrict__ phase,
                              const int* __restrict__ ctrl, int* __restrict__ iters_sample, unsigned char* __restrict__ code,
                              int* __restrict__ blk_cnt /*[2][nblk]*/, float* __restrict__ blk_top, int* __restrict__ blk_flag,
-                             int nblk, float tau, float switch_thresh, int t) {
+                             int nblk) {
   const int n = ctrl[0];
+  const int t = ctrl[CTRL_SWEEP] + 1;
+  const float tau = __int_as_float(ctrl[CTRL_TAU]), switch_thresh = __int_as_float(ctrl[CTRL_SWITCH]);
   const int s = blockIdx.x * FIN_CHUNK + threadIdx.x;
   bool f0 = false, f1 = false;
   float top = 0.f;
@@ -705,6 +713,7 @@ jacobi_finalize_scan_kernel(int* __restrict__ blk_cnt, const float* __restrict__
     ctrl[2] = (flags & 2) ? 0x7fc00000 : __float_as_int(top);
     ctrl[3] = base1;
     ctrl[7] = base0;                   // two-term survivors start here
+    ctrl[CTRL_SWEEP] = ctrl[CTRL_SWEEP] + 1;
   }
 }
 
@@ -728,13 +737,18 @@ jacobi_finalize_scatter_kernel(const int* __restrict__ idx, int* __restrict__ id
 }
 
 __global__ void jacobi_begin_kernel(float* __restrict__ maxdiff, int* __restrict__ idx, int* __restrict__ phase,
-                                    int* __restrict__ ctrl, int B, int start_phase) {
+                                    int* __restrict__ ctrl, int B, int start_phase, float tau, float switch_thresh) {
   for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < B; b += gridDim.x * blockDim.x) {
     maxdiff[b] = 0.f;
     idx[b] = b;
     phase[b] = start_phase;
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0) { ctrl[0] = B; ctrl[1] = 0; ctrl[2] = 0; ctrl[3] = start_phase ? B : 0; }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    ctrl[0] = B; ctrl[1] = 0; ctrl[2] = 0; ctrl[3] = start_phase ? B : 0;
+    ctrl[CTRL_SWEEP] = 0;
+    ctrl[CTRL_TAU] = __float_as_int(tau);
+    ctrl[CTRL_SWITCH] = __float_as_int(switch_thresh);
+  }
 }
 
 // Rows of nf floats each: dst[s] = src[idx[s]] (to_compact != 0) or dst[idx[s]] = src[s] (to_compact == 0), s < n.

@@ -192,6 +192,9 @@ struct tf_model {
   cudaEvent_t seq_fork = nullptr, seq_join[MAX_CHAINS] = {nullptr};
   int seq_chains_force = 0;  // TARFLOW_SEQ_CHAINS=1|2|4: chains per sequential block (0 = by the size of the weights)
   int seq_kbn_force = 0;     // TARFLOW_SEQ_KBN
+  // Jacobi sweeps over few rows are replayed from graphs: one per (block, single-term slots, two-term slots, buffers)
+  std::map<std::tuple<int, int, int, const void*, const void*, const void*, const void*>, SeqGraph> sweep_graphs;
+  int64_t sweep_graph_rows = 4096;  // TARFLOW_SWEEP_GRAPH_ROWS: largest slots x tokens replayed from a graph (0 = never)
   int seq_variant = 0;       // 0: the block's own token buffers, 1: the compact buffers of the sequential fall-back
   size_t seq_part_row_floats = 0;  // floats of partial tiles available per sample
   bool use_graphs = true;
@@ -897,12 +900,12 @@ static int take_labels(tf_model* m, const int** labels, int B) {
     *labels = nullptr;
     return TF_OK;
   }
-  LAUNCH(m, KC_CTRL, labels_check_kernel, (B + 127) / 128, 128, 0, *labels, m->labels_own, B, m->cfg.n_classes, m->ctrl + 5);
+  LAUNCH(m, KC_CTRL, labels_check_kernel, (B + 127) / 128, 128, 0, *labels, m->labels_own, B, m->cfg.n_classes, m->ctrl + CTRL_LABEL_FLAG);
   TF_TRY(check_launch("labels_check_kernel"));
-  CU_OK(cudaMemcpyAsync(m->ctrl_host + 5, m->ctrl + 5, sizeof(int), cudaMemcpyDeviceToHost, m->stream));
+  CU_OK(cudaMemcpyAsync(m->ctrl_host + 5, m->ctrl + CTRL_LABEL_FLAG, sizeof(int), cudaMemcpyDeviceToHost, m->stream));
   CU_OK(cudaStreamSynchronize(m->stream));
   if (m->ctrl_host[5] != 0) {
-    CU_OK(cudaMemsetAsync(m->ctrl + 5, 0, sizeof(int), m->stream));
+    CU_OK(cudaMemsetAsync(m->ctrl + CTRL_LABEL_FLAG, 0, sizeof(int), m->stream));
     return fail(TF_EINVAL, "a class label lies outside [0, %d)", m->cfg.n_classes);
   }
   *labels = m->labels_own;
@@ -951,26 +954,70 @@ static int run_jacobi_block(tf_model* m, int g, int B, const int* labels, const 
     else if (m->precision_mode == 0 && tau >= 0.f && tau < m->single_ok_tau) sw = m->switch_threshold;
   }
   LAUNCH(m, KC_CTRL, jacobi_begin_kernel, (B + 1023) / 1024 < 64 ? (B + 1023) / 1024 : 64, 256, 0, m->maxdiff, m->idx, m->phase,
-         m->ctrl, B, start_phase);
+         m->ctrl, B, start_phase, tau, sw);
   int n_active = B, n_hp = start_phase ? B : 0, t = 0;
   const int cap = (op.fallback_sweeps > 0 && op.fallback_sweeps < max_iters) ? op.fallback_sweeps : max_iters;
-  while (t < cap && n_active > 0) {
-    ++t;
-    const int n_lp = n_active - n_hp;
+  // everything one sweep launches: the pass over the single-term samples, the pass over the two-term samples, the
+  // sweep control (which takes the sweep number and the thresholds from device memory)
+  auto enqueue_sweep = [&](int n_lp, int n_hpp) -> int {
     if (n_lp > 0) TF_TRY(sweep_pass<T>(m, g, n_lp, u, m->idx, labels, v, u, false));
-    if (n_hp > 0) TF_TRY(sweep_pass<T>(m, g, n_hp, u, m->idx + n_lp, labels, v, u, true));
-    if (n_active <= FIN_CHUNK || m->fin_code == nullptr) {
-      LAUNCH_PDL(m, KC_CTRL, jacobi_finalize_kernel, 1, 256, 0, m->maxdiff, m->idx, m->idx_tmp, m->phase, m->ctrl, iters_row,
-                 tau, sw, t);
+    if (n_hpp > 0) TF_TRY(sweep_pass<T>(m, g, n_hpp, u, m->idx + n_lp, labels, v, u, true));
+    const int na = n_lp + n_hpp;
+    if (na <= FIN_CHUNK || m->fin_code == nullptr) {
+      LAUNCH_PDL(m, KC_CTRL, jacobi_finalize_kernel, 1, 256, 0, m->maxdiff, m->idx, m->idx_tmp, m->phase, m->ctrl, iters_row);
     } else {  // large batches: count / scan / scatter over all SMs; the new slot list is written to the other buffer
-      const int nblk = (n_active + FIN_CHUNK - 1) / FIN_CHUNK;
+      const int nblk = (na + FIN_CHUNK - 1) / FIN_CHUNK;
       LAUNCH(m, KC_CTRL, jacobi_finalize_count_kernel, nblk, FIN_CHUNK, 0, m->maxdiff, m->idx, m->phase, m->ctrl, iters_row,
-             m->fin_code, m->fin_cnt, m->fin_top, m->fin_flag, nblk, tau, sw, t);
+             m->fin_code, m->fin_cnt, m->fin_top, m->fin_flag, nblk);
       LAUNCH(m, KC_CTRL, jacobi_finalize_scan_kernel, 1, 256, 0, m->fin_cnt, m->fin_top, m->fin_flag, m->ctrl, nblk);
       LAUNCH(m, KC_CTRL, jacobi_finalize_scatter_kernel, nblk, FIN_CHUNK, 0, m->idx, m->idx_tmp, m->fin_code, m->fin_cnt, m->ctrl,
              nblk);
-      TF_TRY(check_launch("sweep control kernels"));
       int* sw_idx = m->idx; m->idx = m->idx_tmp; m->idx_tmp = sw_idx;
+    }
+    return check_launch("sweep control kernels");
+  };
+  while (t < cap && n_active > 0) {
+    ++t;
+    const int n_lp = n_active - n_hp;
+    // Few rows: a sweep is a chain of short kernels whose launch cost exceeds their run time, so the whole sweep is
+    // captured once per (block, single-term slots, two-term slots) and replayed as a graph afterwards.
+    const bool as_graph = m->use_graphs && m->cap_stream != nullptr && !m->prof_on && n_active <= FIN_CHUNK && (int64_t)n_active * m->L <= m->sweep_graph_rows;
+    if (as_graph) {
+      const auto key = std::make_tuple(g, n_lp, n_hp, (const void*)v, (const void*)u, (const void*)labels, (const void*)iters_row);
+      auto it = m->sweep_graphs.find(key);
+      if (it == m->sweep_graphs.end() && m->sweep_graphs.size() < 2048) {
+        tf_model::SeqGraph sg;
+        const int64_t before = m->launches;
+        cudaStream_t user = m->stream;
+        cudaGraph_t graph = nullptr;
+        m->stream = m->cap_stream;
+        cudaError_t e = cudaStreamBeginCapture(m->cap_stream, cudaStreamCaptureModeRelaxed);
+        int r = TF_OK;
+        if (e == cudaSuccess) {
+          r = enqueue_sweep(n_lp, n_hp);
+          e = cudaStreamEndCapture(m->cap_stream, &graph);
+        }
+        m->stream = user;
+        sg.nodes = (int)(m->launches - before);
+        m->launches = before;
+        if (e != cudaSuccess || r != TF_OK || !graph) {
+          if (graph) cudaGraphDestroy(graph);
+          cudaGetLastError();
+          return r != TF_OK ? r : fail(TF_ECUDA, "capturing a sweep graph failed: %s", cudaGetErrorString(e));
+        }
+        e = cudaGraphInstantiate(&sg.exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (e != cudaSuccess) return fail(TF_ECUDA, "cudaGraphInstantiate: %s", cudaGetErrorString(e));
+        it = m->sweep_graphs.emplace(key, sg).first;
+      }
+      if (it != m->sweep_graphs.end()) {
+        CU_OK(cudaGraphLaunch(it->second.exec, m->stream));
+        m->launches += it->second.nodes;
+      } else {
+        TF_TRY(enqueue_sweep(n_lp, n_hp));
+      }
+    } else {
+      TF_TRY(enqueue_sweep(n_lp, n_hp));
     }
     if (l2 && t <= m->trace_l2_sweeps) {
       LAUNCH(m, KC_CTRL, l2_distance_kernel, B, 256, 0, u, m->ref_seq,
@@ -1362,7 +1409,7 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     TF_TRY(dev_alloc(m, &m->fin_top, nblk));
     TF_TRY(dev_alloc(m, &m->fin_flag, nblk));
   }
-  TF_TRY(dev_alloc(m, &m->ctrl, 8));
+  TF_TRY(dev_alloc(m, &m->ctrl, CTRL_WORDS));
   TF_TRY(dev_alloc(m, &m->err, 1));
   TF_TRY(dev_alloc(m, &m->iters_sample, (size_t)c.n_blocks * B));
   TF_TRY(dev_alloc(m, &m->io_z, B * c.C * c.H * c.W));
@@ -1379,7 +1426,7 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     TF_TRY(dev_alloc(m, &m->seq_part, m->seq_part_floats));
   }
   CU_OK(cudaMemset(m->step_ctr, 0, 16 * tf_model::MAX_CHAINS * sizeof(int)));
-  CU_OK(cudaMemset(m->ctrl, 0, 8 * sizeof(int)));
+  CU_OK(cudaMemset(m->ctrl, 0, CTRL_WORDS * sizeof(int)));
   CU_OK(cudaMemset(m->err, 0, sizeof(int)));
   CU_OK(cudaMemset(m->iters_sample, 0, (size_t)c.n_blocks * B * sizeof(int)));
   CU_OK(cudaMallocHost(&m->ctrl_host, 8 * sizeof(int)));
@@ -1445,6 +1492,7 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     CU_OK(cudaEventCreateWithFlags(&m->seq_fork, cudaEventDisableTiming));
     if (const char* e = getenv("TARFLOW_SEQ_CHAINS")) m->seq_chains_force = atoi(e);
     if (const char* e = getenv("TARFLOW_SEQ_KBN")) m->seq_kbn_force = atoi(e);
+    if (const char* e = getenv("TARFLOW_SWEEP_GRAPH_ROWS")) m->sweep_graph_rows = atoll(e);
   }
   CU_OK(cudaDeviceSynchronize());
   return TF_OK;
@@ -1533,10 +1581,10 @@ static int maf_load_impl(tf_model* m, const void* blob, size_t nbytes, int D, in
     TF_TRY(dev_alloc(m, &m->fin_top, nblk));
     TF_TRY(dev_alloc(m, &m->fin_flag, nblk));
   }
-  TF_TRY(dev_alloc(m, &m->ctrl, 8));
+  TF_TRY(dev_alloc(m, &m->ctrl, CTRL_WORDS));
   TF_TRY(dev_alloc(m, &m->err, 1));
   TF_TRY(dev_alloc(m, &m->iters_sample, (size_t)c.n_blocks * B));
-  CU_OK(cudaMemset(m->ctrl, 0, 8 * sizeof(int)));
+  CU_OK(cudaMemset(m->ctrl, 0, CTRL_WORDS * sizeof(int)));
   CU_OK(cudaMemset(m->err, 0, sizeof(int)));
   CU_OK(cudaMemset(m->maxdiff, 0, B * sizeof(float)));
   CU_OK(cudaMemset(m->iters_sample, 0, (size_t)c.n_blocks * B * sizeof(int)));
@@ -1557,6 +1605,8 @@ static int maf_load_impl(tf_model* m, const void* blob, size_t nbytes, int D, in
     TF_TRY(dev_alloc(m, reinterpret_cast<char**>(&m->maf_store_maps), sizeof(sm)));
     CU_OK(cudaMemcpy(m->maf_store_maps, sm, sizeof(sm), cudaMemcpyHostToDevice));
     if (const char* e = getenv("TARFLOW_PAIR_GEMM")) m->use_pair_gemm = atoi(e) != 0;
+    if (const char* e = getenv("TARFLOW_SWEEP_GRAPH_ROWS")) m->sweep_graph_rows = atoll(e);
+    CU_OK(cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking));
   }
   CU_OK(cudaDeviceSynchronize());
   return TF_OK;
@@ -1617,6 +1667,7 @@ void tf_free(tf_model* m) {
   for (cudaEvent_t e : m->ev_pool) cudaEventDestroy(e);
   for (cudaEvent_t e : m->block_ev) if (e) cudaEventDestroy(e);
   for (auto& kv : m->seq_graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+  for (auto& kv : m->sweep_graphs) if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
   if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
   for (int c = 0; c < tf_model::MAX_CHAINS; ++c) {
     if (m->seq_streams[c]) cudaStreamDestroy(m->seq_streams[c]);
