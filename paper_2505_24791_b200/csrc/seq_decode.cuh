@@ -223,6 +223,46 @@ seq_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W, int B, i
 // Every wait is bounded (see gemm_tc.cuh); a wait that expires records a code in *err and the CTA
 // leaves without storing.
 // ---------------------------------------------------------------------------------------------
+// Fixed-order sum of the K-slice partials of 4 consecutive outputs of row b, plus their bias.
+__device__ __forceinline__ float4 sum_partials4(const float* __restrict__ part, const float* __restrict__ bias, int nsplit,
+                                                int B, int N, int b, int n4) {
+  float4 acc = *reinterpret_cast<const float4*>(bias + 4 * n4);
+  float4 p[8];
+  for (int s0 = 0; s0 < nsplit; s0 += 8) {
+#pragma unroll
+    for (int sl = 0; sl < 8; ++sl)
+      if (s0 + sl < nsplit) p[sl] = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)(s0 + sl) * B + b) * N) + n4);
+#pragma unroll
+    for (int sl = 0; sl < 8; ++sl)
+      if (s0 + sl < nsplit) { acc.x += p[sl].x; acc.y += p[sl].y; acc.z += p[sl].z; acc.w += p[sl].w; }
+  }
+  return acc;
+}
+
+// What the LAST K slice of a column tile to finish does with the complete sums (the CTAs of a tile take a ticket after
+// their partial tile is visible; no CTA waits for another):
+//   mode 1: out_bf16[row, n] = bf16(GELU(bias[n] + sum of partials))          (the MLP hidden layer)
+//   mode 2: h[row, n] += bias[n] + sum of partials, and stats[tile][row] = (sum, sum of squares) of the new h over
+//           the tile's 128 columns                                            (a residual projection; the statistics
+//           are what the LayerNorm of the next projection's input needs)
+// The sums run over the K slices in index order whoever arrives last, so results do not depend on scheduling.
+struct SeqFin {
+  int mode = 0;
+  int* tickets = nullptr;     // [row tiles][column tiles], zero between launches (the last arriver resets its own)
+  const float* bias = nullptr;
+  bf16* out_bf16 = nullptr;   // mode 1: [B, N]
+  float* h = nullptr;         // mode 2: [B, N]
+  float2* stats = nullptr;    // mode 2: [column tiles][B]
+};
+// Non-null h: the activation operand is bf16(LayerNorm(h) * gamma + beta), computed by the CTA for its own K slice
+// from the fp32 rows and the per-tile statistics a SeqFin mode-2 launch left, instead of a TMA load of a stored copy.
+struct SeqLnA {
+  const float* h = nullptr;       // [B, K]
+  const float2* stats = nullptr;  // [K / 128][B]
+  const float* gamma = nullptr;
+  const float* beta = nullptr;
+};
+
 // NS = slab buffers (kbn <= NS).  With gelu_out != null (one K slice only: gridDim.y == 1) the CTA holds finished
 // sums and writes bf16(GELU(sum + bias)) itself instead of a partial tile, which saves the consumer kernel.
 template <int RT, int NS = 4>
@@ -232,9 +272,12 @@ template <int RT, int NS = 4>
 __global__ void __launch_bounds__(128)
 seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a, int row_base, int B,
                    int N, int kbn, float* __restrict__ part, const int* __restrict__ step_base, int step_off, int n_steps,
-                   int check_steps, int* err, const float* __restrict__ gelu_bias, bf16* __restrict__ gelu_out) {
+                   int check_steps, int* err, const float* __restrict__ gelu_bias, bf16* __restrict__ gelu_out, SeqFin fin,
+                   SeqLnA lna) {
   using namespace tc;
   pdl_launch_dependents();
+  __shared__ float s_mean[RT], s_rstd[RT];
+  __shared__ int s_last;
   constexpr int W_BYTES = 128 * 64 * 2, A_BYTES = RT * 64 * 2, STAGE = W_BYTES + A_BYTES;
   constexpr uint32_t TMEM_COLS = RT < 32 ? 32 : RT;
   extern __shared__ uint8_t smem_seq_tc[];
@@ -263,16 +306,58 @@ seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
 
   if (threadIdx.x == 0) {  // weight slabs: constants, requested before the previous kernel has finished
     for (int kb = 0; kb < kbn; ++kb) {
-      mbar_arrive_expect_tx(bar_base + 8u * kb, STAGE);
+      mbar_arrive_expect_tx(bar_base + 8u * kb, lna.h != nullptr ? W_BYTES : STAGE);
       tma_load_2d(smem_base + kb * STAGE, &map_w, k0 + kb * 64, n0, bar_base + 8u * kb);
     }
   }
   pdl_wait();  // activations and the step counter are complete from here on
   const bool skip = check_steps && (*step_base + step_off >= n_steps);
   bool ok = true;
+  if (lna.h != nullptr) {
+    // the activation slabs: LayerNorm of this CTA's K slice of the fp32 rows, written in the 128-byte-swizzled
+    // K-major layout the tensor core reads (what the TMA load of a stored copy would have produced)
+    const int K = kbn * 64 * (int)gridDim.y, stat_tiles = K >> 7;
+    const int nrows_a = (B - row0) < RT ? (B - row0) : RT;
+    if (threadIdx.x < RT) {
+      float sum = 0.f, sq = 0.f;
+      if ((int)threadIdx.x < nrows_a)
+        for (int tl = 0; tl < stat_tiles; ++tl) {
+          const float2 st = __ldcg(lna.stats + (size_t)tl * B + row0 + threadIdx.x);
+          sum += st.x;
+          sq += st.y;
+        }
+      const float mean = sum / K;
+      s_mean[threadIdx.x] = mean;
+      s_rstd[threadIdx.x] = rsqrtf(fmaxf(sq / K - mean * mean, 0.f) + 1e-5f);
+    }
+    __syncthreads();
+    const int chunks_per_row = kbn * 8;  // 16-byte chunks (8 bf16) of a row of this K slice
+    for (int c = threadIdx.x; c < RT * chunks_per_row; c += 128) {
+      const int r = c / chunks_per_row, q = c - r * chunks_per_row, kb = q >> 3, kk = q & 7;
+      uint4 pk = make_uint4(0u, 0u, 0u, 0u);
+      if (r < nrows_a) {
+        const int col = k0 + kb * 64 + kk * 8;
+        const float4 x0 = __ldcg(reinterpret_cast<const float4*>(lna.h + (size_t)(row0 + r) * K + col));
+        const float4 x1 = __ldcg(reinterpret_cast<const float4*>(lna.h + (size_t)(row0 + r) * K + col) + 1);
+        const float4 g0 = *reinterpret_cast<const float4*>(lna.gamma + col), g1 = *reinterpret_cast<const float4*>(lna.gamma + col + 4);
+        const float4 b0 = *reinterpret_cast<const float4*>(lna.beta + col), b1 = *reinterpret_cast<const float4*>(lna.beta + col + 4);
+        const float mean = s_mean[r], rstd = s_rstd[r];
+        const __nv_bfloat162 o0 = __floats2bfloat162_rn((x0.x - mean) * rstd * g0.x + b0.x, (x0.y - mean) * rstd * g0.y + b0.y);
+        const __nv_bfloat162 o1 = __floats2bfloat162_rn((x0.z - mean) * rstd * g0.z + b0.z, (x0.w - mean) * rstd * g0.w + b0.w);
+        const __nv_bfloat162 o2 = __floats2bfloat162_rn((x1.x - mean) * rstd * g1.x + b1.x, (x1.y - mean) * rstd * g1.y + b1.y);
+        const __nv_bfloat162 o3 = __floats2bfloat162_rn((x1.z - mean) * rstd * g1.z + b1.z, (x1.w - mean) * rstd * g1.w + b1.w);
+        pk.x = *reinterpret_cast<const uint32_t*>(&o0); pk.y = *reinterpret_cast<const uint32_t*>(&o1);
+        pk.z = *reinterpret_cast<const uint32_t*>(&o2); pk.w = *reinterpret_cast<const uint32_t*>(&o3);
+      }
+      *reinterpret_cast<uint4*>(smem + kb * STAGE + W_BYTES + swz128(r, kk)) = pk;
+    }
+    fence_proxy_async_smem();  // generic-proxy writes above are read by the tensor core through the async proxy
+    __syncthreads();
+  }
   if (threadIdx.x == 0) {
-    for (int kb = 0; kb < kbn; ++kb)
-      tma_load_2d(smem_base + kb * STAGE + W_BYTES, &map_a, k0 + kb * 64, row_base + row0, bar_base + 8u * kb);
+    if (lna.h == nullptr)
+      for (int kb = 0; kb < kbn; ++kb)
+        tma_load_2d(smem_base + kb * STAGE + W_BYTES, &map_a, k0 + kb * 64, row_base + row0, bar_base + 8u * kb);
     constexpr uint32_t idesc = make_idesc(RT);
     for (int kb = 0; kb < kbn && ok; ++kb) {
       ok = mbar_wait(bar_base + 8u * kb, 0u, err, TFERR_WAIT_FULL);
@@ -300,8 +385,8 @@ seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         if (c * 32 + j < RT) tile[(c * 32 + j) * TP + warp * 32 + lane] = v[j];
     }
   }
-  __syncthreads();
-  if (ok && !skip) {
+  const bool good = __syncthreads_and(ok && !skip) != 0;  // the same for every thread of the CTA
+  if (good) {
     const int nrows = (B - row0) < RT ? (B - row0) : RT;
     const int n = n0 + 4 * lane;
     float* out = part + ((size_t)ks * B + row0) * N + n;
@@ -331,6 +416,48 @@ seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
       }
     }
   }
+  if (fin.mode != 0 && good) {
+    __threadfence();  // this CTA's partial tile is visible device-wide before its ticket is taken
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int* tk = fin.tickets + blockIdx.z * gridDim.x + blockIdx.x;
+      const int got = atomicAdd(tk, 1);
+      s_last = got == (int)gridDim.y - 1;
+      if (s_last) *tk = 0;  // nobody else touches the ticket of this tile any more: ready for the next launch
+    }
+    __syncthreads();
+    if (s_last) {
+      __threadfence();
+      const int nrows = (B - row0) < RT ? (B - row0) : RT;
+      const int n = n0 + 4 * lane, nsplit = (int)gridDim.y;  // N % 4 == 0 (checked by the host)
+      for (int r = warp; r < nrows; r += 4) {
+        float sum = 0.f, sq = 0.f;
+        if (n < N) {
+          float4 x = sum_partials4(part, fin.bias, nsplit, B, N, row0 + r, n >> 2);
+          if (fin.mode == 1) {
+            const __nv_bfloat162 o0 = __floats2bfloat162_rn(gelu_erf(x.x), gelu_erf(x.y));
+            const __nv_bfloat162 o1 = __floats2bfloat162_rn(gelu_erf(x.z), gelu_erf(x.w));
+            uint2 w2;
+            w2.x = *reinterpret_cast<const uint32_t*>(&o0);
+            w2.y = *reinterpret_cast<const uint32_t*>(&o1);
+            *reinterpret_cast<uint2*>(fin.out_bf16 + (size_t)(row0 + r) * N + n) = w2;
+          } else {
+            float4* hp = reinterpret_cast<float4*>(fin.h + (size_t)(row0 + r) * N + n);
+            const float4 old = __ldcg(hp);
+            x.x += old.x; x.y += old.y; x.z += old.z; x.w += old.w;
+            *hp = x;
+            sum = (x.x + x.y) + (x.z + x.w);
+            sq = (x.x * x.x + x.y * x.y) + (x.z * x.z + x.w * x.w);
+          }
+        }
+        if (fin.mode == 2) {  // the warp holds the 128 columns of row r of this tile
+          sum = warp_sum(sum);
+          sq = warp_sum(sq);
+          if (lane == 0) fin.stats[(size_t)blockIdx.x * B + row0 + r] = make_float2(sum, sq);
+        }
+      }
+    }
+  }
   tcgen05_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -341,22 +468,6 @@ seq_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     tcgen05_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
-}
-
-// Fixed-order sum of the K-slice partials of 4 consecutive outputs of row b, plus their bias.
-__device__ __forceinline__ float4 sum_partials4(const float* __restrict__ part, const float* __restrict__ bias, int nsplit,
-                                                int B, int N, int b, int n4) {
-  float4 acc = *reinterpret_cast<const float4*>(bias + 4 * n4);
-  float4 p[8];
-  for (int s0 = 0; s0 < nsplit; s0 += 8) {
-#pragma unroll
-    for (int sl = 0; sl < 8; ++sl)
-      if (s0 + sl < nsplit) p[sl] = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)(s0 + sl) * B + b) * N) + n4);
-#pragma unroll
-    for (int sl = 0; sl < 8; ++sl)
-      if (s0 + sl < nsplit) { acc.x += p[sl].x; acc.y += p[sl].y; acc.z += p[sl].z; acc.w += p[sl].w; }
-  }
-  return acc;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -552,7 +663,8 @@ seq_attention_kernel(const float* __restrict__ part, int nsplit, const float* __
 // grid = (B, ceil(d / blockDim.x)): every CTA of a sample recomputes the D values of the token (cheap) and
 // embeds blockDim.x channels, one per thread; the CTA with blockIdx.y == 0 stores the token.  With
 // first != 0 the step is the block's start: u[b, 0, :] = v[b, 0, :] (Eq. 5, first row) and the
-// embedding of token 0.
+// embedding of token 0.  stats != null (128 threads per CTA, d % 128 == 0): also (sum, sum of squares) of the CTA's 128
+// channels per sample, the statistics layer 0's projection needs to normalise the row itself.
 // ---------------------------------------------------------------------------------------------
 __global__ void seq_update_embed_kernel(const float* __restrict__ part, int nsplit, const float* __restrict__ bias,
                                         int B, const float* __restrict__ v, float* __restrict__ u,
@@ -560,7 +672,7 @@ __global__ void seq_update_embed_kernel(const float* __restrict__ part, int nspl
                                         const float* __restrict__ b_in, const float* __restrict__ pos,
                                         const float* __restrict__ cls, float* __restrict__ h, int L, int D, int d,
                                         int reversed, int first, const int* __restrict__ step_base, int step_off,
-                                        int n_steps) {
+                                        int n_steps, float2* __restrict__ stats) {
   pdl_launch_dependents();
   pdl_wait();
   const int t = *step_base + step_off;
@@ -598,7 +710,17 @@ __global__ void seq_update_embed_kernel(const float* __restrict__ part, int nspl
     a3 = fmaf(s_tok[c + 3], w_in_t[(size_t)(c + 3) * d + j], a3);
   }
   for (; c < D; ++c) a0 = fmaf(s_tok[c], w_in_t[(size_t)c * d + j], a0);
-  h[(size_t)b * d + j] = acc + ((a0 + a1) + (a2 + a3));
+  const float hv = acc + ((a0 + a1) + (a2 + a3));
+  h[(size_t)b * d + j] = hv;
+  if (stats != nullptr) {  // blockDim.x == 128 and d % 128 == 0 here: the CTA holds one 128-column tile of the row
+    __shared__ float s_red[2][4];
+    const float sm = warp_sum(hv), sq = warp_sum(hv * hv);
+    if ((threadIdx.x & 31) == 0) { s_red[0][threadIdx.x >> 5] = sm; s_red[1][threadIdx.x >> 5] = sq; }
+    __syncthreads();
+    if (threadIdx.x == 0)
+      stats[(size_t)blockIdx.y * B + b] = make_float2((s_red[0][0] + s_red[0][1]) + (s_red[0][2] + s_red[0][3]),
+                                                      (s_red[1][0] + s_red[1][1]) + (s_red[1][2] + s_red[1][3]));
+  }
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -191,6 +191,16 @@ struct tf_model {
   cudaStream_t seq_streams[MAX_CHAINS] = {nullptr};  // one stream per chain of a sequential block
   cudaEvent_t seq_fork = nullptr, seq_join[MAX_CHAINS] = {nullptr};
   int seq_chains_force = 0;  // TARFLOW_SEQ_CHAINS=1|2|4: chains per sequential block (0 = by the size of the weights)
+  enum { SEQ_TICKETS = 1024 };
+  int* seq_tickets = nullptr;      // [MAX_CHAINS][SEQ_TICKETS]
+  float2* seq_stats = nullptr;     // [MAX_CHAINS][16 column tiles][max_batch]
+  bool seq_kbn8 = true;            // TARFLOW_SEQ_KBN8=0: finishing launches never take eight k slabs per CTA
+  // TARFLOW_SEQ_FIN=1: five kernels per layer instead of eight (the last K slice of a projection finishes its tile, the
+  // next projection normalises its own operand slice).  Off by default: measured 55.8 / 144.7 / 416 ms per block against
+  // 28.3 / 84.1 / 283 ms for the eight-kernel chain (256 tokens width 512, 256 tokens width 1024, 1024 tokens): the
+  // fence + ticket + fence of the last arriver and its one-CTA reduction cost more than the kernel boundary and the
+  // many-CTA consumer kernel they replace.
+  bool seq_fin = false;
   int seq_kbn_force = 0;     // TARFLOW_SEQ_KBN
   // Jacobi sweeps over few rows are replayed from graphs: one per (block, single-term slots, two-term slots, buffers)
   std::map<std::tuple<int, int, int, const void*, const void*, const void*, const void*>, SeqGraph> sweep_graphs;
@@ -604,6 +614,8 @@ struct SeqCtx {
   int b0 = 0, B = 0;
   int* step_ctr = nullptr;
   float* part = nullptr;
+  int* tickets = nullptr;    // last-arriver tickets of the step GEMMs' column tiles (zero between launches)
+  float2* stats = nullptr;   // per column tile and sample: (sum, sum of squares) of the residual row, for the next LayerNorm
 };
 
 // One skinny GEMM of a decoding step: part[ks][B, N] = A[B, K slice ks] W[N, K slice ks]^T.  Returns the number of
@@ -613,7 +625,8 @@ struct SeqCtx {
 // fits one CTA (K <= 512) the GEMM writes that itself and *nsplit = 0; otherwise it writes partial tiles as usual
 // and the caller runs the bias + GELU kernel.
 static int seq_gemm(tf_model* m, const SeqCtx& cx, int cls, int abuf, const Matrix& W, int step_off, int* nsplit,
-                    const float* gelu_bias = nullptr, bf16* gelu_out = nullptr) {
+                    const float* gelu_bias = nullptr, bf16* gelu_out = nullptr, const seq::SeqFin* fin = nullptr,
+                    const seq::SeqLnA* lna = nullptr) {
   const int N = W.N, K = W.K, n_steps = m->L - 1, B = cx.B;
   const bf16* A = reinterpret_cast<const bf16*>(abuf == 0 ? m->xn : abuf == 1 ? m->att : m->mlp) + (size_t)cx.b0 * K;
   const bf16* w = reinterpret_cast<const bf16*>(W.w);
@@ -623,30 +636,46 @@ static int seq_gemm(tf_model* m, const SeqCtx& cx, int cls, int abuf, const Matr
     dim3 grid((N + 127) / 128, 1, (B + 63) / 64);
     return launch_seq(m, cls, seq::seq_gemm_tc_kernel<64, 8>, grid, 128, seq::gemm_tc_smem_bytes<64, 8>(), W.map_seq,
                       m->map_seq_a[abuf][2], cx.b0, B, N, K / 64, cx.part, cx.step_ctr, step_off, n_steps, m->seq_check_steps,
-                      m->err, gelu_bias, gelu_out + (size_t)cx.b0 * N);
+                      m->err, gelu_bias, gelu_out + (size_t)cx.b0 * N, seq::SeqFin{}, seq::SeqLnA{});
   }
   if (m->seq_use_tc) {  // tcgen05 kernel: CTAs of 128 columns x kbn slabs of 64 k
     const int slabs = K / 64;
     int kbn = slabs % 4 == 0 ? 4 : slabs % 2 == 0 ? 2 : 1;
     // two slabs per CTA (more CTAs) while the grid is below one wave and the partial tiles stay <= 16
     if (kbn == 4 && ((N + 127) / 128) * (slabs / 4) < m->num_sms && slabs / 2 <= 16) kbn = 2;
+    // a launch whose last K slice finishes the tile reads all partials of it: keep them to eight where that is possible
+    if (fin != nullptr && slabs / kbn > 8 && slabs % 4 == 0) kbn = 4;
+    if (fin != nullptr && slabs / kbn > 8 && slabs % 8 == 0 && m->seq_kbn8) kbn = 8;  // eight slab buffers per CTA
     if (m->seq_kbn_force > 0 && slabs % m->seq_kbn_force == 0 && slabs / m->seq_kbn_force <= 16) kbn = m->seq_kbn_force;
     const int ksplit = slabs / kbn;
     if (ksplit > 16) return fail(TF_EINVAL, "sequential decoding: reduction length %d not supported", K);
-    *nsplit = ksplit;
+    *nsplit = fin != nullptr ? 0 : ksplit;  // with a finishing launch nothing is left for the consumer to add up
     if ((size_t)ksplit * B * N > part_cap) return fail(TF_EINVAL, "sequential decoding: partial-tile buffer too small");
     const int ri = B <= 16 ? 0 : B <= 32 ? 1 : 2, rt = 16 << ri;
     dim3 grid((N + 127) / 128, ksplit, (B + rt - 1) / rt);
+    if (fin != nullptr && (int)(grid.x * grid.z) > tf_model::SEQ_TICKETS) return fail(TF_EINVAL, "sequential decoding: too many column tiles");
+    const seq::SeqFin fin_v = fin ? *fin : seq::SeqFin{};
+    const seq::SeqLnA lna_v = lna ? *lna : seq::SeqLnA{};
 #define TF_SEQ_TC_CASE(RTV)                                                                                              \
   if (rt == RTV)                                                                                                         \
     return launch_seq(m, cls, seq::seq_gemm_tc_kernel<RTV>, grid, 128, seq::gemm_tc_smem_bytes<RTV>(), W.map_seq,         \
                       m->map_seq_a[abuf][ri], cx.b0, B, N, kbn, cx.part, cx.step_ctr, step_off, n_steps,                 \
-                      m->seq_check_steps, m->err, (const float*)nullptr, (bf16*)nullptr);
+                      m->seq_check_steps, m->err, (const float*)nullptr, (bf16*)nullptr, fin_v, lna_v);
+#define TF_SEQ_TC_CASE8(RTV)                                                                                             \
+  if (rt == RTV && kbn == 8)                                                                                             \
+    return launch_seq(m, cls, seq::seq_gemm_tc_kernel<RTV, 8>, grid, 128, seq::gemm_tc_smem_bytes<RTV, 8>(), W.map_seq,   \
+                      m->map_seq_a[abuf][ri], cx.b0, B, N, kbn, cx.part, cx.step_ctr, step_off, n_steps,                 \
+                      m->seq_check_steps, m->err, (const float*)nullptr, (bf16*)nullptr, fin_v, lna_v);
+    TF_SEQ_TC_CASE8(16)
+    TF_SEQ_TC_CASE8(32)
+    TF_SEQ_TC_CASE8(64)
+#undef TF_SEQ_TC_CASE8
     TF_SEQ_TC_CASE(16)
     TF_SEQ_TC_CASE(32)
     TF_SEQ_TC_CASE(64)
 #undef TF_SEQ_TC_CASE
   }
+  if (fin != nullptr || lna != nullptr) return fail(TF_EINVAL, "fused step kernels need the tcgen05 step GEMM");
   const int row_tiles = (B + seq::ROWS - 1) / seq::ROWS;
   int klen = (K % 256 == 0) ? 256 : K;
   while (K / klen > 16 && K % (klen * 2) == 0) klen *= 2;  // at most 16 partial tiles
@@ -705,6 +734,10 @@ static int seq_tail(tf_model* m, const SeqCtx& cx, int g, const int* labels, con
                     m->L - 1);
 }
 
+static bool seq_chain_fused(const tf_model* m) {
+  return m->seq_fin && m->seq_use_tc && !m->seq_fuse_gelu && m->d % 128 == 0 && m->hid % 4 == 0 && m->d / 128 <= 16;
+}
+
 static int seq_update_embed(tf_model* m, const SeqCtx& cx, int g, const int* labels, const float* v, float* u, int ns,
                             int first, int step_off) {
   const BlockW& bw = m->blocks[g];
@@ -713,7 +746,7 @@ static int seq_update_embed(tf_model* m, const SeqCtx& cx, int g, const int* lab
   return launch_seq(m, KC_SEQ_UPDATE, seq::seq_update_embed_kernel, dim3(cx.B, (d + ethreads - 1) / ethreads), ethreads,
                     (int)(D * sizeof(float)), cx.part, ns, bw.b_out, cx.B, v + tok0, u + tok0, labels ? labels + cx.b0 : nullptr,
                     bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h + (size_t)cx.b0 * d, m->L, D, d, g & 1, first, cx.step_ctr, step_off,
-                    m->L - 1);
+                    m->L - 1, (seq_chain_fused(m) && ethreads == 128) ? cx.stats : (float2*)nullptr);
 }
 
 // kernels of decoding steps step_off .. step_off+count-1 relative to the chain's device step counter
@@ -726,6 +759,11 @@ static int seq_enqueue_steps(tf_model* m, const SeqCtx& cx, int g, const int* la
   const float scale = 1.0f / sqrtf((float)m->hd);
   m->cur_rows = B;
   const bool tail = seq_tail_fused(m);
+  // Fused form (opt-in, measured slower): the last K slice of a residual projection adds the finished sums to h and
+  // leaves the row statistics, the next projection normalises its own K slice of h while staging it, the MLP-up
+  // projection applies bias + GELU itself: five kernels per layer instead of eight.
+  const bool fused = seq_chain_fused(m);
+  float* hrow = m->h + (size_t)cx.b0 * d;
   for (int s = 0; s < count; ++s) {
     const float* pending_bias = nullptr;  // bias of the projection whose partial tiles are not yet in h
     int pending = 0, ns = 0;
@@ -733,6 +771,26 @@ static int seq_enqueue_steps(tf_model* m, const SeqCtx& cx, int g, const int* la
       const LayerW& lw = bw.layers[i];
       bf16* kc = reinterpret_cast<bf16*>(m->kcache) + i * layer_stride + kv0;
       bf16* vc = reinterpret_cast<bf16*>(m->vcache) + i * layer_stride + kv0;
+      if (fused) {
+        const seq::SeqLnA ln1{hrow, cx.stats, lw.ln1_g, lw.ln1_b}, ln2{hrow, cx.stats, lw.ln2_g, lw.ln2_b};
+        const seq::SeqFin fin_o{2, cx.tickets, lw.b_o, nullptr, hrow, cx.stats};
+        const seq::SeqFin fin_1{1, cx.tickets, lw.b_1, mlp, nullptr, nullptr};
+        const seq::SeqFin fin_2{2, cx.tickets, lw.b_2, nullptr, hrow, cx.stats};
+        if (i == 0 && tail) {  // layer 0's input was normalised by the fused tail of the previous step
+          TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, lw.w_qkv, s, &ns));
+        } else {  // (for layer 0 the statistics come from the embedding kernel)
+          TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, lw.w_qkv, s, &ns, nullptr, nullptr, nullptr, &ln1));
+        }
+        TF_TRY(launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, cx.part, ns, lw.b_qkv, kc, vc,
+                          att, B, L, d, heads, scale * 1.4426950408889634f, cx.step_ctr, s, L - 1));
+        int none = 0;
+        TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 1, lw.w_o, s, &none, nullptr, nullptr, &fin_o));
+        TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, lw.w_1, s, &none, nullptr, nullptr, &fin_1, &ln2));
+        TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 2, lw.w_2, s, &none, nullptr, nullptr, &fin_2));
+        pending_bias = nullptr;
+        pending = 0;
+        continue;
+      }
       // layer 0's input comes from the fused tail of the previous step (or of the block's start) when that is on
       if (!(tail && i == 0)) TF_TRY(seq_resid_ln(m, cx, pending_bias, pending, lw.ln1_g, lw.ln1_b, s));
       TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, lw.w_qkv, s, &ns));
@@ -751,8 +809,13 @@ static int seq_enqueue_steps(tf_model* m, const SeqCtx& cx, int g, const int* la
       TF_TRY(seq_tail(m, cx, g, labels, v, u, pending_bias, pending, 0, s));
       continue;
     }
-    TF_TRY(seq_resid_ln(m, cx, pending_bias, pending, bw.lnf_g, bw.lnf_b, s));
-    TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, bw.w_out, s, &ns));
+    if (fused) {  // the head normalises h itself (statistics from the last MLP-down projection)
+      const seq::SeqLnA lnf{hrow, cx.stats, bw.lnf_g, bw.lnf_b};
+      TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, bw.w_out, s, &ns, nullptr, nullptr, nullptr, &lnf));
+    } else {
+      TF_TRY(seq_resid_ln(m, cx, pending_bias, pending, bw.lnf_g, bw.lnf_b, s));
+      TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, bw.w_out, s, &ns));
+    }
     TF_TRY(seq_update_embed(m, cx, g, labels, v, u, ns, 0, s));
   }
   return check_launch("sequential step kernels");
@@ -781,6 +844,7 @@ static int seq_chain_count(const tf_model* m, int B) {
 static int run_sequential_chain(tf_model* m, const SeqCtx& cx, int g, const int* labels, const float* v, float* u) {
   const int n_steps = m->L - 1;
   CU_OK(cudaMemsetAsync(cx.step_ctr, 0, sizeof(int), m->stream));
+  CU_OK(cudaMemsetAsync(cx.tickets, 0, tf_model::SEQ_TICKETS * sizeof(int), m->stream));  // after an aborted launch
   m->cur_rows = cx.B;
   if (seq_tail_fused(m)) TF_TRY(seq_tail(m, cx, g, labels, v, u, nullptr, 0, 1, 0));
   else TF_TRY(seq_update_embed(m, cx, g, labels, v, u, 0, 1, 0));
@@ -836,6 +900,7 @@ static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* label
   if (nch == 1) {
     SeqCtx cx;
     cx.b0 = 0; cx.B = B; cx.step_ctr = m->step_ctr; cx.part = m->seq_part;
+    cx.tickets = m->seq_tickets; cx.stats = m->seq_stats;
     return run_sequential_chain(m, cx, g, labels, v, u);
   }
   // fork: the chains start once everything enqueued on the caller's stream so far has completed; join: the caller's
@@ -848,6 +913,8 @@ static int run_sequential_block_bf16(tf_model* m, int g, int B, const int* label
     cx.B = (int)((int64_t)B * (c + 1) / nch) - cx.b0;
     cx.step_ctr = m->step_ctr + 16 * c;
     cx.part = m->seq_part + (size_t)cx.b0 * m->seq_part_row_floats;
+    cx.tickets = m->seq_tickets + (size_t)c * tf_model::SEQ_TICKETS;
+    cx.stats = m->seq_stats + (size_t)c * 16 * m->cfg.max_batch;
     m->stream = m->seq_streams[c];
     cudaError_t e = cudaStreamWaitEvent(m->stream, m->seq_fork, 0);
     if (e != cudaSuccess) r = fail(TF_ECUDA, "cudaStreamWaitEvent: %s", cudaGetErrorString(e));
@@ -1474,6 +1541,9 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     if (const char* e = getenv("TARFLOW_SEQ_FUSE_GELU")) m->seq_fuse_gelu = atoi(e) != 0;
     if (const char* e = getenv("TARFLOW_SEQ_FUSE_TAIL")) m->seq_fuse_tail = atoi(e) != 0;
     CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<64, 8>()));
+    CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<32, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<32, 8>()));
+    CU_OK(cudaFuncSetAttribute(seq::seq_gemm_tc_kernel<16, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, seq::gemm_tc_smem_bytes<16, 8>()));
+    if (const char* e = getenv("TARFLOW_SEQ_KBN8")) m->seq_kbn8 = atoi(e) != 0;
     if (const char* e = getenv("TARFLOW_PAIR_GEMM")) m->use_pair_gemm = atoi(e) != 0;
     CU_OK(cudaFuncSetAttribute(attn::attention_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                attn::smem_bytes<true>()));
@@ -1492,6 +1562,10 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     CU_OK(cudaEventCreateWithFlags(&m->seq_fork, cudaEventDisableTiming));
     if (const char* e = getenv("TARFLOW_SEQ_CHAINS")) m->seq_chains_force = atoi(e);
     if (const char* e = getenv("TARFLOW_SEQ_KBN")) m->seq_kbn_force = atoi(e);
+    if (const char* e = getenv("TARFLOW_SEQ_FIN")) m->seq_fin = atoi(e) != 0;
+    TF_TRY(dev_alloc(m, &m->seq_tickets, (size_t)tf_model::MAX_CHAINS * tf_model::SEQ_TICKETS));
+    CU_OK(cudaMemset(m->seq_tickets, 0, (size_t)tf_model::MAX_CHAINS * tf_model::SEQ_TICKETS * sizeof(int)));
+    TF_TRY(dev_alloc(m, &m->seq_stats, (size_t)tf_model::MAX_CHAINS * 16 * B));
     if (const char* e = getenv("TARFLOW_SWEEP_GRAPH_ROWS")) m->sweep_graph_rows = atoll(e);
   }
   CU_OK(cudaDeviceSynchronize());

@@ -320,17 +320,20 @@ def test_bf16_two_term_attention_paths_agree(monkeypatch):
 
 @pytest.mark.gpu
 def test_bf16_optional_sequential_paths_agree(monkeypatch):
-    """Sequential decoding: fused bias + GELU, the mma.sync step GEMM and the unfused step tail give the default path's result."""
+    """Sequential decoding: fused bias + GELU, the mma.sync step GEMM, the unfused step tail, the five-kernel layer chain and a
+    single sample chain give the default path's result."""
     cfg = synth.config("cfg2", n_blocks=1, n_layers=2)
-    z = synth.make_latents(cfg, 19, B=5)
+    z = synth.make_latents(cfg, 19, B=40)      # 40 samples: two chains of 20 by default
     outs = {}
     for name, env in (("default", {}), ("gelu_fused", {"TARFLOW_SEQ_FUSE_GELU": "1"}), ("mma_sync", {"TARFLOW_SEQ_MMA": "1"}),
-                      ("tail_kernels", {"TARFLOW_SEQ_FUSE_TAIL": "0"})):
-        for k in ("TARFLOW_SEQ_FUSE_GELU", "TARFLOW_SEQ_MMA", "TARFLOW_SEQ_FUSE_TAIL"):
+                      ("tail_kernels", {"TARFLOW_SEQ_FUSE_TAIL": "0"}), ("fused_chain", {"TARFLOW_SEQ_FIN": "1"}),
+                      ("fused_chain_unfused_tail", {"TARFLOW_SEQ_FIN": "1", "TARFLOW_SEQ_FUSE_TAIL": "0"}),
+                      ("one_chain", {"TARFLOW_SEQ_CHAINS": "1"})):
+        for k in ("TARFLOW_SEQ_FUSE_GELU", "TARFLOW_SEQ_MMA", "TARFLOW_SEQ_FUSE_TAIL", "TARFLOW_SEQ_FIN", "TARFLOW_SEQ_CHAINS"):
             monkeypatch.delenv(k, raising=False)
         for k, v in env.items():
             monkeypatch.setenv(k, v)
-        with Model(cfg, max_batch=5) as m:      # the switches are read when the model is loaded
+        with Model(cfg, max_batch=40) as m:     # the switches are read when the model is loaded
             outs[name], _, _, rc = m.inverse(z, None, [0], -1.0, 3)
             assert rc == 0 and np.isfinite(outs[name]).all()
     xo, _ = O.model_inverse(synth.make_weights(cfg), z, None, cfg, [0], -1.0, 3)
@@ -339,3 +342,6 @@ def test_bf16_optional_sequential_paths_agree(monkeypatch):
     assert rel_l2(outs["gelu_fused"], outs["default"]) <= 5e-3
     assert rel_l2(outs["mma_sync"], outs["default"]) <= 5e-3
     assert rel_l2(outs["tail_kernels"], outs["default"]) <= 5e-3
+    assert rel_l2(outs["fused_chain"], outs["default"]) <= 5e-3
+    assert rel_l2(outs["fused_chain_unfused_tail"], outs["default"]) <= 5e-3
+    assert np.array_equal(outs["one_chain"], outs["default"])     # a sample's arithmetic does not depend on the chain split
