@@ -43,9 +43,11 @@ UNIT = "samples/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 L2_BYTES = 126e6
 
-# dram bytes per launch (read + write) of a kernel class from the committed ncu capture of that class, scaled to
-# a full launch of the workload; None = no capture of the current kernel.  {workload: {class: bytes}}
-NCU_TRAFFIC: dict = {}
+# dram bytes per launch (read + write) of a kernel class from the committed ncu capture of that class
+# (profiles/gemm_tc2_kernel_cfg3_sweep.md: one single-term launch over the full batch of 16 384 rows; the live class
+# also holds two-term launches and launches over fewer rows); None = no capture of the current kernel.
+# {workload: {class: bytes}}
+NCU_TRAFFIC: dict = {"cfg3": {"gemm_qkv": 89.4e6, "gemm_out": 112.5e6, "gemm_mlp_up": 123.4e6, "gemm_mlp_down": 255.1e6}}
 
 
 def peaks():

@@ -54,3 +54,18 @@ def test_class_work_gemm_flops_and_bounds(bench):
     assert w["attention"][1] == 2.0 * 1024 * 256
     assert w["seq_block"][0] == "hbm" and w["seq_block"][2] == bench.seq_block_bytes(cfg, 256, 48, 64)[0]
     assert bench.class_work(synth.config("cfg1"), 64, 12, 4)["gemm_qkv"][0] == "alu"
+
+
+def test_reference_arm_prints_the_contract_line_on_cpu():
+    """`bench.py --impl reference` needs no GPU: it times the oracle on the host cores and prints one JSON line."""
+    import json
+    import subprocess
+    import sys
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "cfg1",
+                          "--steps", "1", "--warmup", "0"], capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["unit"] == "samples/s" and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["e2e"] == {"value": line["value"], "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    assert line["higher_is_better"] is True and line["gpu_launches"] == 0 and "workload" in line["config"]
