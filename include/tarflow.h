@@ -324,6 +324,14 @@ int tf_trace_read_l2(tf_model* m, int32_t block, int32_t B, float* l2_host, int3
  */
 int tf_selftest_wait_timeout(tf_model* m, int32_t limit_us, void* cuda_stream);
 
+/*
+ * tf_debug_check_guards -- every device buffer of a model lies between two 256-byte guard regions filled with a
+ * fixed pattern when the model is loaded.  This call counts, on the device, the guard words that no longer hold the
+ * pattern and returns that number (0 = no kernel has written outside its buffer since the model was loaded;
+ * negative = error).  It synchronises the stream.  A substitute for a memory checker where none can be run.
+ */
+int64_t tf_debug_check_guards(tf_model* m, void* cuda_stream);
+
 /* tf_device_bytes -- device memory owned by the model (weights + workspace + KV cache), bytes. */
 int64_t tf_device_bytes(tf_model* m);
 

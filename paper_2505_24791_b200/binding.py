@@ -74,6 +74,8 @@ def lib():
         L.tf_trace_enable.argtypes = [vp, i32]
         L.tf_trace_read.argtypes = [vp, vp, vp, vp, vp, i32]
         L.tf_selftest_wait_timeout.argtypes = [vp, i32, vp]
+        L.tf_debug_check_guards.argtypes = [vp, vp]
+        L.tf_debug_check_guards.restype = C.c_int64
         L.tf_launch_count.argtypes = [vp]
         L.tf_launch_count.restype = C.c_int64
         L.tf_device_bytes.argtypes = [vp]
@@ -250,6 +252,14 @@ def tf_trace_read(m, cap=4096):
 
 def tf_selftest_wait_timeout(m, limit_us, stream=None):
     return _check(lib().tf_selftest_wait_timeout(m, int(limit_us), _stream(stream)))
+
+
+def tf_debug_check_guards(m, stream=None):
+    """-> number of overwritten guard words around the model's device buffers (0 = clean)."""
+    n = lib().tf_debug_check_guards(m, _stream(stream))
+    if n < 0:
+        _check(int(n))
+    return int(n)
 
 
 def tf_launch_count(m):

@@ -892,6 +892,12 @@ __global__ void labels_check_kernel(const int* __restrict__ labels, int* __restr
   out[b] = y;
 }
 
+// One CTA per guard region (blockDim.x words): counts the words that no longer hold the fill pattern.
+__global__ void guard_check_kernel(unsigned char* const* __restrict__ guards, int* __restrict__ count, unsigned pattern) {
+  const unsigned w = reinterpret_cast<const unsigned*>(guards[blockIdx.x])[threadIdx.x];
+  if (w != pattern) atomicAdd(count, 1);
+}
+
 __global__ void fill_int_kernel(int* p, int n, int v) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) p[i] = v;

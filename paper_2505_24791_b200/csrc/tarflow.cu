@@ -151,6 +151,9 @@ struct tf_model {
   int num_sms = 148;
   std::vector<BlockW> blocks;
   std::vector<void*> allocs;
+  std::vector<unsigned char*> guards;   // start of every guard region (two per allocation)
+  unsigned char** guards_dev = nullptr; // the same list on the device, built by the first check
+  int* guard_count = nullptr;
   int64_t device_bytes = 0;
   // workspace
   float *seq_a = nullptr, *seq_b = nullptr, *h = nullptr, *o = nullptr, *maxdiff = nullptr;
@@ -332,19 +335,30 @@ static int current_device() {
   return dev;
 }
 
+// Every device buffer of a model sits between two guard regions of GUARD_BYTES filled with a fixed pattern.  A kernel
+// that writes outside its buffer (the kind of fault a memory checker would report) damages a guard instead of a
+// neighbouring buffer, and tf_debug_check_guards counts the damaged words after any call.
+constexpr size_t GUARD_BYTES = 256;
+constexpr unsigned char GUARD_BYTE = 0xA5;
+
 template <class T>
 static int dev_alloc(tf_model* m, T** p, size_t count) {
   size_t bytes = ((count * sizeof(T)) + 255) & ~(size_t)255;
   if (bytes == 0) bytes = 256;
   void* q = nullptr;
-  cudaError_t e = cudaMalloc(&q, bytes);
+  cudaError_t e = cudaMalloc(&q, bytes + 2 * GUARD_BYTES);
   if (e != cudaSuccess) {
     cudaGetLastError();
     return fail(TF_ENOMEM, "cudaMalloc(%zu bytes) failed: %s", bytes, cudaGetErrorString(e));
   }
   m->allocs.push_back(q);
-  m->device_bytes += (int64_t)bytes;
-  *p = reinterpret_cast<T*>(q);
+  unsigned char* base = reinterpret_cast<unsigned char*>(q);
+  CU_OK(cudaMemset(base, GUARD_BYTE, GUARD_BYTES));
+  CU_OK(cudaMemset(base + GUARD_BYTES + bytes, GUARD_BYTE, GUARD_BYTES));
+  m->guards.push_back(base);
+  m->guards.push_back(base + GUARD_BYTES + bytes);
+  m->device_bytes += (int64_t)(bytes + 2 * GUARD_BYTES);
+  *p = reinterpret_cast<T*>(base + GUARD_BYTES);
   return TF_OK;
 }
 
@@ -1749,6 +1763,8 @@ void tf_free(tf_model* m) {
   }
   if (m->seq_fork) cudaEventDestroy(m->seq_fork);
   for (void* p : m->allocs) cudaFree(p);
+  if (m->guards_dev) cudaFree(m->guards_dev);
+  if (m->guard_count) cudaFree(m->guard_count);
   if (m->ctrl_host) cudaFreeHost(m->ctrl_host);
   delete m;
 }
@@ -2038,6 +2054,26 @@ int tf_selftest_wait_timeout(tf_model* m, int32_t limit_us, void* cuda_stream) {
   LAUNCH(m, KC_CTRL, tc::wait_selftest_kernel, 1, 32, 0, m->err, (unsigned long long)limit_us * 1000ull);
   TF_TRY(check_launch("wait_selftest_kernel"));
   return sync_check(m);
+}
+
+int64_t tf_debug_check_guards(tf_model* m, void* cuda_stream) {
+  g_err[0] = 0;
+  if (!m) return fail(TF_EINVAL, "model is NULL");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const int n = (int)m->guards.size();
+  if (!m->guards_dev) {  // plain cudaMalloc: these two are not themselves guarded
+    CU_OK(cudaMalloc(&m->guards_dev, (size_t)n * sizeof(unsigned char*)));
+    CU_OK(cudaMalloc(&m->guard_count, sizeof(int)));
+    CU_OK(cudaMemcpy(m->guards_dev, m->guards.data(), (size_t)n * sizeof(unsigned char*), cudaMemcpyHostToDevice));
+  }
+  CU_OK(cudaMemsetAsync(m->guard_count, 0, sizeof(int), st));
+  guard_check_kernel<<<n, (int)(GUARD_BYTES / 4), 0, st>>>(m->guards_dev, m->guard_count, 0x01010101u * GUARD_BYTE);
+  TF_TRY(check_launch("guard_check_kernel"));
+  int bad = 0;
+  CU_OK(cudaMemcpyAsync(&bad, m->guard_count, sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU_OK(cudaStreamSynchronize(st));
+  if (bad != 0) fail(TF_OK, "%d guard words next to the model's device buffers were overwritten", bad);
+  return bad;
 }
 
 int tf_profile_enable(tf_model* m, int32_t on) {

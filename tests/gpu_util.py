@@ -17,8 +17,12 @@ class Model:
 
     def close(self):
         if self.m is not None:
-            binding.tf_free(self.m)
-            self.m = None
+            try:    # no kernel of any call on this model wrote outside its buffer
+                damaged = binding.tf_debug_check_guards(self.m)
+            finally:
+                binding.tf_free(self.m)
+                self.m = None
+            assert damaged == 0, f"{damaged} guard words around the model's device buffers were overwritten"
 
     def __enter__(self):
         return self

@@ -23,7 +23,11 @@ class Maf:
         return self
 
     def __exit__(self, *a):
-        binding.tf_free(self.m)
+        try:
+            damaged = binding.tf_debug_check_guards(self.m)
+        finally:
+            binding.tf_free(self.m)
+        assert damaged == 0, f"{damaged} guard words around the model's device buffers were overwritten"
 
     def jacobi(self, z, tau, max_iters, init_mode=0):
         B = z.shape[0]
@@ -153,3 +157,21 @@ def test_bf16_ragged_dimension_sequential_forward_and_thresholds():
         zo, ldo = MO.model_forward(m.blocks, xso)
         assert rel_l2(zg, zo) <= 2e-2 and np.abs(zg - zo).max() <= 5e-2
         assert np.abs(ld - ldo).max() <= 2e-2 * max(np.abs(ldo).max(), np.sqrt(m.D * m.K) * 0.1)
+
+
+def test_bf16_mnist_shape_ragged_k_and_head_width():
+    """784 dimensions (12.25 k slabs in the first layer: the last one is zero-filled by the tensor map; 1568 head
+    columns, not a multiple of the 256-column pair tile), hidden width 1024, 2 layers, 100 samples."""
+    cfg = synth.maf_config("maf_mnist", n_blocks=2)
+    B = cfg["B"]
+    with Maf(cfg, B) as m:
+        z = synth.make_maf_latents(cfg, 23, B=B)
+        x, ib, its, rc = m.jacobi(z, cfg["tau"], m.D + 1)
+        assert rc == 0 and np.isfinite(x).all() and (its >= 2).all()
+        pick = [0, 1, 57, B - 1]
+        xo, ito = MO.model_inverse(m.blocks, z[pick], cfg["tau"], m.D + 1)
+        assert rel_l2(x[pick], xo) <= 2e-2 and np.abs(x[pick] - xo).max() <= 5e-2
+        assert np.abs(its[:, pick] - ito).max() <= 1
+        xf, _, itf, rc = m.jacobi(z[:3], -1.0, 5)                   # fixed sweeps: the same iterate as the oracle's
+        xfo, _ = MO.model_inverse(m.blocks, z[:3], -1.0, 5)
+        assert rc == 0 and rel_l2(xf, xfo) <= 2e-2 and np.abs(xf - xfo).max() <= 5e-2
