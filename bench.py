@@ -254,6 +254,7 @@ def run_reference(args, cfg, L, rank):
     bs = cpu_sample_size(args.workload)
     policy = [0] + [1] * (cfg["n_blocks"] - 1)
     times = []
+    args.warmup = min(args.warmup, 1)   # a CPU run needs no more than one untimed step; every step costs tens of seconds
     for i in range(args.warmup + args.steps):
         z = synth.make_latents(cfg, 4000 + i, B=bs)
         lab = synth.make_labels(cfg, B=bs)
