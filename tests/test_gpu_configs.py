@@ -206,3 +206,24 @@ def test_bounded_wait_runs_out_is_reported_once_and_model_recovers(sweep_model):
     assert rc == 0 and np.array_equal(x_before, x_after)
     zf, ld = m.forward(x_after, lab)
     assert np.isfinite(zf).all() and np.isfinite(ld).all()
+
+
+# ---------------------------------------------------------------- the long-sequence configuration at its full size
+def test_long_sequence_full_size_properties():
+    """cfg4 as the benchmark runs it (8 blocks x 8 layers, 1024 tokens, batch 16, selective policy, tau 1e-3).  The
+    oracle needs six minutes per sample here, so the checks are properties that hold at any size: the forward
+    direction applied to the sample returns the latent (Eq. 4 and Eq. 5 are mutual inverses, through all 64 layers),
+    the all-sequential sample agrees with the selective one to a few tau, sweep counts lie in Prop. 3.2's range."""
+    cfg = synth.config("cfg4")
+    B = cfg["B"]
+    policy = [0] + [1] * (cfg["n_blocks"] - 1)
+    with Model(cfg, max_batch=B) as m:
+        z = synth.make_latents(cfg, 1000, B=B)
+        x, ib, its, rc = m.inverse(z, None, policy, cfg["tau"], m.L + 1)
+        assert rc == 0 and np.isfinite(x).all()
+        assert (its[0] == m.L - 1).all() and (its[1:] >= 2).all() and (its[1:] <= 12).all()
+        zr, ld = m.forward(x, None)
+        assert np.isfinite(ld).all()
+        assert rel_l2(zr, z.astype(np.float64)) <= BF16_REL_L2 and np.abs(zr - z).max() <= 0.15
+        xs = m.inverse_sequential(z[:4], None)
+        assert rel_l2(x[:4], xs) <= 5e-3 and np.abs(x[:4] - xs).max() <= 5e-2
