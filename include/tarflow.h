@@ -36,7 +36,9 @@
  *     step tail (final LayerNorm, head, update, embedding, next LayerNorm) off or on whatever the head's size.  Sweeps: TARFLOW_PAIR_GEMM=0 runs the projections with
  *     one CTA per 128x256 tile instead of 2-CTA pairs; TARFLOW_ATTN_TC=0 runs attention on the mma.sync kernel
  *     instead of the tcgen05 one, TARFLOW_ATTN_TC_SPLIT=0 does so for two-term operands only.  TARFLOW_SEQ_CHAINS=1|2|4
- *     sets how many sample chains decode a sequential block side by side (default: 2 from 32 samples up);
+ *     sets how many sample chains decode a sequential block side by side (default: 2 from 32 samples up),
+ *     TARFLOW_SEQ_ATTN_THREADS=128|256 the CTA size of the decoding step's attention (default: 128 when there are
+ *     more (sample, head) pairs than three 256-thread CTAs per SM hold at once);
  *     TARFLOW_SEQ_FIN=1 lets the last K slice of a step projection finish its tile (residual add or bias + GELU) and
  *     the next projection normalise its own operand slice, five kernels per layer instead of eight (measured slower
  *     than the default chain), TARFLOW_SEQ_KBN8=0 keeps such launches at four k slabs per CTA;

@@ -540,12 +540,16 @@ seq_resid_ln_kernel(float* __restrict__ h, const float* __restrict__ part, const
 // Attention of the new token of one (sample, head).  The CTA first finishes that token's q, k, v (64
 // channels each) from the QKV projection's partial tiles (+ bias), appends k and v to the cache
 // (layout [B][heads][L][64] bf16: the rows of one (sample, head) are contiguous) and keeps q in fp32.
-// Then a single query against rows 0..t: 8 lanes share a key (16 bytes = 8 channels each); the 32 lane
-// groups of the CTA take keys j = group (mod 32), four keys per round with the K and V rows of all four in
+// Then a single query against rows 0..t: 8 lanes share a key (16 bytes = 8 channels each); the NT / 8 lane
+// groups of the CTA take keys j = group (mod NT / 8), four keys per round with the K and V rows of all four in
 // flight together, and keep an online softmax (running max, sum, output) per group in fp32; the groups
 // are merged through shared memory at the end.  Row t itself is taken from shared memory.  out: [B, d].
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
+// NT threads per CTA = NT / 8 lane groups: 256 for few (sample, head) pairs with long caches, 128 (at most 64
+// registers, eight CTAs per SM) when there are more pairs than three 256-thread CTAs per SM can hold at once, so that
+// the launch is one wave instead of three.
+template <int NT>
+__global__ void __launch_bounds__(NT, NT == 128 ? 8 : 3)
 seq_attention_kernel(const float* __restrict__ part, int nsplit, const float* __restrict__ bias, bf16* __restrict__ kc,
                      bf16* __restrict__ vc, bf16* __restrict__ out, int B, int L, int d, int heads, float scale_log2e,
                      const int* __restrict__ step_base, int step_off, int n_steps) {
@@ -553,7 +557,8 @@ seq_attention_kernel(const float* __restrict__ part, int nsplit, const float* __
   pdl_wait();
   const int t = *step_base + step_off;
   if (t >= n_steps) return;
-  __shared__ float s_m[32], s_l[32], s_o[32][HD];
+  constexpr int NG = NT / 8;  // lane groups
+  __shared__ float s_m[NG], s_l[NG], s_o[NG][HD];
   __shared__ __align__(16) float s_q[HD];
   __shared__ __align__(16) bf16 s_k[HD], s_v[HD];
   const int head = blockIdx.x, b = blockIdx.y;
@@ -584,11 +589,11 @@ seq_attention_kernel(const float* __restrict__ part, int nsplit, const float* __
   float m_run = -INFINITY, l_run = 0.f, o[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) o[i] = 0.f;
-  for (int j0 = 0; j0 < nk; j0 += 128) {
+  for (int j0 = 0; j0 < nk; j0 += 4 * NG) {
     uint4 kv[4], vv[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const int j = j0 + u * 32 + grp;
+      const int j = j0 + u * NG + grp;
       if (j < t) {
         kv[u] = __ldcg(reinterpret_cast<const uint4*>(kr + (size_t)j * HD));
         vv[u] = __ldcg(reinterpret_cast<const uint4*>(vr + (size_t)j * HD));
@@ -614,7 +619,7 @@ seq_attention_kernel(const float* __restrict__ part, int nsplit, const float* __
       s += __shfl_xor_sync(0xffffffffu, s, 1);
       s += __shfl_xor_sync(0xffffffffu, s, 2);
       s += __shfl_xor_sync(0xffffffffu, s, 4);
-      sc[u] = (j0 + u * 32 + grp) < nk ? s : -INFINITY;
+      sc[u] = (j0 + u * NG + grp) < nk ? s : -INFINITY;
     }
     const float m_new = fmaxf(fmaxf(m_run, fmaxf(sc[0], sc[1])), fmaxf(sc[2], sc[3]));
     if (m_new > -INFINITY) {  // this group has seen at least one key
@@ -644,10 +649,10 @@ seq_attention_kernel(const float* __restrict__ part, int nsplit, const float* __
   if (threadIdx.x < HD) {
     float mx = s_m[0];  // group 0 always holds key 0
 #pragma unroll 8
-    for (int gI = 1; gI < 32; ++gI) mx = fmaxf(mx, s_m[gI]);
+    for (int gI = 1; gI < NG; ++gI) mx = fmaxf(mx, s_m[gI]);
     float num = 0.f, den = 0.f;
 #pragma unroll 8
-    for (int gI = 0; gI < 32; ++gI) {
+    for (int gI = 0; gI < NG; ++gI) {
       const float w = exp2f(s_m[gI] - mx);  // 0 for a group without keys
       num = fmaf(w, s_o[gI][threadIdx.x], num);
       den = fmaf(w, s_l[gI], den);

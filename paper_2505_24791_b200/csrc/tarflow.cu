@@ -204,6 +204,7 @@ struct tf_model {
   // fence + ticket + fence of the last arriver and its one-CTA reduction cost more than the kernel boundary and the
   // many-CTA consumer kernel they replace.
   bool seq_fin = false;
+  int seq_attn_threads = 0;  // TARFLOW_SEQ_ATTN_THREADS=128|256: CTA size of the step attention (0 = by the number of CTAs)
   int seq_kbn_force = 0;     // TARFLOW_SEQ_KBN
   // Jacobi sweeps over few rows are replayed from graphs: one per (block, single-term slots, two-term slots, buffers)
   std::map<std::tuple<int, int, int, const void*, const void*, const void*, const void*>, SeqGraph> sweep_graphs;
@@ -763,14 +764,26 @@ static int seq_update_embed(tf_model* m, const SeqCtx& cx, int g, const int* lab
                     m->L - 1, (seq_chain_fused(m) && ethreads == 128) ? cx.stats : (float2*)nullptr);
 }
 
+// attention of the new token of every (sample, head) of the chain over its cache rows
+static int seq_attention(tf_model* m, const SeqCtx& cx, int ns, const float* b_qkv, bf16* kc, bf16* vc, bf16* att, int step_off) {
+  const int heads = m->cfg.n_heads, L = m->L;
+  const float sl2 = 1.4426950408889634f / sqrtf((float)m->hd);
+  // more (sample, head) pairs than three 256-thread CTAs per SM hold at once: the 128-thread form runs as one wave
+  const bool small = m->seq_attn_threads == 128 || (m->seq_attn_threads == 0 && heads * cx.B > 3 * m->num_sms);
+  if (small)
+    return launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel<128>, dim3(heads, cx.B), 128, 0, cx.part, ns, b_qkv, kc, vc, att,
+                      cx.B, L, m->d, heads, sl2, cx.step_ctr, step_off, L - 1);
+  return launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel<256>, dim3(heads, cx.B), 256, 0, cx.part, ns, b_qkv, kc, vc, att,
+                    cx.B, L, m->d, heads, sl2, cx.step_ctr, step_off, L - 1);
+}
+
 // kernels of decoding steps step_off .. step_off+count-1 relative to the chain's device step counter
 static int seq_enqueue_steps(tf_model* m, const SeqCtx& cx, int g, const int* labels, const float* v, float* u, int count) {
   const BlockW& bw = m->blocks[g];
-  const int L = m->L, d = m->d, nl = m->cfg.n_layers, heads = m->cfg.n_heads, B = cx.B;
+  const int L = m->L, d = m->d, nl = m->cfg.n_layers, B = cx.B;
   bf16* att = reinterpret_cast<bf16*>(m->att) + (size_t)cx.b0 * d;
   bf16* mlp = reinterpret_cast<bf16*>(m->mlp) + (size_t)cx.b0 * m->hid;
   const size_t layer_stride = (size_t)m->cfg.max_batch * L * d, kv0 = (size_t)cx.b0 * L * d;
-  const float scale = 1.0f / sqrtf((float)m->hd);
   m->cur_rows = B;
   const bool tail = seq_tail_fused(m);
   // Fused form (opt-in, measured slower): the last K slice of a residual projection adds the finished sums to h and
@@ -795,8 +808,7 @@ static int seq_enqueue_steps(tf_model* m, const SeqCtx& cx, int g, const int* la
         } else {  // (for layer 0 the statistics come from the embedding kernel)
           TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, lw.w_qkv, s, &ns, nullptr, nullptr, nullptr, &ln1));
         }
-        TF_TRY(launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, cx.part, ns, lw.b_qkv, kc, vc,
-                          att, B, L, d, heads, scale * 1.4426950408889634f, cx.step_ctr, s, L - 1));
+        TF_TRY(seq_attention(m, cx, ns, lw.b_qkv, kc, vc, att, s));
         int none = 0;
         TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 1, lw.w_o, s, &none, nullptr, nullptr, &fin_o));
         TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, lw.w_1, s, &none, nullptr, nullptr, &fin_1, &ln2));
@@ -808,8 +820,7 @@ static int seq_enqueue_steps(tf_model* m, const SeqCtx& cx, int g, const int* la
       // layer 0's input comes from the fused tail of the previous step (or of the block's start) when that is on
       if (!(tail && i == 0)) TF_TRY(seq_resid_ln(m, cx, pending_bias, pending, lw.ln1_g, lw.ln1_b, s));
       TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, lw.w_qkv, s, &ns));
-      TF_TRY(launch_seq(m, KC_SEQ_ATTN, seq::seq_attention_kernel, dim3(heads, B), 256, 0, cx.part, ns, lw.b_qkv, kc, vc,
-                        att, B, L, d, heads, scale * 1.4426950408889634f, cx.step_ctr, s, L - 1));
+      TF_TRY(seq_attention(m, cx, ns, lw.b_qkv, kc, vc, att, s));
       TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 1, lw.w_o, s, &pending));
       TF_TRY(seq_resid_ln(m, cx, lw.b_o, pending, lw.ln2_g, lw.ln2_b, s));
       TF_TRY(seq_gemm(m, cx, KC_SEQ_GEMM, 0, lw.w_1, s, &ns, lw.b_1, reinterpret_cast<bf16*>(m->mlp)));
@@ -843,8 +854,8 @@ static int seq_unroll(int n_steps) {  // steps per graph: a divisor of n_steps c
 }
 
 // How many chains decode a batch of B samples side by side.  Measured (one block, ms): width 512, 4 layers, batch 64:
-// 31.5 / 27.4 / 27.5 with 1 / 2 / 4 chains; width 1024, 8 layers, batch 64: 85.5 / 81.0 / 84.1; 1024 tokens, batch 16:
-// 280 / 301 / 338.  A chain of 16 samples takes as long as one of 64: the block's time is the length of the dependent
+// 34.8 / 28.3 / 28.4 with 1 / 2 / 4 chains; width 1024, 8 layers, batch 64: 82.0 / 76.0 / 86.1; 1024 tokens, batch 16:
+// 287 / 303 / 359.  A chain of 16 samples takes as long as one of 64: the block's time is the length of the dependent
 // kernel chain, and a split only hides the small throughput-bound part (attention over the cache, partial sums), while
 // every chain streams the weights again.  So: two chains from 32 samples up, otherwise one.
 static int seq_chain_count(const tf_model* m, int B) {
@@ -1577,6 +1588,7 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     if (const char* e = getenv("TARFLOW_SEQ_CHAINS")) m->seq_chains_force = atoi(e);
     if (const char* e = getenv("TARFLOW_SEQ_KBN")) m->seq_kbn_force = atoi(e);
     if (const char* e = getenv("TARFLOW_SEQ_FIN")) m->seq_fin = atoi(e) != 0;
+    if (const char* e = getenv("TARFLOW_SEQ_ATTN_THREADS")) m->seq_attn_threads = atoi(e);
     TF_TRY(dev_alloc(m, &m->seq_tickets, (size_t)tf_model::MAX_CHAINS * tf_model::SEQ_TICKETS));
     CU_OK(cudaMemset(m->seq_tickets, 0, (size_t)tf_model::MAX_CHAINS * tf_model::SEQ_TICKETS * sizeof(int)));
     TF_TRY(dev_alloc(m, &m->seq_stats, (size_t)tf_model::MAX_CHAINS * 16 * B));
