@@ -793,9 +793,34 @@ __global__ void __launch_bounds__(256) l2_distance_kernel(const float* __restric
 }
 
 // MLP-based flow: input of the first layer, a[s, :] = T(u[idx[s], :]) (+ the second bf16 term when a_lo != null).
+// Four values per thread when D % 4 == 0 (16-byte loads, 8- or 16-byte stores), else one.
 template <class T>
 __global__ void maf_cast_rows_kernel(const float* __restrict__ u, const int* __restrict__ idx, T* __restrict__ a,
                                      T* __restrict__ a_lo, int n_slots, int D) {
+  if ((D & 3) == 0) {
+    const int d4 = D >> 2;
+    const size_t total = (size_t)n_slots * d4;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+      const int s = (int)(i / d4), c4 = (int)(i - (size_t)s * d4);
+      const float4 x = *(reinterpret_cast<const float4*>(u + (size_t)(idx ? idx[s] : s) * D) + c4);
+      const float xs[4] = {x.x, x.y, x.z, x.w};
+      T hi[4], lo[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        hi[k] = from_f32<T>(xs[k]);
+        lo[k] = from_f32<T>(xs[k] - to_f32(hi[k]));
+      }
+      T* dst = a + (size_t)s * D + 4 * c4;
+      if constexpr (sizeof(T) == 2) {
+        *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(hi);
+        if (a_lo != nullptr) *reinterpret_cast<uint2*>(a_lo + (size_t)s * D + 4 * c4) = *reinterpret_cast<const uint2*>(lo);
+      } else {
+        *reinterpret_cast<float4*>(dst) = *reinterpret_cast<const float4*>(hi);
+        if (a_lo != nullptr) *reinterpret_cast<float4*>(a_lo + (size_t)s * D + 4 * c4) = *reinterpret_cast<const float4*>(lo);
+      }
+    }
+    return;
+  }
   const size_t total = (size_t)n_slots * D;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const int s = (int)(i / D), c = (int)(i - (size_t)s * D);

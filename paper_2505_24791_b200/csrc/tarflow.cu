@@ -1262,7 +1262,7 @@ static int maf_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
   T* h1_lo = hp ? reinterpret_cast<T*>(m->maf_h1_lo) : nullptr;
   T* h2_lo = hp ? reinterpret_cast<T*>(m->maf_h2_lo) : nullptr;
   m->cur_rows = M;
-  int cb = (int)(((size_t)M * D + 255) / 256);
+  int cb = (int)(((size_t)M * ((D & 3) == 0 ? D / 4 : D) + 255) / 256);
   if (cb > 148 * 16) cb = 148 * 16;
   LAUNCH(m, KC_EMBED, (maf_cast_rows_kernel<T>), cb, 256, 0, u_src, idx, a0, a0_lo, M, D);
   TF_TRY(check_launch("maf_cast_rows_kernel"));
