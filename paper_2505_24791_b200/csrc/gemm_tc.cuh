@@ -207,7 +207,8 @@ struct SmemLayout {
 template <int BN, int STAGES, class Epi>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_a_lo,
-               const __grid_constant__ CUtensorMap map_w, int M, int N, int K, int split, Epi epi, int* err) {
+               const __grid_constant__ CUtensorMap map_w, int M, int N, int K, int split, Epi epi, int* err,
+               int ksplit, int part_rows) {
   static_assert(SmemLayout<BN, STAGES>::TILE_BIAS_OFFSET + 1024 <= SmemLayout<BN, STAGES>::STAGE_OUT_OFFSET +
                 SmemLayout<BN, STAGES>::STAGE_OUT_BYTES, "bias tile must fit behind the store boxes");
   using SL = SmemLayout<BN, STAGES>;
@@ -225,11 +226,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN;
-  const int num_tiles_all = tiles_m * tiles_n;
+  // ksplit > 1 (bulk-store epilogues only): every output tile is computed ksplit times, each over its own range of
+  // k slabs, and slice s stores its partial tile part_rows * s rows further down; the consumer adds the slices in
+  // index order.  Tile index = (m tile, n tile, slice) with the slice fastest.
+  const int num_tiles_all = tiles_m * tiles_n * ksplit;
   // split != 0: A is an error-compensated pair (hi + lo); the K loop runs over [A_hi | A_lo] against
   // [W | W], i.e. both products accumulate into the same TMEM tile.
   const int kb_per_pass = (K + BK - 1) / BK;
-  const int kblocks = split ? 2 * kb_per_pass : kb_per_pass;
+  auto slab_begin = [&](int slice) { return (int)((long long)kb_per_pass * slice / ksplit); };
   constexpr uint32_t TMEM_COLS = 2 * BN;  // two accumulator buffers (power of two >= 32)
 
   if (threadIdx.x == 0) {
@@ -265,13 +269,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+        const int mn = tile / ksplit, slice = tile - mn * ksplit;
+        const int m0 = (mn / tiles_n) * BM, n0 = (mn % tiles_n) * BN;
+        const int kb0 = slab_begin(slice), nkb = slab_begin(slice + 1) - kb0;
+        const int kblocks = split ? 2 * nkb : nkb;
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, err, TFERR_WAIT_EMPTY)) { ok = false; break; }
           mbar_arrive_expect_tx(full_bar(stage), SL::STAGE_BYTES);
           const uint32_t sa = smem_base + stage * SL::STAGE_BYTES;
-          const int kk = (kb >= kb_per_pass ? kb - kb_per_pass : kb) * BK;
-          tma_load_2d(sa, kb >= kb_per_pass ? &map_a_lo : &map_a, kk, m0, full_bar(stage));
+          const int kk = (kb0 + (kb >= nkb ? kb - nkb : kb)) * BK;
+          tma_load_2d(sa, kb >= nkb ? &map_a_lo : &map_a, kk, m0, full_bar(stage));
           tma_load_2d(sa + SL::A_BYTES, &map_w, kk, n0, full_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -291,6 +298,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, err, TFERR_WAIT_TMEM_EMPTY)) { ok = false; break; }
         tcgen05_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
+        const int slice = tile % ksplit;
+        const int kblocks = (split ? 2 : 1) * (slab_begin(slice + 1) - slab_begin(slice));
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, err, TFERR_WAIT_FULL)) { ok = false; break; }
           tcgen05_fence_after();
@@ -326,7 +335,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint32_t box_addr = smem_u32(box);
       float* tile_bias = reinterpret_cast<float*>(smem + SL::TILE_BIAS_OFFSET);
       for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
-        const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+        const int mn = tile / ksplit, slice = tile - mn * ksplit;
+        const int m0 = (mn / tiles_n) * BM, n0 = (mn % tiles_n) * BN;
         const int acc = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1;
         // the tile's biases, once, while the mainloop still runs
@@ -352,7 +362,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
           for (int g = 0; g < NCH / CPG; ++g) {
             const int cl = (cgroup * NCH + g * CPG) * 32;  // first column of the box inside the tile
-            if (n0 + cl < N) epi.template tma_box<CPG>(v[g * CPG], v[g * CPG + CPG - 1], tile_bias + cl, n0 + cl, row0, box, box_addr, lane);
+            if (n0 + cl < N)
+              epi.template tma_box<CPG>(v[g * CPG], v[g * CPG + CPG - 1], tile_bias + cl, n0 + cl, row0 + slice * part_rows, box,
+                                        box_addr, lane);
           }
         }
       }

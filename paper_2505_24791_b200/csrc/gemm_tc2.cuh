@@ -86,7 +86,8 @@ __host__ __device__ constexpr uint32_t make_idesc_pair(int m, int n) {
 template <class Epi>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_a_lo,
-                const __grid_constant__ CUtensorMap map_w, int M, int N, int K, int split, Epi epi, int* err) {
+                const __grid_constant__ CUtensorMap map_w, int M, int N, int K, int split, Epi epi, int* err, int ksplit,
+                int part_rows) {
   static_assert(Epi::kTmaCols > 0, "the pair kernel has the bulk-store epilogue only");
   using SL = Smem2;
   extern __shared__ uint8_t smem_raw2[];
@@ -104,10 +105,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   const uint32_t rank = cluster_ctarank();  // 0 = leader
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const int tiles_m = (M + 2 * BM - 1) / (2 * BM), tiles_n = (N + BN2 - 1) / BN2;
-  const int num_tiles = tiles_m * tiles_n;
+  // ksplit > 1: every output tile is computed ksplit times, each over its own range of k slabs; slice s stores its
+  // partial tile part_rows * s rows further down and the consumer adds the slices in index order.  Tile index =
+  // (m tile, n tile, slice) with the slice fastest.
+  const int num_tiles = tiles_m * tiles_n * ksplit;
   // split != 0: A is an error-compensated pair (hi + lo).  A stage then holds [A_hi | A_lo | W] of one k slab
   // (48 KB, four stages in the same 192 KB), so the weight slab is fetched once for both products.
-  const int kblocks = (K + BK - 1) / BK;
+  const int kblocks_all = (K + BK - 1) / BK;
+  auto slab_begin = [&](int slice) { return (int)((long long)kblocks_all * slice / ksplit); };
   const uint32_t stage_bytes = split ? (uint32_t)(2 * SL::A_BYTES + SL::B_BYTES) : (uint32_t)SL::STAGE_BYTES;
   const int nstages = split ? 4 : STAGES2;
   const uint32_t w_off = split ? 2u * SL::A_BYTES : (uint32_t)SL::A_BYTES;
@@ -148,13 +153,15 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-        const int m0 = (tile / tiles_n) * (2 * BM) + (int)rank * BM, n0 = (tile % tiles_n) * BN2 + (int)rank * (BN2 / 2);
+        const int mn = tile / ksplit, slice = tile - mn * ksplit;
+        const int m0 = (mn / tiles_n) * (2 * BM) + (int)rank * BM, n0 = (mn % tiles_n) * BN2 + (int)rank * (BN2 / 2);
+        const int kb0 = slab_begin(slice), kblocks = slab_begin(slice + 1) - kb0;
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, err, TFERR_WAIT_EMPTY)) { ok = false; break; }
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * stage_bytes);
           const uint32_t lead_full = map_to_cta(full_bar(stage), 0);
           const uint32_t sa = smem_base + stage * stage_bytes;
-          const int kk = kb * BK;
+          const int kk = (kb0 + kb) * BK;
           tma_load_2d_pair(sa, &map_a, kk, m0, lead_full);
           if (split) tma_load_2d_pair(sa + SL::A_BYTES, &map_a_lo, kk, m0, lead_full);
           tma_load_2d_pair(sa + w_off, &map_w, kk, n0, lead_full);
@@ -176,6 +183,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, err, TFERR_WAIT_TMEM_EMPTY)) { ok = false; break; }
         tcgen05_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN2;
+        const int slice = tile % ksplit;
+        const int kblocks = slab_begin(slice + 1) - slab_begin(slice);
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, err, TFERR_WAIT_FULL)) { ok = false; break; }
           tcgen05_fence_after();
@@ -209,18 +218,19 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     // this thread's bias of the next tile is fetched one tile ahead, so its latency is off the epilogue's path
     float next_bias = 0.f;
     if (pair < num_tiles && etid < BN2) {
-      const int nn = (pair % tiles_n) * BN2 + etid;
+      const int nn = ((pair / ksplit) % tiles_n) * BN2 + etid;
       next_bias = epi.col_const(nn, nn < N);
     }
     for (int tile = pair; tile < num_tiles; tile += num_pairs, ++it) {
-      const int m0 = (tile / tiles_n) * (2 * BM) + (int)rank * BM, n0 = (tile % tiles_n) * BN2;
+      const int mn = tile / ksplit, slice = tile - mn * ksplit;
+      const int m0 = (mn / tiles_n) * (2 * BM) + (int)rank * BM, n0 = (mn % tiles_n) * BN2;
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
       named_bar_sync(1, 32 * NUM_EPI_WARPS);
       if (etid < BN2) tile_bias[etid] = next_bias;
       named_bar_sync(1, 32 * NUM_EPI_WARPS);
       if (tile + num_pairs < num_tiles && etid < BN2) {
-        const int nn = ((tile + num_pairs) % tiles_n) * BN2 + etid;
+        const int nn = (((tile + num_pairs) / ksplit) % tiles_n) * BN2 + etid;
         next_bias = epi.col_const(nn, nn < N);
       }
       if (ok && !mbar_wait(tfull_bar(acc), acc_phase, err, TFERR_WAIT_TMEM_FULL)) ok = false;
@@ -239,7 +249,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll
         for (int g = 0; g < NCH / CPG; ++g) {
           const int cl = (cgroup * NCH + g * CPG) * 32;
-          if (n0 + cl < N) epi.template tma_box<CPG>(v[g * CPG], v[g * CPG + CPG - 1], tile_bias + cl, n0 + cl, row0, box, box_addr, lane);
+          if (n0 + cl < N)
+            epi.template tma_box<CPG>(v[g * CPG], v[g * CPG + CPG - 1], tile_bias + cl, n0 + cl, row0 + slice * part_rows, box, box_addr,
+                                      lane);
         }
       }
     }

@@ -148,7 +148,7 @@ embed_ln_rows_kernel(const float* __restrict__ u, const int* __restrict__ idx, c
   for (int r = 0; r < R; ++r) acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
   if (act) {
     const float4* w4 = reinterpret_cast<const float4*>(w_in_t) + k;
-#pragma unroll 4
+#pragma unroll (R <= 4 ? 16 : 4)
     for (int c = 0; c < D; ++c) {
       const float4 w = __ldg(w4 + (size_t)c * dv);
 #pragma unroll
@@ -289,6 +289,66 @@ __global__ void layernorm_kernel(const float* __restrict__ x, const float* __res
           reinterpret_cast<uint2*>(y_lo + (size_t)warp * d)[k] = w;
         }
       }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Residual add + LayerNorm for sweeps over few rows, where the projection before it left its result as `ksplit`
+// K-slice partial products (slice s of row r at part[(s * part_rows + r) * d]).  One CTA per row, one thread per
+// four columns (blockDim.x = d / 4, a multiple of 32), so that every load of a row is in flight at once:
+//   x[row] <- x[row] + bias + slice 0 + slice 1 + ...   (this order: the sum does not depend on which slice finished first)
+//   y[row] <- LayerNorm(x[row]) (two-pass statistics, eps 1e-5), as T (plus the second term of the pair in y_lo).
+// ------------------------------------------------------------------------------------------------
+template <class T>
+__global__ void __launch_bounds__(1024)
+resid_sum_ln_kernel(float* x, const float* __restrict__ part, int ksplit, int part_rows, const float* __restrict__ rbias,
+                    const float* __restrict__ gamma, const float* __restrict__ beta, T* __restrict__ y,
+                    T* __restrict__ y_lo, int d) {
+  constexpr int MAXS = 8;
+  __shared__ float s_red[2][32];
+  pdl_launch_dependents();
+  const int row = blockIdx.x, k = threadIdx.x, dv = d >> 2;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const float4 g = reinterpret_cast<const float4*>(gamma)[k], bb = reinterpret_cast<const float4*>(beta)[k];
+  const float4 rb = reinterpret_cast<const float4*>(rbias)[k];
+  pdl_wait();
+  float4 a = reinterpret_cast<const float4*>(x)[(size_t)row * dv + k];
+  float4 p[MAXS];
+#pragma unroll
+  for (int s = 0; s < MAXS; ++s)
+    if (s < ksplit) p[s] = reinterpret_cast<const float4*>(part)[((size_t)s * part_rows + row) * dv + k];
+  a.x += rb.x; a.y += rb.y; a.z += rb.z; a.w += rb.w;
+#pragma unroll
+  for (int s = 0; s < MAXS; ++s)
+    if (s < ksplit) { a.x += p[s].x; a.y += p[s].y; a.z += p[s].z; a.w += p[s].w; }
+  reinterpret_cast<float4*>(x)[(size_t)row * dv + k] = a;
+  float v = warp_sum((a.x + a.y) + (a.z + a.w));
+  if (lane == 0) s_red[0][warp] = v;
+  __syncthreads();
+  float tot = 0.f;
+  for (int w = 0; w < nwarps; ++w) tot += s_red[0][w];
+  const float mean = tot / d;
+  const float e0 = a.x - mean, e1 = a.y - mean, e2 = a.z - mean, e3 = a.w - mean;
+  v = warp_sum((e0 * e0 + e1 * e1) + (e2 * e2 + e3 * e3));
+  if (lane == 0) s_red[1][warp] = v;
+  __syncthreads();
+  tot = 0.f;
+  for (int w = 0; w < nwarps; ++w) tot += s_red[1][w];
+  const float rstd = rsqrtf(tot / d + 1e-5f);
+  const float o0 = e0 * rstd * g.x + bb.x, o1 = e1 * rstd * g.y + bb.y, o2 = e2 * rstd * g.z + bb.z, o3 = e3 * rstd * g.w + bb.w;
+  if constexpr (sizeof(T) == 4) {
+    reinterpret_cast<float4*>(y)[(size_t)row * dv + k] = make_float4(o0, o1, o2, o3);
+  } else {
+    __nv_bfloat162 p0 = __floats2bfloat162_rn(o0, o1), p1 = __floats2bfloat162_rn(o2, o3);
+    uint2 w;
+    w.x = *reinterpret_cast<uint32_t*>(&p0); w.y = *reinterpret_cast<uint32_t*>(&p1);
+    reinterpret_cast<uint2*>(y)[(size_t)row * dv + k] = w;
+    if (y_lo != nullptr) {
+      float2 f0 = __bfloat1622float2(p0), f1 = __bfloat1622float2(p1);
+      __nv_bfloat162 q0 = __floats2bfloat162_rn(o0 - f0.x, o1 - f0.y), q1 = __floats2bfloat162_rn(o2 - f1.x, o3 - f1.y);
+      w.x = *reinterpret_cast<uint32_t*>(&q0); w.y = *reinterpret_cast<uint32_t*>(&q1);
+      reinterpret_cast<uint2*>(y_lo)[(size_t)row * dv + k] = w;
     }
   }
 }

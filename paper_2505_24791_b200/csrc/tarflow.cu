@@ -160,7 +160,7 @@ struct tf_model {
   void *xn = nullptr, *qkv = nullptr, *att = nullptr, *mlp = nullptr, *kcache = nullptr, *vcache = nullptr;
   void *xn_lo = nullptr, *qkv_lo = nullptr, *att_lo = nullptr, *mlp_lo = nullptr;  // second terms (bf16 engine)
   CUtensorMap map_xn, map_att, map_mlp, map_xn_lo, map_att_lo, map_mlp_lo;
-  enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_ATT3, SM_ATT3_LO, SM_COUNT };
+  enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_ATT3, SM_ATT3_LO, SM_PART, SM_COUNT };
   CUtensorMap map_qkv3, map_kv3, map_qkv3_lo, map_kv3_lo;  // qkv as [slot][position][3d] for the tensor-core attention (query / key boxes)
   bool use_tc_attention = true;   // single-operand attention on tcgen05 (TARFLOW_ATTN_TC=0: the mma.sync kernel)
   bool use_tc_attention_split = true;  // two-term attention on tcgen05 too (TARFLOW_ATTN_TC_SPLIT=0: mma.sync)
@@ -208,6 +208,11 @@ struct tf_model {
   int seq_kbn_force = 0;     // TARFLOW_SEQ_KBN
   // Jacobi sweeps over few rows are replayed from graphs: one per (block, single-term slots, two-term slots, buffers)
   std::map<std::tuple<int, int, int, const void*, const void*, const void*, const void*>, SeqGraph> sweep_graphs;
+  int small_m_rows = 1024;      // TARFLOW_SMALL_M_ROWS: sweeps of at most this many rows use 128 x 128 single-CTA tiles
+  int split_m_rows = 4096;      // TARFLOW_SPLIT_M_ROWS: up to this many rows the residual projections on pair tiles are cut in K too
+  bool small_m_split = true;    // TARFLOW_SMALL_M_SPLIT=0: the residual projections of such sweeps keep whole-K tiles
+  float* sweep_part = nullptr;  // K-slice partial products of the residual projections of such sweeps [part_cap_rows, d]
+  int part_cap_rows = 0;
   int64_t sweep_graph_rows = 4096;  // TARFLOW_SWEEP_GRAPH_ROWS: largest slots x tokens replayed from a graph (0 = never)
   int seq_variant = 0;       // 0: the block's own token buffers, 1: the compact buffers of the sequential fall-back
   size_t seq_part_row_floats = 0;  // floats of partial tiles available per sample
@@ -369,8 +374,10 @@ static int dev_alloc(tf_model* m, T** p, size_t count) {
 template <int BN, int STAGES, class Epi>
 static int launch_gemm_tc(tf_model* m, int cls, cudaStream_t stream, const CUtensorMap& ma, const CUtensorMap* ma_lo,
                           const CUtensorMap& mw, int M, int N, int K, const Epi& epi, int* err, int num_sms,
-                          int64_t* launches) {
+                          int64_t* launches, int ksplit = 1, int part_rows = 0) {
   using SL = tc::SmemLayout<BN, STAGES>;
+  if (ksplit < 1 || ksplit > (K + tc::BK - 1) / tc::BK || (ksplit > 1 && Epi::kTmaCols == 0))
+    return fail(TF_EINVAL, "gemm_tc_kernel: bad K split %d", ksplit);
   auto kern = tc::gemm_tc_kernel<BN, STAGES, Epi>;
   static bool configured[kMaxDevices] = {false};  // per instantiation and device
   const int dev = current_device();
@@ -379,11 +386,11 @@ static int launch_gemm_tc(tf_model* m, int cls, cudaStream_t stream, const CUten
     CU_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::TOTAL));
     configured[dev] = true;
   }
-  int tiles = ((M + tc::BM - 1) / tc::BM) * ((N + BN - 1) / BN);
+  int tiles = ((M + tc::BM - 1) / tc::BM) * ((N + BN - 1) / BN) * ksplit;
   int grid = tiles < num_sms ? tiles : num_sms;
   if (m) m->pre(cls);
   launch_pdl_raw(stream, kern, dim3(grid), dim3(tc::NUM_THREADS), (size_t)SL::TOTAL, ma, ma_lo ? *ma_lo : ma, mw, M, N, K,
-                 ma_lo ? 1 : 0, epi, err);
+                 ma_lo ? 1 : 0, epi, err, ksplit, part_rows);
   if (m) m->post(cls); else if (launches) ++*launches;
   return check_launch("gemm_tc_kernel");
 }
@@ -391,7 +398,8 @@ static int launch_gemm_tc(tf_model* m, int cls, cudaStream_t stream, const CUten
 // pair kernel: 256 x 256 tiles on clusters of two CTAs (N % 256 == 0, bulk-store epilogues)
 template <class Epi>
 static int launch_gemm_tc2(tf_model* m, int cls, const CUtensorMap& ma, const CUtensorMap* ma_lo, const CUtensorMap& mw, int M,
-                           int N, int K, const Epi& epi) {
+                           int N, int K, const Epi& epi, int ksplit = 1, int part_rows = 0) {
+  if (ksplit < 1 || ksplit > (K + tc::BK - 1) / tc::BK) return fail(TF_EINVAL, "gemm_tc2_kernel: bad K split %d", ksplit);
   auto kern = tc2::gemm_tc2_kernel<Epi>;
   static bool configured[kMaxDevices] = {false};  // per instantiation and device
   const int dev = current_device();
@@ -400,7 +408,7 @@ static int launch_gemm_tc2(tf_model* m, int cls, const CUtensorMap& ma, const CU
     CU_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::Smem2::TOTAL));
     configured[dev] = true;
   }
-  const int tiles = ((M + 2 * tc::BM - 1) / (2 * tc::BM)) * (N / tc2::BN2);
+  const int tiles = ((M + 2 * tc::BM - 1) / (2 * tc::BM)) * (N / tc2::BN2) * ksplit;
   int pairs = m->num_sms / 2;
   if (tiles < pairs) pairs = tiles;
   cudaLaunchConfig_t lc = {};
@@ -418,7 +426,7 @@ static int launch_gemm_tc2(tf_model* m, int cls, const CUtensorMap& ma, const CU
   lc.attrs = at;
   lc.numAttrs = 2;
   m->pre(cls);
-  cudaError_t e = cudaLaunchKernelEx(&lc, kern, ma, ma_lo ? *ma_lo : ma, mw, M, N, K, ma_lo ? 1 : 0, epi, m->err);
+  cudaError_t e = cudaLaunchKernelEx(&lc, kern, ma, ma_lo ? *ma_lo : ma, mw, M, N, K, ma_lo ? 1 : 0, epi, m->err, ksplit, part_rows);
   m->post(cls);
   if (e != cudaSuccess) return fail(TF_ECUDA, "gemm_tc2_kernel launch failed: %s", cudaGetErrorString(e));
   return TF_OK;
@@ -435,12 +443,18 @@ static int launch_gemm_simt(tf_model* m, int cls, const T* A, const Matrix& W, i
 // two-term pair); fp32 engine: SIMT kernel.
 template <class T, class Epi>
 static int gemm(tf_model* m, int cls, const T* A, const CUtensorMap* map_a, const CUtensorMap* map_a_lo,
-                const Matrix& W, int M, const Epi& epi) {
+                const Matrix& W, int M, const Epi& epi, int ksplit = 1, int part_rows = 0) {
   if constexpr (sizeof(T) == 2) {
     if constexpr (Epi::kTmaCols > 0) {
+      // few rows: 128 x 128 tiles on single CTAs put four times as many SMs on the weights as 256 x 256 pair tiles,
+      // and K slices (ksplit > 1: partial products, added by the consumer) fill the rest of the GPU
+      if (M <= m->small_m_rows && W.N % 128 == 0)
+        return launch_gemm_tc<128, 6, Epi>(m, cls, m->stream, *map_a, map_a_lo, W.map_seq, M, W.N, W.K, epi, m->err,
+                                           m->num_sms, nullptr, ksplit, part_rows);
       if (m->use_pair_gemm && W.N % 256 == 0 && M >= 256)
-        return launch_gemm_tc2<Epi>(m, cls, *map_a, map_a_lo, W.map_seq, M, W.N, W.K, epi);
+        return launch_gemm_tc2<Epi>(m, cls, *map_a, map_a_lo, W.map_seq, M, W.N, W.K, epi, ksplit, part_rows);
     }
+    if (ksplit > 1) return fail(TF_EINVAL, "no K-split kernel for this shape");
     if (W.bn == 256)
       return launch_gemm_tc<256, 4, Epi>(m, cls, m->stream, *map_a, map_a_lo, W.map, M, W.N, W.K, epi, m->err,
                                          m->num_sms, nullptr);
@@ -454,9 +468,22 @@ static int gemm(tf_model* m, int cls, const T* A, const CUtensorMap* map_a, cons
 // ------------------------------------------------------------------------------------------------
 // one causal pass over n_slots * L rows (a Jacobi sweep, or the forward direction)
 // ------------------------------------------------------------------------------------------------
+// A projection into the residual stream that was left as K-slice partial products: the LayerNorm after it adds them.
+struct SplitSum {
+  const float* part;
+  int ksplit, part_rows;
+  const float* bias;
+};
+
 template <class T>
-static int layernorm(tf_model* m, int cls, const float* x, const float* g, const float* b, T* y, T* y_lo, int rows) {
+static int layernorm(tf_model* m, int cls, const float* x, const float* g, const float* b, T* y, T* y_lo, int rows,
+                     const SplitSum* ss = nullptr) {
   int d = m->d;
+  if (ss != nullptr) {  // d % 128 == 0 and d <= 4096 on this path
+    LAUNCH_PDL(m, cls, resid_sum_ln_kernel<T>, rows, d / 4, 0, const_cast<float*>(x), ss->part, ss->ksplit, ss->part_rows, ss->bias,
+               g, b, y, y_lo, d);
+    return check_launch("resid_sum_ln_kernel");
+  }
   int blocks = (rows * 32 + 255) / 256;
   if (d <= 128 * 1) LAUNCH_PDL(m, cls, (layernorm_kernel<T, 1>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
   else if (d <= 128 * 4) LAUNCH_PDL(m, cls, (layernorm_kernel<T, 4>), blocks, 256, 0, x, g, b, y, y_lo, rows, d);
@@ -490,16 +517,39 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
   const bool fused_embed = d % 4 == 0 && d <= 1024 && (size_t)16 * D * sizeof(float) <= 40 * 1024;
   if (fused_embed) {
     const LayerW& l0 = bw.layers[0];
-    LAUNCH_PDL(m, KC_EMBED, (embed_ln_rows_kernel<T, 16>), (M + 15) / 16, ((d / 4 + 31) / 32) * 32, 16 * D * sizeof(float), u_src,
-               idx, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, l0.ln1_g, l0.ln1_b, xn, xn_lo, L, D, d, rev, M);
+    if (M <= m->small_m_rows)  // few rows: four per CTA instead of sixteen, for four times the CTAs
+      LAUNCH_PDL(m, KC_EMBED, (embed_ln_rows_kernel<T, 4>), (M + 3) / 4, ((d / 4 + 31) / 32) * 32, 4 * D * sizeof(float), u_src,
+                 idx, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, l0.ln1_g, l0.ln1_b, xn, xn_lo, L, D, d, rev, M);
+    else
+      LAUNCH_PDL(m, KC_EMBED, (embed_ln_rows_kernel<T, 16>), (M + 15) / 16, ((d / 4 + 31) / 32) * 32, 16 * D * sizeof(float), u_src,
+                 idx, labels, bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, l0.ln1_g, l0.ln1_b, xn, xn_lo, L, D, d, rev, M);
   } else {
     LAUNCH_PDL(m, KC_EMBED, embed_rows_kernel<16>, (M + 15) / 16, ethreads, 16 * D * sizeof(float), u_src, idx, labels,
                bw.w_in_t, bw.b_in, bw.pos, bw.cls, m->h, L, D, d, rev, M);
   }
   TF_TRY(check_launch("embed_kernel"));
+  // Few rows (bf16 engine): the two projections into the residual stream have d / 128 column tiles per 128 rows, too few
+  // CTAs to stream their weights, so they are cut into K slices that leave partial products; the LayerNorm that follows
+  // (this layer's second, the next layer's first, or the block's last) adds them to the stream in slice order.
+  const int m_pad = (M + 127) / 128 * 128;
+  auto slices_for = [&](int K) -> int {
+    if (sizeof(T) != 2 || m->sweep_part == nullptr || !m->small_m_split || d > 4096) return 1;
+    int ks;
+    if (M <= m->small_m_rows) ks = m->num_sms / ((m_pad / 128) * (d / 128));  // 128 x 128 tiles
+    else if (M <= m->split_m_rows && m->use_pair_gemm && d % 256 == 0 && M >= 256)
+      ks = (m->num_sms / 2) / (((M + 255) / 256) * (d / 256));                // pair tiles
+    else return 1;
+    if (ks > K / (2 * tc::BK)) ks = K / (2 * tc::BK);  // at least two k slabs per slice
+    if (ks > 8) ks = 8;
+    if (ks > m->part_cap_rows / m_pad) ks = m->part_cap_rows / m_pad;
+    return ks < 1 ? 1 : ks;
+  };
+  SplitSum pend{nullptr, 0, 0, nullptr};
+  bool has_pend = false;
   bool first_layer = true;
   for (const LayerW& lw : bw.layers) {
-    if (!(first_layer && fused_embed)) TF_TRY(layernorm<T>(m, KC_LN, m->h, lw.ln1_g, lw.ln1_b, xn, xn_lo, M));
+    if (!(first_layer && fused_embed)) TF_TRY(layernorm<T>(m, KC_LN, m->h, lw.ln1_g, lw.ln1_b, xn, xn_lo, M, has_pend ? &pend : nullptr));
+    has_pend = false;
     first_layer = false;
     if constexpr (sizeof(T) == 2) {
       const CUtensorMap* sm = m->store_maps;
@@ -534,22 +584,39 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
              1.0f / sqrtf((float)m->hd));
     }
     TF_TRY(check_launch("attention kernel"));
-    if constexpr (sizeof(T) == 2)
-      TF_TRY(gemm<T>(m, KC_GEMM_O, att, &m->map_att, mal, lw.w_o, M, EpiResidTma{lw.b_o, m->store_maps + tf_model::SM_H}));
-    else
+    if constexpr (sizeof(T) == 2) {
+      const int ks = slices_for(d);
+      if (ks > 1) {
+        TF_TRY(gemm<T>(m, KC_GEMM_O, att, &m->map_att, mal, lw.w_o, M, EpiStoreF32Tma{nullptr, m->store_maps + tf_model::SM_PART},
+                       ks, m_pad));
+        pend = SplitSum{m->sweep_part, ks, m_pad, lw.b_o};
+        has_pend = true;
+      } else {
+        TF_TRY(gemm<T>(m, KC_GEMM_O, att, &m->map_att, mal, lw.w_o, M, EpiResidTma{lw.b_o, m->store_maps + tf_model::SM_H}));
+      }
+    } else {
       TF_TRY(gemm<T>(m, KC_GEMM_O, att, &m->map_att, mal, lw.w_o, M, EpiResid{m->h, lw.b_o, d}));
-    TF_TRY(layernorm<T>(m, KC_LN, m->h, lw.ln2_g, lw.ln2_b, xn, xn_lo, M));
+    }
+    TF_TRY(layernorm<T>(m, KC_LN, m->h, lw.ln2_g, lw.ln2_b, xn, xn_lo, M, has_pend ? &pend : nullptr));
+    has_pend = false;
     if constexpr (sizeof(T) == 2) {
       const CUtensorMap* sm = m->store_maps;
       TF_TRY(gemm<T>(m, KC_GEMM_MLP1, xn, &m->map_xn, mxl, lw.w_1, M,
                      EpiStoreTma<true>{lw.b_1, sm + tf_model::SM_MLP, hp ? sm + tf_model::SM_MLP_LO : nullptr}));
-      TF_TRY(gemm<T>(m, KC_GEMM_MLP2, mlp, &m->map_mlp, mml, lw.w_2, M, EpiResidTma{lw.b_2, sm + tf_model::SM_H}));
+      const int ks = slices_for(m->hid);
+      if (ks > 1) {
+        TF_TRY(gemm<T>(m, KC_GEMM_MLP2, mlp, &m->map_mlp, mml, lw.w_2, M, EpiStoreF32Tma{nullptr, sm + tf_model::SM_PART}, ks, m_pad));
+        pend = SplitSum{m->sweep_part, ks, m_pad, lw.b_2};
+        has_pend = true;
+      } else {
+        TF_TRY(gemm<T>(m, KC_GEMM_MLP2, mlp, &m->map_mlp, mml, lw.w_2, M, EpiResidTma{lw.b_2, sm + tf_model::SM_H}));
+      }
     } else {
       TF_TRY(gemm<T>(m, KC_GEMM_MLP1, xn, &m->map_xn, mxl, lw.w_1, M, EpiStore<T, true>{mlp, lw.b_1, m->hid, mlp_lo}));
       TF_TRY(gemm<T>(m, KC_GEMM_MLP2, mlp, &m->map_mlp, mml, lw.w_2, M, EpiResid{m->h, lw.b_2, d}));
     }
   }
-  TF_TRY(layernorm<T>(m, KC_LN, m->h, bw.lnf_g, bw.lnf_b, xn, xn_lo, M));
+  TF_TRY(layernorm<T>(m, KC_LN, m->h, bw.lnf_g, bw.lnf_b, xn, xn_lo, M, has_pend ? &pend : nullptr));
   if (mode == PASS_JACOBI) {
     EpiHeadUpdate epi{v, u_upd, m->maxdiff, idx, bw.b_out, L, D, rev};
     TF_TRY(gemm<T>(m, KC_GEMM_HEAD_UPDATE, xn, &m->map_xn, mxl, bw.w_out, M, epi));
@@ -1538,6 +1605,16 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
       TF_TRY(make_map_store(&sm[tf_model::SM_MLP], m->mlp, M, hid, 2));
       TF_TRY(make_map_store(&sm[tf_model::SM_MLP_LO], m->mlp_lo, M, hid, 2));
       TF_TRY(make_map_store(&sm[tf_model::SM_H], m->h, M, d, 4));
+      if (const char* e = getenv("TARFLOW_SMALL_M_ROWS")) m->small_m_rows = atoi(e);
+      if (const char* e = getenv("TARFLOW_SPLIT_M_ROWS")) m->split_m_rows = atoi(e);
+      if (const char* e = getenv("TARFLOW_SMALL_M_SPLIT")) m->small_m_split = atoi(e) != 0;
+      if ((m->small_m_rows > 0 || m->split_m_rows > 0) && d % 128 == 0) {
+        m->part_cap_rows = 8192;
+        TF_TRY(dev_alloc(m, &m->sweep_part, (size_t)m->part_cap_rows * d));
+        TF_TRY(make_map_store(&sm[tf_model::SM_PART], m->sweep_part, (uint64_t)m->part_cap_rows, d, 4));
+      } else {
+        sm[tf_model::SM_PART] = sm[tf_model::SM_H];
+      }
       TF_TRY(make_map_3d(&sm[tf_model::SM_ATT3], m->att, B, L, d, 32));
       TF_TRY(make_map_3d(&m->map_qkv3, m->qkv, B, L, 3 * (uint64_t)d, attn_tc::BQ));
       TF_TRY(make_map_3d(&m->map_kv3, m->qkv, B, L, 3 * (uint64_t)d, attn_tc::BKV));
@@ -1896,6 +1973,7 @@ int tf_maf_load(const tf_maf_config* cfg, const void* weights_host, size_t nbyte
   tf_model* m = new (std::nothrow) tf_model();
   if (!m) return fail(TF_ENOMEM, "host allocation failed");
   m->is_maf = true;
+  m->small_m_rows = m->split_m_rows = 0;  // the MLP flow keeps one tile shape from 256 rows up: results do not depend on the batch
   m->cfg = tf_config{1, cfg->D, 1, 1, cfg->n_blocks, 2, cfg->hidden, 1, 1, 0, cfg->dtype, cfg->max_batch};
   m->L = cfg->D;  // D values per sample, token dimension 1
   m->D = 1;
