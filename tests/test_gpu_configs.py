@@ -227,3 +227,36 @@ def test_long_sequence_full_size_properties():
         assert rel_l2(zr, z.astype(np.float64)) <= BF16_REL_L2 and np.abs(zr - z).max() <= 0.15
         xs = m.inverse_sequential(z[:4], None)
         assert rel_l2(x[:4], xs) <= 5e-3 and np.abs(x[:4] - xs).max() <= 5e-2
+
+
+# ---------------------------------------------------------------- sweeps over few rows (K-split residual projections)
+@pytest.mark.parametrize("name", ["cfg2", "cfg3"])
+def test_few_row_sweeps_agree_with_the_one_shape_path_and_the_oracle(name, monkeypatch):
+    """Sweeps of up to 1024 rows run on 128 x 128 tiles with the residual projections cut into K slices that the next
+    LayerNorm adds; up to 4096 rows the pair tiles are cut.  Batches 1 (256 rows, 8 slices at width 1024 / 4 at 512),
+    3 (768 rows), 5 (1280 rows: pair tiles, 3 to 6 slices) and 8 (2048 rows) against the oracle, and against
+    the same library with both paths switched off (every sweep on one tile shape, reduce-add epilogue).  The forward
+    direction takes the same path."""
+    cfg = synth.config(name, n_blocks=2, n_layers=2)
+    L = synth.seq_len(cfg)
+    lab_of = (lambda B: synth.make_labels(cfg, B=B)) if cfg.get("n_classes", 0) else (lambda B: None)
+    with Model(cfg, max_batch=8) as m:
+        monkeypatch.setenv("TARFLOW_SMALL_M_ROWS", "0")
+        monkeypatch.setenv("TARFLOW_SPLIT_M_ROWS", "0")
+        with Model(cfg, max_batch=8) as ref:
+            for B in (1, 3, 5, 8):
+                z = synth.make_latents(cfg, 5200 + B, B=B)
+                lab = lab_of(B)
+                x, ib, its, rc = m.inverse(z, lab, [1, 1], 1e-3, L + 1)
+                xr, ibr, itsr, rcr = ref.inverse(z, lab, [1, 1], 1e-3, L + 1)
+                assert rc == 0 and rcr == 0 and np.isfinite(x).all()
+                assert np.abs(x - xr).max() <= 2e-3 and np.abs(its - itsr).max() <= 1
+                x2, _, its2, _ = m.inverse(z, lab, [1, 1], 1e-3, L + 1)          # fixed summation order: run-to-run identical
+                assert np.array_equal(x, x2) and np.array_equal(its, its2)
+                pick = [B - 1]
+                xo, ito = O.model_inverse(m.blocks, z[pick], None if lab is None else lab[pick], cfg, [1, 1], 1e-3, L + 1)
+                _close(x[pick], xo)
+                assert np.abs(its[:, pick] - ito).max() <= 1
+                zf, ld = m.forward(xo, None if lab is None else lab[pick])
+                zo, ldo = O.model_forward(m.blocks, xo, None if lab is None else lab[pick], cfg)
+                assert rel_l2(zf, zo) <= 2e-2 and np.abs(ld - ldo).max() <= 2e-2 * max(1.0, np.abs(ldo).max())
