@@ -277,6 +277,27 @@ def test_bf16_ragged_sequence_length_and_classes():
     assert rc == 0 and bf16_close(x, xo) and np.abs(its - ito).max() <= 1
 
 
+def test_bf16_ragged_rows_on_k_split_pair_tiles():
+    """L = 81 tokens, 20 samples: 1620 rows = six 256-row pair tiles and a ragged seventh (84 rows, its second CTA
+    empty), the residual projections cut into K slices whose partial tiles the next LayerNorm adds; as samples
+    converge the row count passes through further ragged sizes down to the 128-row tiles.  All-Jacobi, tau 1e-3;
+    three samples against the oracle, the forward direction on the same shapes."""
+    cfg = synth.config("cfg3", H=36, W=36, n_blocks=2, n_layers=2, width=256, n_heads=4, n_classes=10)
+    B = 20
+    lab = synth.make_labels(cfg, B=B)
+    with Model(cfg, max_batch=B) as m:
+        z = synth.make_latents(cfg, 77, B=B)
+        x, ib, its, rc = m.inverse(z, lab, [1, 1], 1e-3, m.L + 1)
+        assert rc == 0 and np.isfinite(x).all() and np.array_equal(ib, its.max(axis=1))
+        pick = [0, 9, B - 1]
+        xo, ito = O.model_inverse(m.blocks, z[pick], lab[pick], cfg, [1, 1], 1e-3, m.L + 1)
+        assert bf16_close(x[pick], xo) and np.abs(its[:, pick] - ito).max() <= 1
+        zf, ld = m.forward(x, lab)
+        zo, ldo = O.model_forward(m.blocks, x[pick], lab[pick], cfg)
+        assert bf16_close(zf[pick], zo)
+        assert np.abs(ld[pick] - ldo).max() <= 2e-2 * max(np.abs(ldo).max(), np.sqrt(m.L * synth.token_dim(cfg)) * 0.1)
+
+
 def test_bf16_optional_kernel_paths_agree(monkeypatch):
     """The mma.sync attention and the one-CTA-per-tile GEMM give the same sweep as the default kernels."""
     cfg = synth.config("cfg2", n_blocks=1, n_layers=2)
