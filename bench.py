@@ -350,11 +350,11 @@ def main():
                          "'seq' = one sequentially decoded block; run twice, the second call timed; not a bench value")
     ap.add_argument("--sweeps", type=int, default=2)
     ap.add_argument("--launch-list", action="store_true",
-                    help="for an ncu launch-list capture: one warm-up and one step of the timed leg only; the line it "
+                    help="for an ncu launch-list capture: one warm-up (none with --warmup 0) and one step of the timed leg only; the line it "
                          "prints is marked as a profiling run and is not a bench value")
     args = ap.parse_args()
     if args.launch_list:
-        args.warmup, args.steps, args.no_cpu, args.no_policies, args.no_legs = 1, 1, True, True, True
+        args.warmup, args.steps, args.no_cpu, args.no_policies, args.no_legs = min(args.warmup, 1), 1, True, True, True
     elif args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
 

@@ -43,7 +43,8 @@
  *     the next projection normalise its own operand slice, five kernels per layer instead of eight (measured slower
  *     than the default chain), TARFLOW_SEQ_KBN8=0 keeps such launches at four k slabs per CTA;
  *     TARFLOW_SWEEP_GRAPH_ROWS=n replays Jacobi sweeps of at most n rows (slots x tokens, default 4096) from CUDA
- *     graphs, 0 launches every kernel directly.  TARFLOW_SMALL_M_ROWS=n (default 1024): sweeps of at most n rows run
+ *     graphs, 0 launches every kernel directly; TARFLOW_GRAPHS=0 replays nothing from graphs, the decoding steps of a
+ *     sequential block included (same kernels in the same order, for tools that list launches).  TARFLOW_SMALL_M_ROWS=n (default 1024): sweeps of at most n rows run
  *     their projections on 128 x 128 single-CTA tiles; TARFLOW_SPLIT_M_ROWS=n (default 4096): up to n rows the two
  *     projections into the residual stream are cut into K slices whose partial products the next LayerNorm adds in
  *     slice order (TARFLOW_SMALL_M_SPLIT=0: never); 0 for both keeps one tile shape for every sweep.  These paths

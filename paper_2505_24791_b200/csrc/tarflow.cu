@@ -1670,6 +1670,7 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
     CU_OK(cudaMemset(m->seq_tickets, 0, (size_t)tf_model::MAX_CHAINS * tf_model::SEQ_TICKETS * sizeof(int)));
     TF_TRY(dev_alloc(m, &m->seq_stats, (size_t)tf_model::MAX_CHAINS * 16 * B));
     if (const char* e = getenv("TARFLOW_SWEEP_GRAPH_ROWS")) m->sweep_graph_rows = atoll(e);
+    if (const char* e = getenv("TARFLOW_GRAPHS")) m->use_graphs = atoi(e) != 0;
   }
   CU_OK(cudaDeviceSynchronize());
   return TF_OK;
