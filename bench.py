@@ -47,7 +47,7 @@ L2_BYTES = 126e6
 # (profiles/gemm_tc2_kernel_cfg3_sweep.md: one single-term launch over the full batch of 16 384 rows; the live class
 # also holds two-term launches and launches over fewer rows); None = no capture of the current kernel.
 # {workload: {class: bytes}}
-NCU_TRAFFIC: dict = {"cfg3": {"gemm_qkv": 89.4e6, "gemm_out": 112.5e6, "gemm_mlp_up": 123.4e6, "gemm_mlp_down": 255.1e6}}
+NCU_TRAFFIC: dict = {"cfg3": {"gemm_qkv": 89.9e6, "gemm_out": 111.9e6, "gemm_mlp_up": 124.5e6, "gemm_mlp_down": 253.9e6}}
 
 
 def peaks():
