@@ -538,6 +538,45 @@ __global__ void jacobi_update_kernel(const float* __restrict__ o, const float* _
   }
 }
 
+// Jacobi update of sweeps over few rows, where the head projection left its result as `ksplit` K-slice partial
+// products (slice s of row r at part[(s * part_rows + r) * npad], columns interleaved (mu~_c, alpha~_c), npad >= 2D):
+// head = bias + slice 0 + slice 1 + ... (this order), then Algorithm 1's update line as in the fused epilogue: row
+// (slot s, position l) updates token l + 1 of sample idx[s], the last position's row copies token 0.  One warp per
+// row; per-row max|du| merged with the order-independent atomic max (NaN propagates).
+__global__ void __launch_bounds__(256)
+jacobi_update_split_kernel(const float* __restrict__ part, int ksplit, int part_rows, int npad, const float* __restrict__ bias,
+                           const float* __restrict__ v, float* __restrict__ u, float* __restrict__ maxdiff,
+                           const int* __restrict__ idx, int n_rows, int L, int D, int reversed) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (row >= n_rows) return;
+  const int s = row / L, l = row - s * L;
+  const int b = idx ? idx[s] : s;
+  const bool upd = l < L - 1;
+  const size_t e0 = ((size_t)b * L + tok_index(upd ? l + 1 : 0, L, reversed)) * D;
+  float df = 0.f;
+  for (int c = lane; c < D; c += 32) {
+    float2 o = *reinterpret_cast<const float2*>(bias + 2 * c);
+    for (int k = 0; k < ksplit; ++k) {
+      const float2 p = __ldcg(reinterpret_cast<const float2*>(part + ((size_t)k * part_rows + row) * npad + 2 * c));
+      o.x += p.x;
+      o.y += p.y;
+    }
+    const float old = u[e0 + c], vv = v[e0 + c];
+    const float nw = upd ? fmaf(vv, expf(o.y), o.x) : vv;
+    u[e0 + c] = nw;
+    const float dd = fabsf(nw - old);
+    df = (dd > df || dd != dd) ? dd : df;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float other = __shfl_xor_sync(0xffffffffu, df, o);
+    df = (other > df || other != other) ? other : df;
+  }
+  if (lane == 0) atomic_max_nonneg(maxdiff + b, df);
+}
+
 // Sequential decoding: token t+1 of every sample from the head output of token t (Eq. 5).
 // o: [B, 2D] interleaved.
 __global__ void seq_update_kernel(const float* __restrict__ o, const float* __restrict__ v, float* __restrict__ u,

@@ -160,7 +160,7 @@ struct tf_model {
   void *xn = nullptr, *qkv = nullptr, *att = nullptr, *mlp = nullptr, *kcache = nullptr, *vcache = nullptr;
   void *xn_lo = nullptr, *qkv_lo = nullptr, *att_lo = nullptr, *mlp_lo = nullptr;  // second terms (bf16 engine)
   CUtensorMap map_xn, map_att, map_mlp, map_xn_lo, map_att_lo, map_mlp_lo;
-  enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_ATT3, SM_ATT3_LO, SM_PART, SM_COUNT };
+  enum { SM_QKV, SM_QKV_LO, SM_MLP, SM_MLP_LO, SM_H, SM_ATT3, SM_ATT3_LO, SM_PART, SM_PART_HEAD, SM_COUNT };
   CUtensorMap map_qkv3, map_kv3, map_qkv3_lo, map_kv3_lo;  // qkv as [slot][position][3d] for the tensor-core attention (query / key boxes)
   bool use_tc_attention = true;   // single-operand attention on tcgen05 (TARFLOW_ATTN_TC=0: the mma.sync kernel)
   bool use_tc_attention_split = true;  // two-term attention on tcgen05 too (TARFLOW_ATTN_TC_SPLIT=0: mma.sync)
@@ -213,6 +213,7 @@ struct tf_model {
   bool small_m_split = true;    // TARFLOW_SMALL_M_SPLIT=0: the residual projections of such sweeps keep whole-K tiles
   float* sweep_part = nullptr;  // K-slice partial products of the residual projections of such sweeps [part_cap_rows, d]
   int part_cap_rows = 0;
+  int part_head_npad = 0, part_head_rows = 0;  // the same buffer seen as [part_head_rows, part_head_npad] for the head's slices
   int64_t sweep_graph_rows = 4096;  // TARFLOW_SWEEP_GRAPH_ROWS: largest slots x tokens replayed from a graph (0 = never)
   int seq_variant = 0;       // 0: the block's own token buffers, 1: the compact buffers of the sequential fall-back
   size_t seq_part_row_floats = 0;  // floats of partial tiles available per sample
@@ -618,8 +619,31 @@ static int run_pass(tf_model* m, int g, int n_slots, const float* u_src, const i
   }
   TF_TRY(layernorm<T>(m, KC_LN, m->h, bw.lnf_g, bw.lnf_b, xn, xn_lo, M, has_pend ? &pend : nullptr));
   if (mode == PASS_JACOBI) {
-    EpiHeadUpdate epi{v, u_upd, m->maxdiff, idx, bw.b_out, L, D, rev};
-    TF_TRY(gemm<T>(m, KC_GEMM_HEAD_UPDATE, xn, &m->map_xn, mxl, bw.w_out, M, epi));
+    // few rows: the head projection has one or two CTAs that walk K alone, so it is cut into K slices too and a small
+    // kernel adds them and applies the update (otherwise the update is the projection's epilogue)
+    int ks_head = 1;
+    if constexpr (sizeof(T) == 2) {
+      if (M <= m->small_m_rows && m->sweep_part != nullptr && m->small_m_split && bw.w_out.bn == 128 && D % 2 == 0 && d % 128 == 0) {
+        ks_head = m->num_sms / ((m_pad / 128) * ((2 * D + 127) / 128));
+        if (ks_head > d / (2 * tc::BK)) ks_head = d / (2 * tc::BK);
+        if (ks_head > 8) ks_head = 8;
+        if (ks_head > m->part_head_rows / m_pad) ks_head = m->part_head_rows / m_pad;
+        if (ks_head < 1) ks_head = 1;
+      }
+    }
+    if (ks_head > 1) {
+      if constexpr (sizeof(T) == 2) {
+        TF_TRY((launch_gemm_tc<128, 6, EpiStoreF32Tma>(m, KC_GEMM_HEAD_UPDATE, m->stream, m->map_xn, mxl, bw.w_out.map, M, 2 * D, d,
+                                                       EpiStoreF32Tma{nullptr, m->store_maps + tf_model::SM_PART_HEAD}, m->err,
+                                                       m->num_sms, nullptr, ks_head, m_pad)));
+        LAUNCH_PDL(m, KC_GEMM_HEAD_UPDATE, jacobi_update_split_kernel, (M * 32 + 255) / 256, 256, 0, m->sweep_part, ks_head, m_pad,
+                   m->part_head_npad, bw.b_out, v, u_upd, m->maxdiff, idx, M, L, D, rev);
+        TF_TRY(check_launch("jacobi_update_split_kernel"));
+      }
+    } else {
+      EpiHeadUpdate epi{v, u_upd, m->maxdiff, idx, bw.b_out, L, D, rev};
+      TF_TRY(gemm<T>(m, KC_GEMM_HEAD_UPDATE, xn, &m->map_xn, mxl, bw.w_out, M, epi));
+    }
   } else {
     TF_TRY(gemm<T>(m, KC_GEMM_HEAD, xn, &m->map_xn, mxl, bw.w_out, M, EpiStore<float, false>{m->o, bw.b_out, 2 * D}));
   }
@@ -1612,8 +1636,12 @@ static int load_impl(tf_model* m, const void* blob, size_t nbytes) {
         m->part_cap_rows = 8192;
         TF_TRY(dev_alloc(m, &m->sweep_part, (size_t)m->part_cap_rows * d));
         TF_TRY(make_map_store(&sm[tf_model::SM_PART], m->sweep_part, (uint64_t)m->part_cap_rows, d, 4));
+        m->part_head_npad = (2 * m->D + 31) / 32 * 32;
+        m->part_head_rows = (int)((size_t)m->part_cap_rows * d / m->part_head_npad);
+        TF_TRY(make_map_store(&sm[tf_model::SM_PART_HEAD], m->sweep_part, (uint64_t)m->part_head_rows, m->part_head_npad, 4));
       } else {
         sm[tf_model::SM_PART] = sm[tf_model::SM_H];
+        sm[tf_model::SM_PART_HEAD] = sm[tf_model::SM_H];
       }
       TF_TRY(make_map_3d(&sm[tf_model::SM_ATT3], m->att, B, L, d, 32));
       TF_TRY(make_map_3d(&m->map_qkv3, m->qkv, B, L, 3 * (uint64_t)d, attn_tc::BQ));
